@@ -1,0 +1,272 @@
+"""Python face of the CPU oracle (TEST INFRASTRUCTURE ONLY).
+
+Thin ctypes wrappers over `it_oracle.c` plus the layer-by-layer driver that strings
+them together the way the paper does: k layers = k passes over every vertex, each
+vertex used once per layer, no sampling (Section "Alternative Backends and
+Implementation Details", Execution: "after k iterations we get the result of a k-layer
+model").  Nothing here is shared with, or imported by, the CUDA library.
+
+Storage points.  The method itself is exact, but a deployment stores layer inputs and
+outputs in a narrow type.  `storage=None` keeps everything in fp64 (mode A).  With
+`storage='f32'|'bf16'` (mode B) the oracle still accumulates in fp64 but rounds to the
+storage type (nearest even) at the points where the layer contract says a tensor is
+stored: the aggregate handed to apply, the transformed rows Z (GAT and
+transform-before-aggregate) and the layer output.  The self term of a reordered layer
+and the GAT scores are contract-fp32 and are rounded to fp32.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libit_oracle.so")
+_SRC = os.path.join(_HERE, "it_oracle.c")
+
+OPS = {"sum": 0, "mean": 1, "max": 2}
+ACTS = {"none": 0, "relu": 1, "elu": 2}
+
+
+def build(force: bool = False) -> str:
+    """Compile it_oracle.c into libit_oracle.so next to it (gcc, OpenMP)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99",
+                               "-o", _SO, _SRC, "-lm"])
+    return _SO
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.ito_split_count.restype = C.c_int64
+        _lib.ito_buckets.restype = C.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f64(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+# ----------------------------------------------------------------- rounding helpers
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """fp64 -> nearest bfloat16 (ties to even), returned as fp64.  Done directly on the
+    fp64 bit pattern (keep 7 fraction bits) for values in bfloat16's normal range; tiny
+    values go through fp32 first so subnormals and underflow behave like hardware."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    u = x.view(np.uint64)
+    drop = np.uint64(52 - 7)
+    lsb = (u >> drop) & np.uint64(1)
+    r = (u + ((np.uint64(1) << (drop - np.uint64(1))) - np.uint64(1)) + lsb) >> drop << drop
+    out = r.view(np.float64).copy()
+    small = np.abs(x) < 2.0 ** -120
+    if small.any():
+        f = x[small].astype(np.float32)
+        b = f.view(np.uint32)
+        b = ((b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)) << np.uint32(16)
+        out[small] = b.view(np.float32).astype(np.float64)
+    big = np.abs(out) > 3.3895313892515355e38  # bfloat16 max
+    out[big] = np.sign(out[big]) * np.inf
+    out[np.isnan(x)] = np.nan
+    return out
+
+
+def round_f32(x: np.ndarray) -> np.ndarray:
+    return np.asarray(x, dtype=np.float64).astype(np.float32).astype(np.float64)
+
+
+def round_to(x: np.ndarray, storage: str | None) -> np.ndarray:
+    if storage is None:
+        return x
+    if storage == "f32":
+        return round_f32(x)
+    if storage == "bf16":
+        return round_bf16(x)
+    raise ValueError(storage)
+
+
+# ----------------------------------------------------------------- index side
+
+def split_hubs(indptr, threshold: int):
+    """Shadow rows of every vertex: (shadow_indptr int64[R+1], shadow_owner int32[R],
+    owner_indptr int64[n+1])."""
+    indptr = _i64(indptr)
+    n = indptr.shape[0] - 1
+    R = lib().ito_split_count(C.c_int64(n), _p(indptr), C.c_int64(threshold))
+    sp = np.empty(R + 1, np.int64)
+    so = np.empty(R, np.int32)
+    op = np.empty(n + 1, np.int64)
+    lib().ito_split_hubs(C.c_int64(n), _p(indptr), C.c_int64(threshold), _p(sp), _p(so), _p(op))
+    return sp, so, op
+
+
+def buckets(shadow_indptr, bounds):
+    """Stable partition of shadow rows by length class: (bucket_offsets int64[nb+1],
+    bucket_rows int32[R])."""
+    sp = _i64(shadow_indptr)
+    bounds = _i64(bounds)
+    R = sp.shape[0] - 1
+    off = np.empty(bounds.shape[0] + 1, np.int64)
+    rows = np.empty(R, np.int32)
+    rc = lib().ito_buckets(C.c_int64(R), _p(sp), C.c_int32(bounds.shape[0]), _p(bounds), _p(off), _p(rows))
+    if rc != 0:
+        raise ValueError("a row is longer than the last bucket bound")
+    return off, rows
+
+
+# ----------------------------------------------------------------- stages
+
+def aggregate(indptr, indices, w, H, op: str):
+    indptr, indices, w, H = _i64(indptr), _i32(indices), _f64(w), _f64(H)
+    n, F = indptr.shape[0] - 1, H.shape[1]
+    A = np.empty((n, F), np.float64)
+    lib().ito_aggregate(C.c_int64(n), _p(indptr), _p(indices), _p(w), _p(H), C.c_int32(F),
+                        C.c_int32(OPS[op]), _p(A))
+    return A
+
+
+def partial_gather(shadow_indptr, indices, w, H, op: str):
+    sp, indices, w, H = _i64(shadow_indptr), _i32(indices), _f64(w), _f64(H)
+    R, F = sp.shape[0] - 1, H.shape[1]
+    P = np.empty((R, F), np.float64)
+    lib().ito_partial_gather(C.c_int64(R), _p(sp), _p(indices), _p(w), _p(H), C.c_int32(F),
+                             C.c_int32(OPS[op]), _p(P))
+    return P
+
+
+def combine(owner_indptr, indptr, P, op: str):
+    op_, indptr, P = _i64(owner_indptr), _i64(indptr), _f64(P)
+    n, F = indptr.shape[0] - 1, P.shape[1]
+    A = np.empty((n, F), np.float64)
+    lib().ito_combine(C.c_int64(n), _p(op_), _p(indptr), _p(P), C.c_int32(F), C.c_int32(OPS[op]), _p(A))
+    return A
+
+
+def linear(X, W):
+    X, W = _f64(X), _f64(W)
+    out = np.empty((X.shape[0], W.shape[1]), np.float64)
+    lib().ito_linear(C.c_int64(X.shape[0]), _p(X), C.c_int32(X.shape[1]), _p(W), C.c_int32(W.shape[1]), _p(out))
+    return out
+
+
+def sage_apply(H, A, W, bias, act: str):
+    H, A, W, bias = _f64(H), _f64(A), _f64(W), _f64(bias)
+    n, Fi, Fo = H.shape[0], H.shape[1], W.shape[1]
+    assert W.shape[0] == 2 * Fi and A.shape == H.shape
+    out = np.empty((n, Fo), np.float64)
+    lib().ito_sage_apply(C.c_int64(n), _p(H), _p(A), C.c_int32(Fi), _p(W), _p(bias), C.c_int32(Fo),
+                         C.c_int32(ACTS[act]), _p(out))
+    return out
+
+
+def bias_act(X, bias, act: str):
+    X, bias = _f64(X), _f64(bias)
+    out = np.empty_like(X)
+    lib().ito_bias_act(C.c_int64(X.shape[0]), C.c_int32(X.shape[1]), _p(X), _p(bias), C.c_int32(ACTS[act]), _p(out))
+    return out
+
+
+def gat_scores(Z, att, heads: int):
+    Z, att = _f64(Z), _f64(att)
+    n, F = Z.shape
+    s = np.empty((n, heads), np.float64)
+    lib().ito_gat_scores(C.c_int64(n), _p(Z), C.c_int32(heads), C.c_int32(F // heads), _p(att), _p(s))
+    return s
+
+
+def gat_aggregate(indptr, indices, Z, s_src, s_dst, heads: int, slope: float):
+    indptr, indices, Z, s_src, s_dst = _i64(indptr), _i32(indices), _f64(Z), _f64(s_src), _f64(s_dst)
+    n, F = indptr.shape[0] - 1, Z.shape[1]
+    O = np.empty((n, F), np.float64)
+    lib().ito_gat_aggregate(C.c_int64(n), _p(indptr), _p(indices), _p(Z), _p(s_src), _p(s_dst),
+                            C.c_int32(heads), C.c_int32(F // heads), C.c_double(slope), _p(O))
+    return O
+
+
+# ----------------------------------------------------------------- layers
+
+def _gathered(indptr, indices, w, H, op, threshold):
+    """aggregate, optionally through shadow rows + partial gather + combine (the result is
+    the same by associativity; Section "Optimization Strategies", Partial-Gather)."""
+    if threshold and threshold > 0:
+        sp, _, owner = split_hubs(indptr, threshold)
+        return combine(owner, indptr, partial_gather(sp, indices, w, H, op), op)
+    return aggregate(indptr, indices, w, H, op)
+
+
+def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False):
+    """One GraphSAGE layer for every vertex.  `layer` has op, act, in_dim, out_dim, W
+    [2*in, out], bias, use_edge_weights.  reorder=True evaluates the algebraically equal
+    transform-before-aggregate form (sum and mean only): gather Z = H W_neigh instead of H."""
+    H = _f64(H)
+    W = _f64(layer.W)
+    Fi = layer.in_dim
+    w = edge_weights if layer.use_edge_weights else None
+    if reorder:
+        if layer.op == "max":
+            raise ValueError("transform-before-aggregate is not valid for max")
+        Z = round_to(linear(H, W[Fi:]), storage)
+        S = linear(H, W[:Fi])
+        if layer.bias is not None:
+            S = S + _f64(layer.bias)[None, :]
+        if storage is not None:
+            S = round_f32(S)
+        out = bias_act(S + _gathered(indptr, indices, w, Z, layer.op, threshold), None, layer.act)
+    else:
+        A = round_to(_gathered(indptr, indices, w, H, layer.op, threshold), storage)
+        out = sage_apply(H, A, W, layer.bias, layer.act)
+    return round_to(out, storage)
+
+
+def gat_layer(indptr, indices, H, layer, storage=None):
+    """One GAT layer: z = h W; additive attention per head with LeakyReLU; softmax over the
+    in-edges of each destination; heads concatenated; bias; activation."""
+    z = linear(_f64(H), _f64(layer.W))
+    s_src = gat_scores(z, layer.att_src, layer.heads)
+    s_dst = gat_scores(z, layer.att_dst, layer.heads)
+    if storage is not None:
+        s_src, s_dst = round_f32(s_src), round_f32(s_dst)
+    O = gat_aggregate(indptr, indices, round_to(z, storage), s_src, s_dst, layer.heads, layer.leaky_slope)
+    return round_to(bias_act(O, layer.bias, layer.act), storage)
+
+
+def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False):
+    if layer.op == "gat":
+        return gat_layer(indptr, indices, H, layer, storage)
+    return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder)
+
+
+def will_reorder(layer) -> bool:
+    """The layer contract: transform first when it shrinks the rows that are gathered and
+    the aggregate is linear."""
+    return bool(layer.allow_reorder) and layer.op in ("sum", "mean") and layer.out_dim < layer.in_dim
+
+
+def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, follow_reorder=False):
+    """L layers in order over the whole graph; returns the list of every layer's output."""
+    H = _f64(X)
+    outs = []
+    for layer in layers:
+        H = layer_forward(indptr, indices, edge_weights, H, layer, storage, threshold,
+                          reorder=follow_reorder and will_reorder(layer))
+        outs.append(H)
+    return outs

@@ -1,0 +1,478 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something that is
+not the oracle — hand-worked values, closed forms, invariants, textbook special cases,
+and a brute-force per-vertex computation tree written in pure Python."""
+import json
+import math
+import os
+from types import SimpleNamespace as NS
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "w5.json")))
+
+
+def L(op="sum", act="none", W=None, bias=None, heads=1, att_src=None, att_dst=None, slope=0.2,
+      use_edge_weights=False, allow_reorder=True):
+    W = np.asarray(W, dtype=np.float64)
+    in_dim = W.shape[0] if op == "gat" else W.shape[0] // 2
+    return NS(op=op, act=act, in_dim=in_dim, out_dim=W.shape[1], W=W,
+              bias=None if bias is None else np.asarray(bias, dtype=np.float64), heads=heads,
+              att_src=None if att_src is None else np.asarray(att_src, dtype=np.float64),
+              att_dst=None if att_dst is None else np.asarray(att_dst, dtype=np.float64),
+              leaky_slope=slope, use_edge_weights=use_edge_weights, allow_reorder=allow_reorder)
+
+
+def random_graph(rng, n, max_deg, p_zero=0.2):
+    deg = rng.integers(0, max_deg + 1, size=n)
+    deg[rng.random(n) < p_zero] = 0
+    indptr = np.zeros(n + 1, np.int64)
+    np.cumsum(deg, out=indptr[1:])
+    indices = rng.integers(0, n, size=int(indptr[-1])).astype(np.int32)  # multi-edges and self-edges allowed
+    return indptr, indices
+
+
+# ------------------------------------------------------------------ hand-worked example
+
+class TestW5:
+    ip = np.array(GOLD["indptr"], np.int64)
+    ix = np.array(GOLD["indices"], np.int32)
+    x = np.array(GOLD["x"], np.float64)
+    w = np.array(GOLD["w"], np.float64)
+
+    @pytest.mark.parametrize("op", ["sum", "mean", "max"])
+    def test_aggregates(self, op):
+        assert np.array_equal(O.aggregate(self.ip, self.ix, None, self.x, op), np.array(GOLD[op], np.float64))
+
+    def test_weighted_sum(self):
+        assert np.array_equal(O.aggregate(self.ip, self.ix, self.w, self.x, "sum"), np.array(GOLD["weighted_sum"], np.float64))
+
+    def test_split(self):
+        sp, so, op = O.split_hubs(self.ip, GOLD["split_T"])
+        assert sp.tolist() == GOLD["shadow_indptr"]
+        assert so.tolist() == GOLD["shadow_owner"]
+        assert op.tolist() == GOLD["owner_indptr"]
+        ps = O.partial_gather(sp, self.ix, None, self.x, "sum")
+        pm = O.partial_gather(sp, self.ix, None, self.x, "max")
+        assert ps[:2].tolist() == GOLD["partial_sum_v0"]
+        assert pm[:2].tolist() == GOLD["partial_max_v0"]
+        for o in ("sum", "mean", "max"):
+            P = O.partial_gather(sp, self.ix, None, self.x, o)
+            assert np.array_equal(O.combine(op, self.ip, P, o), np.array(GOLD[o], np.float64))
+
+    def test_two_layer_sage_mean(self):
+        g1, g2 = GOLD["sage_mean_l1"], GOLD["sage_mean_l2"]
+        l1 = L("mean", g1["act"], g1["W"], g1["b"])
+        l2 = L("mean", g2["act"], g2["W"], g2["b"])
+        for thr in (0, 2):
+            for fr in (False, True):
+                outs = O.infer(self.ip, self.ix, None, self.x, [l1, l2], threshold=thr, follow_reorder=fr)
+                assert np.array_equal(outs[0], np.array(g1["out"], np.float64))
+                assert np.array_equal(outs[1], np.array(g2["out"], np.float64))
+        H1 = np.array(g1["out"], np.float64)
+        Z = O.linear(H1, np.array(g2["W"], np.float64)[2:])
+        assert Z.tolist() == g2["Z"]
+        assert O.aggregate(self.ip, self.ix, None, Z, "mean").tolist() == g2["mean_Z"]
+
+    def test_gat(self):
+        g = GOLD["gat"]
+        layer = L("gat", "none", g["W"], None, 1, g["att_src"], g["att_dst"], g["slope"])
+        out = O.gat_layer(self.ip, self.ix, self.x, layer)
+        assert np.abs(out - np.array(g["out"])).max() < g["out_tol"]
+        # the printed alphas reproduce the printed outputs (fixture self-consistency, by hand rule)
+        for v, al in g["alpha"].items():
+            v = int(v)
+            src = self.ix[self.ip[v]:self.ip[v + 1]]
+            assert abs(sum(al) - 1) < 1e-6
+            assert np.abs((np.array(al)[:, None] * self.x[src]).sum(0) - np.array(g["out"][v])).max() < 2e-6
+
+
+# ------------------------------------------------------------------ brute-force computation tree
+
+def py_act(x, act):
+    if act == "relu":
+        return x if x > 0 else 0.0
+    if act == "elu":
+        return x if x > 0 else math.exp(x) - 1.0
+    return x
+
+
+def tree_eval(v, depth, ip, ix, w, x, layers, memo=None):
+    """h_v^depth by direct recursion over the in-neighbourhood (Eq. (1)); pure Python floats.
+    No memo: every path of the computation tree is evaluated, as a k-hop pipeline would."""
+    if depth == 0:
+        return [float(t) for t in x[v]]
+    lay = layers[depth - 1]
+    hv = tree_eval(v, depth - 1, ip, ix, w, x, layers)
+    nb = [(int(ix[j]), (float(w[j]) if (w is not None and lay.use_edge_weights) else 1.0)) for j in range(ip[v], ip[v + 1])]
+    hn = [tree_eval(u, depth - 1, ip, ix, w, x, layers) for u, _ in nb]
+    Fi, Fo = lay.in_dim, lay.out_dim
+    W = lay.W
+    if lay.op == "gat":
+        D = Fo // lay.heads
+        zl = lambda h: [sum(h[k] * W[k][c] for k in range(Fi)) for c in range(Fo)]
+        zv, zn = zl(hv), [zl(h) for h in hn]
+        out = [0.0] * Fo
+        for hd in range(lay.heads):
+            sd = sum(lay.att_dst[hd][c] * zv[hd * D + c] for c in range(D))
+            es = []
+            for z in zn:
+                e = sum(lay.att_src[hd][c] * z[hd * D + c] for c in range(D)) + sd
+                es.append(e if e > 0 else lay.leaky_slope * e)
+            if es:
+                m = max(es)
+                ex = [math.exp(e - m) for e in es]
+                tot = sum(ex)
+                for z, p in zip(zn, ex):
+                    for c in range(D):
+                        out[hd * D + c] += p / tot * z[hd * D + c]
+        return [py_act(out[c] + (lay.bias[c] if lay.bias is not None else 0.0), lay.act) for c in range(Fo)]
+    agg = [0.0] * Fi
+    if hn:
+        for f in range(Fi):
+            msgs = [wj * h[f] for (_, wj), h in zip(nb, hn)]
+            agg[f] = max(msgs) if lay.op == "max" else sum(msgs)
+            if lay.op == "mean":
+                agg[f] /= len(msgs)
+    out = []
+    for c in range(Fo):
+        t = lay.bias[c] if lay.bias is not None else 0.0
+        t += sum(hv[k] * W[k][c] for k in range(Fi)) + sum(agg[k] * W[Fi + k][c] for k in range(Fi))
+        out.append(py_act(t, lay.act))
+    return out
+
+
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "gat"])
+@pytest.mark.parametrize("depth", [1, 2, 3])
+def test_layerwise_equals_computation_tree(op, depth):
+    rng = np.random.default_rng(100 + depth)
+    n = 14
+    ip, ix = random_graph(rng, n, 3)
+    w = rng.random(ix.shape[0])
+    dims = [3, 4, 2, 3][:depth + 1]
+    x = rng.standard_normal((n, dims[0]))
+    layers = []
+    for i in range(depth):
+        fi, fo = dims[i], dims[i + 1]
+        act = ["relu", "elu", "none"][i % 3]
+        if op == "gat":
+            fo = 4
+            dims[i + 1] = 4
+            layers.append(L("gat", act, rng.standard_normal((fi, fo)), rng.standard_normal(fo), 2,
+                            rng.standard_normal((2, 2)), rng.standard_normal((2, 2)), 0.2))
+        else:
+            layers.append(L(op, act, rng.standard_normal((2 * fi, fo)), rng.standard_normal(fo),
+                            use_edge_weights=(op != "mean")))
+    full = O.infer(ip, ix, w, x, layers)[-1]
+    split = O.infer(ip, ix, w, x, layers, threshold=2, follow_reorder=True)[-1]
+    for v in range(n):
+        ref = np.array(tree_eval(v, depth, ip, ix, w, x, layers))
+        assert np.allclose(full[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+        assert np.allclose(split[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+
+
+def khop_in_neighbourhood(v, k, ip, ix):
+    seen, frontier = {v}, {v}
+    for _ in range(k):
+        nxt = set()
+        for t in frontier:
+            nxt.update(int(u) for u in ix[ip[t]:ip[t + 1]])
+        frontier = nxt - seen
+        seen |= nxt
+    return sorted(seen)
+
+
+@pytest.mark.parametrize("op", ["mean", "max", "gat"])
+def test_khop_neighbourhood_is_sufficient(op):
+    """A k-layer model on the induced k-hop neighbourhood of v gives the full-graph value at v
+    (Section "K-hop Neighborhood and Sampling"; the paper's consistency property)."""
+    rng = np.random.default_rng(7)
+    n, k = 60, 2
+    ip, ix = random_graph(rng, n, 3)
+    x = rng.standard_normal((n, 4))
+    if op == "gat":
+        layers = [L("gat", "elu", rng.standard_normal((4, 4)), rng.standard_normal(4), 2,
+                    rng.standard_normal((2, 2)), rng.standard_normal((2, 2))) for _ in range(k)]
+    else:
+        layers = [L(op, "relu", rng.standard_normal((8, 4)), rng.standard_normal(4)) for _ in range(k)]
+    full = O.infer(ip, ix, None, x, layers)[-1]
+    for v in range(0, n, 7):
+        keep = khop_in_neighbourhood(v, k, ip, ix)
+        new_id = {u: i for i, u in enumerate(keep)}
+        sub_ip, sub_ix = [0], []
+        for u in keep:   # induced subgraph: every edge between kept vertices
+            sub_ix += [new_id[int(s)] for s in ix[ip[u]:ip[u + 1]] if int(s) in new_id]
+            sub_ip.append(len(sub_ix))
+        # vertices at distance < k keep all their in-edges, which is what the value at v needs
+        sub = O.infer(np.array(sub_ip, np.int64), np.array(sub_ix, np.int32), None, x[keep], layers)[-1]
+        assert np.allclose(sub[new_id[v]], full[v], rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ split / combine / buckets
+
+def brute_split(deg, T):
+    sp, so, op, pos = [], [], [], 0
+    for v, d in enumerate(deg):
+        n = 1 if (T <= 0 or d <= T) else -(-d // T)
+        op.append(len(so))
+        sizes = [d // n + (1 if g < d % n else 0) for g in range(n)]
+        for s in sizes:
+            sp.append(pos)
+            so.append(v)
+            pos += s
+    op.append(len(so))
+    sp.append(pos)
+    return sp, so, op
+
+
+@pytest.mark.parametrize("T", [0, 1, 2, 3, 7, 16, 1000])
+def test_split_rule_closed_forms(T):
+    rng = np.random.default_rng(T)
+    deg = np.concatenate([rng.integers(0, 40, size=200), [0, 1, T, T + 1, 2 * T, 2 * T + 1, 997]]).astype(np.int64)
+    deg = np.maximum(deg, 0)
+    ip = np.zeros(deg.size + 1, np.int64)
+    np.cumsum(deg, out=ip[1:])
+    sp, so, op = O.split_hubs(ip, T)
+    bs, bo, bp = brute_split(deg.tolist(), T)
+    assert sp.tolist() == bs and so.tolist() == bo and op.tolist() == bp
+    lens = np.diff(sp)
+    for v, d in enumerate(deg):
+        g = lens[op[v]:op[v + 1]]
+        assert g.sum() == d
+        assert g.max() - g.min() <= 1
+        if T > 0:
+            assert g.max() <= max(T, 0) or d == 0
+            assert g.size == (1 if d <= T else math.ceil(d / T))
+            if g.size > 1:
+                assert (g.size - 1) * T < d   # smallest n that keeps every group <= T
+        else:
+            assert g.size == 1
+        assert sp[op[v]] == ip[v] and sp[op[v + 1]] == ip[v + 1]
+        assert np.all(np.diff(g) <= 0)        # the larger groups come first
+
+
+@pytest.mark.parametrize("op", ["sum", "mean", "max"])
+def test_split_invariance(op):
+    """Partial gather + combine does not change the result (associativity): bit-exact for
+    max and for integer-valued inputs, to rounding for general floats."""
+    rng = np.random.default_rng(3)
+    ip, ix = random_graph(rng, 300, 90)
+    w = rng.random(ix.shape[0])
+    H = rng.standard_normal((300, 5))
+    Hi = rng.integers(-8, 9, size=(300, 5)).astype(np.float64)
+    wi = rng.integers(1, 4, size=ix.shape[0]).astype(np.float64)
+    base, base_i = O.aggregate(ip, ix, w, H, op), O.aggregate(ip, ix, wi, Hi, op)
+    for T in (1, 2, 5, 17, 64, 89, 90, 1000):
+        sp, so, owner = O.split_hubs(ip, T)
+        got = O.combine(owner, ip, O.partial_gather(sp, ix, w, H, op), op)
+        got_i = O.combine(owner, ip, O.partial_gather(sp, ix, wi, Hi, op), op)
+        if op == "max":
+            assert np.array_equal(got, base)
+        else:
+            assert np.allclose(got, base, rtol=1e-12, atol=1e-12)
+        if op != "mean":
+            assert np.array_equal(got_i, base_i)
+        else:
+            assert np.allclose(got_i, base_i, rtol=1e-15, atol=0)
+
+
+def test_buckets_brute_force_and_stability():
+    rng = np.random.default_rng(5)
+    lens = np.concatenate([rng.integers(0, 50, size=500), [0, 0, 8, 9, 32, 33, 256, 257, 300]]).astype(np.int64)
+    sp = np.zeros(lens.size + 1, np.int64)
+    np.cumsum(lens, out=sp[1:])
+    bounds = [0, 8, 32, 256, 300]
+    off, rows = O.buckets(sp, bounds)
+    assert off[0] == 0 and off[-1] == lens.size
+    assert sorted(rows.tolist()) == list(range(lens.size))
+    lo = -1
+    for b, hi in enumerate(bounds):
+        r = rows[off[b]:off[b + 1]]
+        assert np.all(np.diff(r) > 0)                       # stable: ascending row id
+        assert np.all((lens[r] > lo) & (lens[r] <= hi))
+        assert r.tolist() == [i for i in range(lens.size) if lo < lens[i] <= hi]
+        lo = hi
+    with pytest.raises(ValueError):
+        O.buckets(sp, [0, 8, 32])
+
+
+# ------------------------------------------------------------------ textbook special cases
+
+def dense_adjacency(ip, ix, w, n):
+    A = np.zeros((n, n))
+    for v in range(n):
+        for j in range(ip[v], ip[v + 1]):
+            A[v, ix[j]] += 1.0 if w is None else w[j]
+    return A
+
+
+def test_sum_layer_is_sparse_times_dense():
+    """W_self = 0, W_neigh = I, no bias, no activation: the layer is (weighted adjacency) x H."""
+    rng = np.random.default_rng(11)
+    n, F = 50, 6
+    ip, ix = random_graph(rng, n, 9)
+    w = rng.random(ix.shape[0])
+    H = rng.standard_normal((n, F))
+    layer = L("sum", "none", np.vstack([np.zeros((F, F)), np.eye(F)]), None, use_edge_weights=True)
+    out = O.sage_layer(ip, ix, w, H, layer)
+    assert np.allclose(out, dense_adjacency(ip, ix, w, n) @ H, rtol=1e-13, atol=1e-13)
+    layer.use_edge_weights = False
+    out = O.sage_layer(ip, ix, w, H, layer)
+    assert np.allclose(out, dense_adjacency(ip, ix, None, n) @ H, rtol=1e-13, atol=1e-13)
+
+
+def test_self_and_neighbour_blocks_are_not_swapped():
+    """Rows 0..in-1 of W multiply the vertex's own state, rows in..2in-1 the aggregate."""
+    rng = np.random.default_rng(12)
+    n, F = 30, 3
+    ip, ix = random_graph(rng, n, 4)
+    H = rng.standard_normal((n, F))
+    Ws, Wn, b = rng.standard_normal((F, 2)), rng.standard_normal((F, 2)), rng.standard_normal(2)
+    out = O.sage_layer(ip, ix, None, H, L("sum", "none", np.vstack([Ws, Wn]), b))
+    assert np.allclose(out, H @ Ws + (dense_adjacency(ip, ix, None, n) @ H) @ Wn + b, rtol=1e-13, atol=1e-13)
+
+
+def test_linear_and_activations_against_numpy():
+    rng = np.random.default_rng(13)
+    X, W, b = rng.standard_normal((40, 7)), rng.standard_normal((7, 5)), rng.standard_normal(5)
+    assert np.allclose(O.linear(X, W), X @ W, rtol=1e-13, atol=1e-13)
+    Y = X[:, :5] * 3
+    assert np.array_equal(O.bias_act(Y, b, "relu"), np.maximum(Y + b, 0))
+    assert np.allclose(O.bias_act(Y, b, "elu"), np.where(Y + b > 0, Y + b, np.expm1(Y + b)), rtol=1e-15)
+    assert np.array_equal(O.bias_act(Y, None, "none"), Y)
+    A = rng.standard_normal((40, 7))
+    W2 = rng.standard_normal((14, 5))
+    assert np.allclose(O.sage_apply(X, A, W2, b, "none"), np.hstack([X, A]) @ W2 + b, rtol=1e-13, atol=1e-13)
+
+
+def test_mean_of_constant_is_constant_and_max_dominates_mean():
+    rng = np.random.default_rng(14)
+    n = 200
+    ip, ix = random_graph(rng, n, 12)
+    deg = np.diff(ip)
+    H = np.full((n, 3), 2.5)
+    m = O.aggregate(ip, ix, None, H, "mean")
+    assert np.array_equal(m[deg > 0], H[deg > 0]) and np.all(m[deg == 0] == 0)
+    H = rng.standard_normal((n, 3))
+    mx, mn, sm = (O.aggregate(ip, ix, None, H, o) for o in ("max", "mean", "sum"))
+    assert np.all(mx[deg > 0] >= mn[deg > 0] - 1e-15)
+    assert np.allclose(sm, mn * deg[:, None], rtol=1e-13, atol=1e-13)
+    assert np.all(mx[deg == 0] == 0)
+    # max of all-negative messages stays negative (no spurious 0 from the initial value)
+    mxn = O.aggregate(ip, ix, None, -np.abs(H) - 1, "max")
+    assert np.all(mxn[deg > 0] < 0)
+
+
+def test_permutation_invariance_inside_segments():
+    rng = np.random.default_rng(15)
+    n = 120
+    ip, ix = random_graph(rng, n, 10)
+    w = rng.random(ix.shape[0])
+    H = rng.standard_normal((n, 4))
+    ix2, w2 = ix.copy(), w.copy()
+    for v in range(n):
+        p = rng.permutation(ip[v + 1] - ip[v]) + ip[v]
+        ix2[ip[v]:ip[v + 1]], w2[ip[v]:ip[v + 1]] = ix[p], w[p]
+    assert np.array_equal(O.aggregate(ip, ix, w, H, "max"), O.aggregate(ip, ix2, w2, H, "max"))
+    assert np.allclose(O.aggregate(ip, ix, w, H, "sum"), O.aggregate(ip, ix2, w2, H, "sum"), rtol=1e-12, atol=1e-13)
+    gl = L("gat", "none", rng.standard_normal((4, 4)), None, 2, rng.standard_normal((2, 2)), rng.standard_normal((2, 2)))
+    assert np.allclose(O.gat_layer(ip, ix, H, gl), O.gat_layer(ip, ix2, H, gl), rtol=1e-12, atol=1e-13)
+
+
+def test_gat_softmax_special_cases():
+    rng = np.random.default_rng(16)
+    n, F, heads = 150, 6, 3
+    ip, ix = random_graph(rng, n, 8)
+    deg = np.diff(ip)
+    H = rng.standard_normal((n, F))
+    W = rng.standard_normal((F, F))
+    zero = np.zeros((heads, F // heads))
+    # all-equal scores: attention is uniform, the reduce is a mean of z
+    out = O.gat_layer(ip, ix, H, L("gat", "none", W, None, heads, zero, zero))
+    assert np.allclose(out, O.aggregate(ip, ix, None, H @ W, "mean"), rtol=1e-12, atol=1e-13)
+    # destination score is common to a segment, so it cannot change alpha when e > 0 everywhere
+    a_s, a_d = rng.standard_normal((heads, F // heads)), rng.standard_normal((heads, F // heads))
+    lay = L("gat", "none", W, None, heads, a_s, a_d, slope=1.0)       # slope 1: LeakyReLU is the identity
+    lay0 = L("gat", "none", W, None, heads, a_s, zero, slope=1.0)
+    assert np.allclose(O.gat_layer(ip, ix, H, lay), O.gat_layer(ip, ix, H, lay0), rtol=1e-10, atol=1e-12)
+    # weights sum to one: constant z comes back unchanged where there is an in-edge, 0 elsewhere
+    Hc = np.ones((n, F))
+    out = O.gat_layer(ip, ix, Hc, L("gat", "none", np.eye(F), None, heads, a_s, a_d))
+    assert np.allclose(out[deg > 0], 1.0, rtol=1e-13) and np.all(out[deg == 0] == 0)
+    # single in-edge: alpha = 1
+    one = np.flatnonzero(deg == 1)
+    full = O.gat_layer(ip, ix, H, L("gat", "none", W, None, heads, a_s, a_d))
+    assert one.size > 0 and np.allclose(full[one], (H @ W)[ix[ip[one]]], rtol=1e-13, atol=1e-14)
+    # two in-edges: closed-form two-way softmax (a logistic of the score difference)
+    two = np.flatnonzero(deg == 2)
+    z = H @ W
+    D = F // heads
+    for v in two[:10]:
+        u0, u1 = ix[ip[v]], ix[ip[v] + 1]
+        for k in range(heads):
+            sl = slice(k * D, (k + 1) * D)
+            lrelu = lambda t: t if t > 0 else 0.2 * t
+            e0 = lrelu(a_s[k] @ z[u0, sl] + a_d[k] @ z[v, sl])
+            e1 = lrelu(a_s[k] @ z[u1, sl] + a_d[k] @ z[v, sl])
+            a0 = 1.0 / (1.0 + math.exp(e1 - e0))
+            assert np.allclose(full[v, sl], a0 * z[u0, sl] + (1 - a0) * z[u1, sl], rtol=1e-11, atol=1e-13)
+
+
+def test_gat_softmax_is_shift_safe():
+    """Large scores must not overflow: the max is subtracted before exp."""
+    ip = np.array([0, 3], np.int64)
+    ix = np.array([0, 0, 0], np.int32)
+    lay = L("gat", "none", [[1000.0]], None, 1, [[1.0]], [[0.0]])
+    out = O.gat_layer(ip, ix, np.array([[1.0]]), lay)
+    assert np.isfinite(out).all() and abs(out[0, 0] - 1000.0) < 1e-9
+
+
+def test_reorder_is_algebraically_equal():
+    rng = np.random.default_rng(17)
+    n = 100
+    ip, ix = random_graph(rng, n, 20)
+    w = rng.random(ix.shape[0])
+    H = rng.standard_normal((n, 8))
+    for op in ("sum", "mean"):
+        lay = L(op, "relu", rng.standard_normal((16, 3)), rng.standard_normal(3), use_edge_weights=True)
+        a = O.sage_layer(ip, ix, w, H, lay, reorder=False)
+        b = O.sage_layer(ip, ix, w, H, lay, reorder=True, threshold=4)
+        assert np.allclose(a, b, rtol=1e-11, atol=1e-12)
+    with pytest.raises(ValueError):
+        O.sage_layer(ip, ix, w, H, L("max", "relu", rng.standard_normal((16, 3))), reorder=True)
+    assert O.will_reorder(L("sum", W=np.zeros((16, 3)))) and not O.will_reorder(L("max", W=np.zeros((16, 3))))
+    assert not O.will_reorder(L("sum", W=np.zeros((16, 8)))) and not O.will_reorder(L("sum", W=np.zeros((16, 3)), allow_reorder=False))
+
+
+# ------------------------------------------------------------------ rounding helpers
+
+def test_round_bf16_matches_torch_and_ties_to_even():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(18)
+    x32 = np.concatenate([rng.standard_normal(20000).astype(np.float32) * 10.0 ** rng.integers(-30, 30, 20000).astype(np.float32),
+                          np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3e38, -3.3e38, 1e-40, 65504.0], np.float32)])
+    ref = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
+    got = O.round_bf16(x32.astype(np.float64))
+    assert np.array_equal(got, ref)
+    # exact ties in fp64 that fp32 cannot hold a hair away from: 1 + 2^-8 is a tie -> even (1.0);
+    # 1 + 2^-8 + 2^-40 is above the tie -> 1 + 2^-7
+    assert O.round_bf16(np.array([1 + 2.0 ** -8]))[0] == 1.0
+    assert O.round_bf16(np.array([1 + 2.0 ** -8 + 2.0 ** -40]))[0] == 1 + 2.0 ** -7
+    assert O.round_bf16(np.array([1 + 3 * 2.0 ** -8]))[0] == 1 + 2.0 ** -6
+    assert O.round_f32(np.array([1 + 2.0 ** -30]))[0] == 1.0
+
+
+def test_storage_mode_stays_close_to_exact_mode():
+    rng = np.random.default_rng(19)
+    n = 300
+    ip, ix = random_graph(rng, n, 30)
+    X = rng.standard_normal((n, 8))
+    layers = [L("mean", "relu", rng.uniform(-.4, .4, (16, 8)), rng.uniform(-.1, .1, 8)),
+              L("mean", "none", rng.uniform(-.4, .4, (16, 4)), rng.uniform(-.1, .1, 4))]
+    a = O.infer(ip, ix, None, X, layers)[-1]
+    for storage, tol in (("f32", 1e-6), ("bf16", 3e-2)):
+        b = O.infer(ip, ix, None, X, layers, storage=storage, threshold=7, follow_reorder=True)[-1]
+        assert np.abs(a - b).max() / np.sqrt((a ** 2).mean()) < tol
+        assert not np.array_equal(a, b)
