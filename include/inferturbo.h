@@ -1,0 +1,192 @@
+/*
+ * inferturbo.h — C ABI of the B200 (sm_100a) layer-pass library.
+ *
+ * One Gather-Apply-Scatter layer pass of full-graph GNN inference over every vertex,
+ * repeated layer after layer with no sampling (InferTurbo, arXiv 2307.00228).
+ *
+ * Conventions for every call
+ *   - "device pointer" = memory on the current CUDA device, allocated by the caller.
+ *     The library BORROWS caller arrays (never frees, never writes inputs) and OWNS
+ *     only what it derives inside an it_graph (freed by it_graph_destroy).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *     enqueued on it; a call synchronises that stream only where it must read a status
+ *     or a count back (it_graph_create, it_split_hubs).
+ *   - Matrices are row-major and dense.  Feature rows must be a multiple of 16 bytes.
+ *   - Errors are return codes only: nothing throws, aborts or traps the device.  On
+ *     error no output is defined.  it_status_string() names a code;
+ *     it_last_error_message() gives the detail of the calling thread's last failure.
+ */
+#ifndef INFERTURBO_H
+#define INFERTURBO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct it_graph it_graph; /* opaque, library-owned */
+
+typedef enum {
+  IT_OK = 0,
+  IT_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, bad enum, dims not supported by shape rules */
+  IT_ERR_BAD_GRAPH = 2,   /* indptr not monotone / wrong ends, or a source id outside [0, n) */
+  IT_ERR_UNSUPPORTED = 3, /* a valid request this build has no kernel for */
+  IT_ERR_WORKSPACE = 4,   /* workspace NULL, misaligned or smaller than it_workspace_bytes() */
+  IT_ERR_OOM = 5,         /* device allocation of library-owned arrays failed */
+  IT_ERR_CUDA = 6,        /* a CUDA call or kernel launch failed */
+  IT_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up */
+} it_status;
+
+typedef enum { IT_F32 = 0, IT_BF16 = 1 } it_dtype;
+typedef enum { IT_I32 = 0, IT_I64 = 1 } it_itype;
+typedef enum { IT_GATHER_SUM = 0, IT_GATHER_MEAN = 1, IT_GATHER_MAX = 2, IT_GATHER_GAT = 3 } it_gather_op;
+typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
+
+#define IT_MAX_BUCKETS 8
+
+/*
+ * One GNN layer in the paper's stage vocabulary (Section "InferTurbo Abstraction"):
+ * `op` is the aggregate of the Gather stage, W / bias / act are apply_node, and
+ * use_edge_weights selects the minimal apply_edge (message = w_e * h_src).
+ *
+ * GraphSAGE (op = SUM | MEAN | MAX):
+ *     a_v  = op_{e = (u -> v)} ( w_e * h_u )            (0 for a vertex with no in-edge;
+ *                                                        MEAN divides by the edge count)
+ *     h'_v = act( h_v * W[0:in_dim, :] + a_v * W[in_dim:2*in_dim, :] + bias )
+ *   W is [2*in_dim, out_dim].
+ * GAT (op = GAT; out_dim = heads * head_dim):
+ *     z_u = h_u * W                                      W is [in_dim, out_dim]
+ *     e   = LeakyReLU_slope( att_src[k] . z_u^k + att_dst[k] . z_v^k )    per head k
+ *     h'_v = act( concat_k sum_e softmax_e(e) z_u^k + bias )
+ *   The message-passing form is Eq. (1); the paper places GAT's reduce in apply_node
+ *   because attention is not associative.
+ *
+ * Storage contract: h_in, h_out (and the internal Z / aggregate tensors) are feat_dtype,
+ * rounded to nearest even when written; all accumulation is fp32.  W is weight_dtype and
+ * must equal feat_dtype.  bias, att_src, att_dst are fp32.  All are device pointers.
+ */
+typedef struct {
+  it_gather_op op;
+  it_act act;
+  int32_t in_dim, out_dim, heads;       /* heads = 1 unless GAT */
+  it_dtype feat_dtype, weight_dtype;
+  const void *W;
+  const float *bias;                    /* [out_dim], may be NULL */
+  const float *att_src, *att_dst;       /* GAT only: [heads, out_dim / heads] */
+  float leaky_slope;                    /* GAT only */
+  int32_t use_edge_weights;             /* 0/1; needs a graph created with edge weights */
+  int32_t allow_reorder;                /* 0/1: allow transform-before-aggregate (see it_layer_forward) */
+} it_layer_desc;
+
+/*
+ * it_graph_create — accept a directed, weighted graph G = {V, E, X, E} (Section
+ * "K-hop Neighborhood and Sampling") as CSR by destination: the in-edges of vertex v
+ * are entries [indptr[v], indptr[v+1]) of `indices` (source ids) and `edge_weights`.
+ * Multi-edges and self-edges are allowed; each entry is one message.
+ *   n_vertices in [0, 2^31 - 2]; n_edges >= 0 (int64).
+ *   indptr: device, n_vertices + 1 entries of indptr_type.  indices: device int32.
+ *   edge_weights: device fp32 [n_edges] or NULL.
+ * The CSR is validated on the device (indptr[0] = 0, non-decreasing, indptr[n] = n_edges,
+ * 0 <= source < n): IT_ERR_BAD_GRAPH if not.  The arrays are borrowed until
+ * it_graph_destroy.  The new graph starts unsplit (as after it_split_hubs(g, 0)).
+ * Synchronises `stream`.
+ */
+it_status it_graph_create(int64_t n_vertices, int64_t n_edges, const void *indptr,
+                          it_itype indptr_type, const int32_t *indices,
+                          const float *edge_weights, void *stream, it_graph **out);
+
+/*
+ * it_split_hubs — the shadow-node rule ("divide the edges into n groups evenly ... the id
+ * of each mirror is appended with the group information", Section "Optimization
+ * Strategies", Shadow Nodes) applied to the in-edge segment of every vertex whose
+ * in-degree d exceeds `threshold` T, so that each group can be gathered on its own and
+ * the partial results combined (Partial-Gather, same section).
+ *   n = 1 if d <= T (or T <= 0), else ceil(d / T) groups; group g takes the next
+ *   d / n + (g < d % n) consecutive edges.  Row id = owner_indptr[v] + g.
+ * Also builds the degree buckets: shadow rows partitioned stably by length class
+ * (bounds from it_graph_get_split).  Rebuilds everything derived; edge arrays are not
+ * permuted.  out_n_rows / out_n_split_owners may be NULL.  Synchronises `stream`.
+ */
+it_status it_split_hubs(it_graph *g, int64_t threshold, void *stream, int64_t *out_n_rows,
+                        int64_t *out_n_split_owners);
+
+/*
+ * it_graph_get_split — borrowed device pointers to the derived index arrays (valid until
+ * the next it_split_hubs / it_graph_destroy):
+ *   shadow_indptr int64[R+1], shadow_owner int32[R], owner_indptr int64[n+1],
+ *   bucket_offsets int64[n_buckets+1], bucket_rows int32[R] (ascending row id inside a
+ *   bucket), and the bucket upper bounds copied to the HOST array bucket_bounds
+ *   (IT_MAX_BUCKETS entries; row of length L is in the first bucket with L <= bound).
+ * Any out pointer may be NULL.
+ */
+it_status it_graph_get_split(const it_graph *g, int64_t *n_rows, const int64_t **shadow_indptr,
+                             const int32_t **shadow_owner, const int64_t **owner_indptr,
+                             const int64_t **bucket_offsets, const int32_t **bucket_rows,
+                             int32_t *n_buckets, int64_t *bucket_bounds);
+
+/*
+ * it_workspace_bytes — bytes of caller-provided device scratch that it_infer needs for
+ * these layers on this graph (with its current split); it_layer_forward of any one of
+ * them needs no more.  Layer pointers inside `layers` are not dereferenced.
+ */
+it_status it_workspace_bytes(const it_graph *g, const it_layer_desc *layers, int32_t n_layers,
+                             size_t *out_bytes);
+
+/*
+ * it_layer_forward — one layer for every vertex: gather (per shadow row, by degree
+ * bucket) -> combine the partial results of split vertices -> apply -> write h_out, which
+ * the next layer reads ("scatter": on one device sending along out-edges is a store).
+ *   h_in  [n, in_dim], h_out [n, out_dim], feat_dtype, device, must not overlap.
+ *   workspace: device, 256-byte aligned, >= it_workspace_bytes(g, layer, 1).
+ * If allow_reorder and op is SUM or MEAN and out_dim < in_dim, the neighbour transform is
+ * done before the gather (the paper's "computation flow would be reorganized", Section
+ * "Inference"): Z = h_in * W[in_dim:, :] is stored in feat_dtype and gathered instead of
+ * h_in; the self term h_in * W[0:in_dim, :] + bias stays fp32.
+ * Asynchronous on `stream`.  Results are bit-identical from run to run.
+ */
+it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const void *h_in,
+                           void *h_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * it_infer — L layers in order ("after k iterations we get the result of a k-layer
+ * model", Section "InferTurbo on Graph Processing System"): exactly the sequence of
+ * it_layer_forward calls, intermediate layer outputs double-buffered inside the
+ * workspace.  x [n, layers[0].in_dim]; out [n, layers[L-1].out_dim]; layers[i].out_dim must
+ * equal layers[i+1].in_dim and all feat_dtype agree.  Bit-identical to calling
+ * it_layer_forward layer by layer.  Asynchronous on `stream`.
+ */
+it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, const void *x,
+                   void *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Frees the library-owned arrays of the graph.  NULL is accepted. */
+it_status it_graph_destroy(it_graph *g);
+
+const char *it_status_string(it_status s);
+const char *it_last_error_message(void);
+
+/*
+ * Instrumentation (no counterpart in the paper, which reports per-instance latency and IO
+ * bytes of its cluster workers; this is the per-kernel equivalent).  Between it_profile_begin
+ * and it_profile_end every kernel the library launches is bracketed by CUDA events on its
+ * own stream.  it_profile_end waits for those events and returns, per kernel kind, the number
+ * of launches, the summed device time, and the summed ALGORITHMIC bytes and flops of those
+ * launches (what the method must move / compute: per edge one index, one optional weight and
+ * one source row; per row its bounds and one output row; for the dense transform its operands
+ * once and 2*M*K*N flops).  `stats` is a HOST array of `capacity` entries; *n_stats receives
+ * the number of kinds seen.  it_kernel_launch_count: kernels launched by this process so far.
+ */
+typedef struct {
+  char name[32];
+  int64_t launches;
+  double total_ms, algo_bytes, algo_flops;
+} it_kernel_stat;
+it_status it_profile_begin(void);
+it_status it_profile_end(it_kernel_stat *stats, int32_t capacity, int32_t *n_stats);
+int64_t it_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INFERTURBO_H */

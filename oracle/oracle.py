@@ -204,6 +204,17 @@ def gat_aggregate(indptr, indices, Z, s_src, s_dst, heads: int, slope: float):
 
 # ----------------------------------------------------------------- layers
 
+def _sub_csr(indptr, indices, w, rows):
+    """CSR restricted to the destination vertices `rows` (source ids stay global)."""
+    indptr = _i64(indptr)
+    rows = _i64(rows)
+    deg = indptr[rows + 1] - indptr[rows]
+    sub = np.zeros(rows.shape[0] + 1, np.int64)
+    np.cumsum(deg, out=sub[1:])
+    pos = np.repeat(indptr[rows] - sub[:-1], deg) + np.arange(sub[-1], dtype=np.int64)
+    return sub, _i32(indices)[pos], (None if w is None else np.asarray(w)[pos])
+
+
 def _gathered(indptr, indices, w, H, op, threshold):
     """aggregate, optionally through shadow rows + partial gather + combine (the result is
     the same by associativity; Section "Optimization Strategies", Partial-Gather)."""
@@ -213,19 +224,38 @@ def _gathered(indptr, indices, w, H, op, threshold):
     return aggregate(indptr, indices, w, H, op)
 
 
-def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False):
-    """One GraphSAGE layer for every vertex.  `layer` has op, act, in_dim, out_dim, W
-    [2*in, out], bias, use_edge_weights.  reorder=True evaluates the algebraically equal
-    transform-before-aggregate form (sum and mean only): gather Z = H W_neigh instead of H."""
+def _sources_of(indptr, indices, rows):
+    """Sorted unique vertex ids that `rows` read: themselves and their in-neighbours."""
+    sub, idx, _ = _sub_csr(indptr, indices, None, rows)
+    return np.union1d(_i64(rows), idx.astype(np.int64))
+
+
+def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
+    """One GraphSAGE layer.  `layer` has op, act, in_dim, out_dim, W [2*in, out], bias,
+    use_edge_weights.  reorder=True evaluates the algebraically equal transform-before-
+    aggregate form (sum and mean only): gather Z = H W_neigh instead of H.
+    rows=None: every vertex.  rows=array: only those destination vertices (H is still indexed
+    by global vertex id; rows of H that they do not read are never touched); returns
+    [len(rows), out]."""
     H = _f64(H)
     W = _f64(layer.W)
     Fi = layer.in_dim
     w = edge_weights if layer.use_edge_weights else None
+    if rows is None:
+        Hself = H
+    else:
+        indptr, indices, w = _sub_csr(indptr, indices, w, rows)
+        Hself = H[_i64(rows)]
     if reorder:
         if layer.op == "max":
             raise ValueError("transform-before-aggregate is not valid for max")
-        Z = round_to(linear(H, W[Fi:]), storage)
-        S = linear(H, W[:Fi])
+        if rows is None:
+            Z = round_to(linear(H, W[Fi:]), storage)
+        else:   # transform only the rows that are read
+            need = np.unique(indices.astype(np.int64))
+            Z = np.full((H.shape[0], layer.out_dim), np.nan)
+            Z[need] = round_to(linear(H[need], W[Fi:]), storage)
+        S = linear(Hself, W[:Fi])
         if layer.bias is not None:
             S = S + _f64(layer.bias)[None, :]
         if storage is not None:
@@ -233,26 +263,37 @@ def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=
         out = bias_act(S + _gathered(indptr, indices, w, Z, layer.op, threshold), None, layer.act)
     else:
         A = round_to(_gathered(indptr, indices, w, H, layer.op, threshold), storage)
-        out = sage_apply(H, A, W, layer.bias, layer.act)
+        out = sage_apply(Hself, A, W, layer.bias, layer.act)
     return round_to(out, storage)
 
 
-def gat_layer(indptr, indices, H, layer, storage=None):
+def gat_layer(indptr, indices, H, layer, storage=None, rows=None):
     """One GAT layer: z = h W; additive attention per head with LeakyReLU; softmax over the
-    in-edges of each destination; heads concatenated; bias; activation."""
-    z = linear(_f64(H), _f64(layer.W))
-    s_src = gat_scores(z, layer.att_src, layer.heads)
-    s_dst = gat_scores(z, layer.att_dst, layer.heads)
+    in-edges of each destination; heads concatenated; bias; activation.  `rows` as in
+    sage_layer."""
+    H = _f64(H)
+    if rows is None:
+        z = linear(H, _f64(layer.W))
+        s_src = gat_scores(z, layer.att_src, layer.heads)
+        s_dst = gat_scores(z, layer.att_dst, layer.heads)
+    else:
+        need = _sources_of(indptr, indices, rows)
+        indptr, indices, _ = _sub_csr(indptr, indices, None, rows)
+        z = np.full((H.shape[0], layer.out_dim), np.nan)
+        z[need] = linear(H[need], _f64(layer.W))
+        s_src = np.full((H.shape[0], layer.heads), np.nan)
+        s_src[need] = gat_scores(z[need], layer.att_src, layer.heads)
+        s_dst = gat_scores(z[_i64(rows)], layer.att_dst, layer.heads)
     if storage is not None:
         s_src, s_dst = round_f32(s_src), round_f32(s_dst)
     O = gat_aggregate(indptr, indices, round_to(z, storage), s_src, s_dst, layer.heads, layer.leaky_slope)
     return round_to(bias_act(O, layer.bias, layer.act), storage)
 
 
-def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False):
+def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
     if layer.op == "gat":
-        return gat_layer(indptr, indices, H, layer, storage)
-    return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder)
+        return gat_layer(indptr, indices, H, layer, storage, rows)
+    return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows)
 
 
 def will_reorder(layer) -> bool:
@@ -270,3 +311,24 @@ def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, f
                           reorder=follow_reorder and will_reorder(layer))
         outs.append(H)
     return outs
+
+
+def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, threshold=0, follow_reorder=False):
+    """The L-layer result at the vertices `targets` only, computed from their L-hop
+    in-neighbourhood (which is sufficient and necessary for an L-layer model, Section
+    "K-hop Neighborhood and Sampling"): layer l is evaluated only where layer l+1 reads it.
+    Everything else stays NaN, so a read outside the neighbourhood would poison the result.
+    Returns [len(targets), out_dim] in the order of `targets`."""
+    targets = _i64(targets)
+    need = [None] * (len(layers) + 1)
+    need[len(layers)] = np.unique(targets)
+    for l in range(len(layers) - 1, 0, -1):
+        need[l] = _sources_of(indptr, indices, need[l + 1])
+    H = _f64(X)
+    n = H.shape[0]
+    for l, layer in enumerate(layers, start=1):
+        out_rows = layer_forward(indptr, indices, edge_weights, H, layer, storage, threshold,
+                                 reorder=follow_reorder and will_reorder(layer), rows=need[l])
+        H = np.full((n, layer.out_dim), np.nan)
+        H[need[l]] = out_rows
+    return H[targets]

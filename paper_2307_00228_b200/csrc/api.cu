@@ -1,0 +1,192 @@
+// it_layer_forward / it_infer / it_workspace_bytes: argument checks, workspace carving and the
+// launch sequence of one layer.  All arithmetic lives in the kernels of the other files.
+#include "common.cuh"
+
+namespace {
+
+enum LayerPlan { PLAN_SAGE = 0, PLAN_SAGE_REORDER = 1, PLAN_GAT = 2 };
+
+struct LayerWs {
+  LayerPlan plan;
+  size_t off_B, off_partials, off_a, off_b;  // a: aggregate A | self term S | scores ; b: Z
+  size_t bytes;
+};
+
+it_status check_layer(const it_graph *g, const it_layer_desc *L) {
+  IT_REQUIRE(L != nullptr, IT_ERR_INVALID_ARG, "layer is NULL");
+  IT_REQUIRE(L->op >= IT_GATHER_SUM && L->op <= IT_GATHER_GAT, IT_ERR_INVALID_ARG, "bad gather op %d", (int)L->op);
+  IT_REQUIRE(L->act >= IT_ACT_NONE && L->act <= IT_ACT_ELU, IT_ERR_INVALID_ARG, "bad activation %d", (int)L->act);
+  IT_REQUIRE(L->feat_dtype == IT_F32 || L->feat_dtype == IT_BF16, IT_ERR_INVALID_ARG, "bad feat_dtype");
+  IT_REQUIRE(L->weight_dtype == L->feat_dtype, IT_ERR_UNSUPPORTED, "weight_dtype must equal feat_dtype");
+  IT_REQUIRE(L->in_dim > 0 && L->out_dim > 0, IT_ERR_INVALID_ARG, "dims must be positive");
+  const int s = it_dtype_size(L->feat_dtype);
+  IT_REQUIRE((L->in_dim * s) % 16 == 0 && (L->out_dim * s) % 16 == 0, IT_ERR_INVALID_ARG,
+             "feature rows must be a multiple of 16 bytes (in %d, out %d, %d-byte elements)", L->in_dim, L->out_dim, s);
+  if (L->op == IT_GATHER_GAT) {
+    IT_REQUIRE(L->heads >= 1 && L->out_dim % L->heads == 0, IT_ERR_INVALID_ARG, "out_dim must be heads * head_dim");
+    IT_REQUIRE(!L->use_edge_weights, IT_ERR_UNSUPPORTED, "GAT layers take no edge weights");
+  } else {
+    IT_REQUIRE(L->heads <= 1, IT_ERR_INVALID_ARG, "heads > 1 needs op = IT_GATHER_GAT");
+    IT_REQUIRE(!L->use_edge_weights || g->edge_weights, IT_ERR_INVALID_ARG, "layer uses edge weights but the graph has none");
+  }
+  return IT_OK;
+}
+
+bool reorders(const it_layer_desc *L) {
+  return L->allow_reorder && (L->op == IT_GATHER_SUM || L->op == IT_GATHER_MEAN) && L->out_dim < L->in_dim;
+}
+
+LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
+  LayerWs w;
+  const size_t n = (size_t)g->n, s = (size_t)it_dtype_size(L->feat_dtype);
+  const size_t fi = (size_t)L->in_dim, fo = (size_t)L->out_dim;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += it_align_up(bytes); return o; };
+  if (L->op == IT_GATHER_GAT) {
+    w.plan = PLAN_GAT;
+    w.off_B = take(fi * (fo + 2 * (size_t)L->heads) * 4);
+    w.off_partials = off;
+    w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
+    w.off_b = take(n * fo * s);                    // Z
+  } else if (reorders(L)) {
+    w.plan = PLAN_SAGE_REORDER;
+    w.off_B = take(fi * 2 * fo * 4);
+    w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
+    w.off_a = take(n * fo * 4);  // S (fp32)
+    w.off_b = take(n * fo * s);  // Z
+  } else {
+    w.plan = PLAN_SAGE;
+    w.off_B = take(2 * fi * fo * 4);
+    w.off_partials = take((size_t)g->n_partial_rows * fi * 4);
+    w.off_a = take(n * fi * s);  // A
+    w.off_b = off;
+  }
+  w.bytes = off;
+  return w;
+}
+
+it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const void *h_in, void *h_out, char *ws,
+                             size_t ws_bytes, cudaStream_t st) {
+  const LayerWs w = plan_layer(g, L);
+  IT_REQUIRE(ws_bytes >= w.bytes, IT_ERR_WORKSPACE, "workspace has %zu bytes, layer needs %zu", ws_bytes, w.bytes);
+  IT_REQUIRE(L->W != nullptr, IT_ERR_INVALID_ARG, "W is NULL");
+  float *B = reinterpret_cast<float *>(ws + w.off_B);
+  float *partials = g->n_partial_rows > 0 ? reinterpret_cast<float *>(ws + w.off_partials) : nullptr;
+  const it_dtype dt = L->feat_dtype;
+
+  if (w.plan == PLAN_GAT) {
+    IT_REQUIRE(L->att_src && L->att_dst, IT_ERR_INVALID_ARG, "GAT layer needs att_src and att_dst");
+    float *scores = reinterpret_cast<float *>(ws + w.off_a);
+    void *Z = ws + w.off_b;
+    IT_TRY(it_launch_prep_weights(IT_PREP_GAT, L, B, st));
+    it_gemm_args ga{};
+    ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
+    ga.B = B; ga.NB = L->out_dim + 2 * L->heads;
+    ga.n0 = 0; ga.out0 = nullptr; ga.dt0 = dt; ga.bias0 = nullptr; ga.act0 = IT_ACT_NONE;
+    ga.n1 = L->out_dim; ga.out1 = Z; ga.dt1 = dt; ga.out2 = scores;
+    IT_TRY(it_launch_gemm(ga, st));
+    it_gat_args aa{};
+    aa.g = g; aa.dtype = dt; aa.heads = L->heads; aa.head_dim = L->out_dim / L->heads; aa.z = Z; aa.scores = scores;
+    aa.slope = L->leaky_slope; aa.bias = L->bias; aa.act = L->act; aa.dst = h_out;
+    return it_launch_gat(aa, st);
+  }
+
+  it_gather_args gg{};
+  gg.g = g; gg.op = L->op; gg.use_edge_weights = L->use_edge_weights; gg.dtype = dt; gg.partials = partials;
+  if (w.plan == PLAN_SAGE_REORDER) {
+    float *S = reinterpret_cast<float *>(ws + w.off_a);
+    void *Z = ws + w.off_b;
+    IT_TRY(it_launch_prep_weights(IT_PREP_SAGE_REORDER, L, B, st));
+    it_gemm_args ga{};
+    ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
+    ga.B = B; ga.NB = 2 * L->out_dim;
+    ga.n0 = L->out_dim; ga.out0 = S; ga.dt0 = IT_F32; ga.bias0 = L->bias; ga.act0 = IT_ACT_NONE;
+    ga.n1 = L->out_dim; ga.out1 = Z; ga.dt1 = dt; ga.out2 = nullptr;
+    IT_TRY(it_launch_gemm(ga, st));
+    gg.dim = L->out_dim; gg.src = Z; gg.dst = h_out; gg.epi = IT_EPI_ADD_ACT; gg.self_term = S; gg.act = L->act;
+    return it_launch_gather(gg, st);
+  }
+  void *A = ws + w.off_a;
+  IT_TRY(it_launch_prep_weights(IT_PREP_SAGE, L, B, st));
+  gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.act = IT_ACT_NONE;
+  IT_TRY(it_launch_gather(gg, st));
+  it_gemm_args ga{};
+  ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = A; ga.K2 = L->in_dim;
+  ga.B = B; ga.NB = L->out_dim;
+  ga.n0 = L->out_dim; ga.out0 = h_out; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = L->act;
+  ga.n1 = 0; ga.out1 = nullptr; ga.dt1 = dt; ga.out2 = nullptr;
+  return it_launch_gemm(ga, st);
+}
+
+struct InferWs { size_t layer_bytes, buf_bytes, off_buf0, off_buf1, bytes; };
+
+it_status plan_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, InferWs *out) {
+  IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
+  IT_REQUIRE(layers != nullptr && n_layers >= 1, IT_ERR_INVALID_ARG, "need at least one layer");
+  InferWs w{0, 0, 0, 0, 0};
+  for (int i = 0; i < n_layers; ++i) {
+    IT_TRY(check_layer(g, &layers[i]));
+    if (i > 0) {
+      IT_REQUIRE(layers[i].in_dim == layers[i - 1].out_dim, IT_ERR_INVALID_ARG, "layer %d in_dim %d != layer %d out_dim %d", i,
+                 layers[i].in_dim, i - 1, layers[i - 1].out_dim);
+      IT_REQUIRE(layers[i].feat_dtype == layers[0].feat_dtype, IT_ERR_INVALID_ARG, "all layers must share feat_dtype");
+    }
+    size_t b = plan_layer(g, &layers[i]).bytes;
+    if (b > w.layer_bytes) w.layer_bytes = b;
+    if (i < n_layers - 1) {
+      size_t hb = it_align_up((size_t)g->n * (size_t)layers[i].out_dim * (size_t)it_dtype_size(layers[i].feat_dtype));
+      if (hb > w.buf_bytes) w.buf_bytes = hb;
+    }
+  }
+  w.off_buf0 = w.layer_bytes;
+  w.off_buf1 = w.off_buf0 + (n_layers >= 2 ? w.buf_bytes : 0);
+  w.bytes = w.off_buf1 + (n_layers >= 3 ? w.buf_bytes : 0);
+  *out = w;
+  return IT_OK;
+}
+
+bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
+  const char *x = (const char *)a, *y = (const char *)b;
+  return x < y + nb && y < x + na;
+}
+
+}  // namespace
+
+extern "C" it_status it_workspace_bytes(const it_graph *g, const it_layer_desc *layers, int32_t n_layers,
+                                        size_t *out_bytes) {
+  IT_REQUIRE(out_bytes != nullptr, IT_ERR_INVALID_ARG, "out_bytes is NULL");
+  InferWs w;
+  IT_TRY(plan_infer(g, layers, n_layers, &w));
+  *out_bytes = w.bytes > 0 ? w.bytes : 256;
+  return IT_OK;
+}
+
+extern "C" it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const void *h_in, void *h_out,
+                                      void *workspace, size_t workspace_bytes, void *stream) {
+  IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
+  IT_TRY(check_layer(g, layer));
+  IT_REQUIRE((h_in && h_out) || g->n == 0, IT_ERR_INVALID_ARG, "h_in / h_out is NULL");
+  IT_REQUIRE(workspace != nullptr && ((uintptr_t)workspace % 256) == 0, IT_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
+  const size_t s = (size_t)it_dtype_size(layer->feat_dtype);
+  IT_REQUIRE(g->n == 0 || !overlaps(h_in, (size_t)g->n * layer->in_dim * s, h_out, (size_t)g->n * layer->out_dim * s),
+             IT_ERR_INVALID_ARG, "h_in and h_out overlap");
+  return layer_forward_impl(g, layer, h_in, h_out, (char *)workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+extern "C" it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, const void *x, void *out,
+                              void *workspace, size_t workspace_bytes, void *stream) {
+  InferWs w;
+  IT_TRY(plan_infer(g, layers, n_layers, &w));
+  IT_REQUIRE((x && out) || g->n == 0, IT_ERR_INVALID_ARG, "x / out is NULL");
+  IT_REQUIRE(workspace != nullptr && ((uintptr_t)workspace % 256) == 0, IT_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
+  IT_REQUIRE(workspace_bytes >= w.bytes, IT_ERR_WORKSPACE, "workspace has %zu bytes, it_infer needs %zu", workspace_bytes, w.bytes);
+  char *ws = (char *)workspace;
+  void *buf[2] = {ws + w.off_buf0, ws + w.off_buf1};
+  const void *cur = x;
+  for (int i = 0; i < n_layers; ++i) {
+    void *dst = (i == n_layers - 1) ? out : buf[i & 1];
+    IT_TRY(layer_forward_impl(g, &layers[i], cur, dst, ws, w.layer_bytes, (cudaStream_t)stream));
+    cur = dst;
+  }
+  return IT_OK;
+}

@@ -1,0 +1,150 @@
+// Shared declarations of the layer-pass library (host + device helpers, the graph handle,
+// the launch entry points of each kernel file).  sm_100a only.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "inferturbo.h"
+
+#define IT_NUM_SMS_FALLBACK 148
+
+// ----------------------------------------------------------------------------- errors
+void it_set_error(const char *fmt, ...);
+
+#define IT_CUDA_TRY(expr)                                                            \
+  do {                                                                               \
+    cudaError_t _e = (expr);                                                         \
+    if (_e != cudaSuccess) {                                                         \
+      it_set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(_e), __FILE__, \
+                   __LINE__);                                                        \
+      return (_e == cudaErrorMemoryAllocation) ? IT_ERR_OOM : IT_ERR_CUDA;           \
+    }                                                                                \
+  } while (0)
+
+#define IT_TRY(expr)               \
+  do {                             \
+    it_status _s = (expr);         \
+    if (_s != IT_OK) return _s;    \
+  } while (0)
+
+#define IT_REQUIRE(cond, code, ...) \
+  do {                              \
+    if (!(cond)) {                  \
+      it_set_error(__VA_ARGS__);    \
+      return (code);                \
+    }                               \
+  } while (0)
+
+// ----------------------------------------------------------------------------- instrumentation
+enum it_kernel_id {
+  IT_K_VALIDATE = 0, IT_K_SPLIT_SCAN, IT_K_SPLIT_FILL, IT_K_BUCKET_SCAN, IT_K_PREP, IT_K_GATHER_CTA, IT_K_GATHER_WARP,
+  IT_K_GATHER_SUBWARP, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_WARP, IT_K_GAT_SUBWARP,
+  IT_K_COUNT
+};
+// Wraps one kernel launch: counts it and, while profiling is on, brackets it with events on `st`.
+struct it_prof_scope {
+  it_prof_scope(int kid, double algo_bytes, double algo_flops, cudaStream_t st);
+  ~it_prof_scope();
+  int slot_;
+  cudaStream_t st_;
+};
+#define IT_LAUNCH(kid, bytes, flops, st, ...) \
+  do {                                        \
+    it_prof_scope _scope((kid), (bytes), (flops), (st)); \
+    __VA_ARGS__;                              \
+  } while (0)
+
+// ----------------------------------------------------------------------------- graph handle
+struct it_graph {
+  int64_t n = 0, e = 0;
+  const void *indptr = nullptr;
+  it_itype indptr_type = IT_I64;
+  const int32_t *indices = nullptr;
+  const float *edge_weights = nullptr;
+  int device = 0;
+  int num_sms = IT_NUM_SMS_FALLBACK;
+
+  // derived by the split (library-owned, device)
+  int64_t threshold = 0;
+  int64_t n_rows = 0;           // R
+  int64_t n_split_owners = 0;   // vertices with more than one shadow row
+  int64_t n_partial_rows = 0;   // shadow rows that belong to split owners
+  int64_t *shadow_indptr = nullptr;  // [R+1]
+  int32_t *shadow_owner = nullptr;   // [R]
+  int64_t *owner_indptr = nullptr;   // [n+1]
+  int32_t *row_dest = nullptr;       // [R]  v >= 0: row is the whole segment of v; < 0: ~index into the partial buffer
+  int32_t *split_owners = nullptr;   // [n_split_owners] ascending vertex ids
+  int32_t n_buckets = 0;
+  int64_t bucket_bounds[IT_MAX_BUCKETS] = {0};
+  int64_t h_bucket_offsets[IT_MAX_BUCKETS + 1] = {0};
+  int64_t h_bucket_edges[IT_MAX_BUCKETS] = {0};  // edges held by the rows of each bucket
+  int64_t *bucket_offsets = nullptr;  // device [n_buckets+1]
+  int32_t *bucket_rows = nullptr;     // [R]
+};
+
+static inline size_t it_align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+static inline int it_dtype_size(it_dtype t) { return t == IT_F32 ? 4 : 2; }
+
+// ----------------------------------------------------------------------------- gather.cu
+// What a gather / combine kernel does with the finished aggregate of vertex v.
+enum it_epilogue_kind {
+  IT_EPI_STORE = 0,      // dst[v, :] = agg                      (feat dtype)
+  IT_EPI_ADD_ACT = 1     // dst[v, :] = act(self[v, :] + agg)    (self fp32, dst feat dtype)
+};
+
+struct it_gather_args {
+  const it_graph *g;
+  it_gather_op op;         // SUM / MEAN / MAX
+  int use_edge_weights;
+  it_dtype dtype;          // of src rows and of dst rows
+  int dim;                 // row length in elements
+  const void *src;         // [n, dim] rows that are gathered
+  float *partials;         // [n_partial_rows, dim] fp32 scratch (may be NULL when nothing is split)
+  void *dst;               // [n, dim]
+  it_epilogue_kind epi;
+  const float *self_term;  // [n, dim] fp32, IT_EPI_ADD_ACT only
+  it_act act;              // IT_EPI_ADD_ACT only
+};
+it_status it_launch_gather(const it_gather_args &a, cudaStream_t stream);
+
+// ----------------------------------------------------------------------------- gat.cu
+struct it_gat_args {
+  const it_graph *g;
+  it_dtype dtype;
+  int heads, head_dim;
+  const void *z;          // [n, heads*head_dim] messages
+  const float *scores;    // [n, 2*heads]: source scores of the vertex, then its destination scores
+  float slope;
+  const float *bias;      // may be NULL
+  it_act act;
+  void *dst;              // [n, heads*head_dim]
+};
+it_status it_launch_gat(const it_gat_args &a, cudaStream_t stream);
+
+// ----------------------------------------------------------------------------- apply.cu
+// C[M, NB] = X1[M, K1] * B[0:K1, :] + X2[M, K2] * B[K1:K1+K2, :]   (X2 may be NULL, K2 = 0)
+// B is an fp32 [K1+K2, NB] matrix assembled by it_launch_prep_weights.  Column ranges of C
+// go to up to three destinations:
+//   [0, n0)        -> out0 (dtype dt0) = act0(C + bias0)
+//   [n0, n0+n1)    -> out1 (dtype dt1), raw
+//   [n0+n1, NB)    -> out2 (fp32), raw, row stride n2 = NB - n0 - n1
+struct it_gemm_args {
+  int64_t M;
+  it_dtype x_dtype;
+  const void *X1; int K1;
+  const void *X2; int K2;
+  const float *B; int NB;
+  int n0; void *out0; it_dtype dt0; const float *bias0; it_act act0;
+  int n1; void *out1; it_dtype dt1;
+  void *out2;
+};
+it_status it_launch_gemm(const it_gemm_args &a, cudaStream_t stream);
+
+enum it_prep_kind { IT_PREP_SAGE = 0, IT_PREP_SAGE_REORDER = 1, IT_PREP_GAT = 2 };
+// Assemble the fp32 B matrix for a layer: SAGE [2*in, out] copy; REORDER [in, 2*out] =
+// [W_self | W_neigh]; GAT [in, out + 2*heads] = [W | W a_src | W a_dst].
+it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *layer, float *B,
+                                 cudaStream_t stream);

@@ -1,0 +1,85 @@
+"""Helpers shared by the GPU parity tests: run a workload through the C ABI and through the
+oracle and compare.  The oracle never sees a value produced by the CUDA path."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import oracle as O
+from paper_2307_00228_b200 import binding as B
+from paper_2307_00228_b200 import host
+from workloads import Layer, Workload, compare
+from workloads import rng as wrng
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}   # max relative error: fp32 paths / bf16 apply paths
+
+
+def to_numpy(t: torch.Tensor) -> np.ndarray:
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def storage_exact(a: np.ndarray, dtype: str) -> np.ndarray:
+    """float32 values that are exactly representable in the storage dtype."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return wrng.bf16_bits_to_f32(wrng.f32_to_bf16_bits(a)) if dtype == "bf16" else a
+
+
+def small_workload(seed, n, max_deg, dtype, layers, hubs=(), weights=False, threshold=0, p_zero=0.2) -> Workload:
+    rng = np.random.default_rng(seed)
+    deg = rng.integers(0, max_deg + 1, size=n)
+    deg[rng.random(n) < p_zero] = 0
+    for i, d in enumerate(hubs):
+        deg[(7 * i + 3) % n] = d
+    indptr = np.zeros(n + 1, np.int64)
+    np.cumsum(deg, out=indptr[1:])
+    e = int(indptr[-1])
+    indices = rng.integers(0, n, size=e).astype(np.int32)
+    w = rng.random(e, dtype=np.float32) if weights else None
+    x = rng.standard_normal((n, layers[0].in_dim)).astype(np.float32)
+    xs = x if dtype == "f32" else wrng.f32_to_bf16_bits(x)
+    return Workload("small", n, e, indptr, indices, w, dtype, xs, layers, threshold)
+
+
+def make_sage_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=True, bias=True) -> Layer:
+    rng = np.random.default_rng(seed)
+    lim = np.sqrt(6.0 / (2 * fi + fo))
+    return Layer(op=op, act=act, in_dim=fi, out_dim=fo,
+                 W=storage_exact(rng.uniform(-lim, lim, (2 * fi, fo)), dtype),
+                 bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None,
+                 use_edge_weights=weights, allow_reorder=allow_reorder)
+
+
+def make_gat_layer(seed, act, fi, heads, hd, dtype, bias=True) -> Layer:
+    rng = np.random.default_rng(seed)
+    fo = heads * hd
+    lim = np.sqrt(6.0 / (fi + fo))
+    return Layer(op="gat", act=act, in_dim=fi, out_dim=fo, W=storage_exact(rng.uniform(-lim, lim, (fi, fo)), dtype),
+                 bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None, heads=heads,
+                 att_src=rng.uniform(-0.4, 0.4, (heads, hd)).astype(np.float32),
+                 att_dst=rng.uniform(-0.4, 0.4, (heads, hd)).astype(np.float32))
+
+
+def run_device(w: Workload, int32_indptr=False, threshold=None):
+    """it_infer through the C ABI; returns (final output as fp64 numpy, DeviceWorkload)."""
+    d = host.upload(w, int32_indptr=int32_indptr, threshold=threshold)
+    d.infer()
+    torch.cuda.synchronize()
+    return to_numpy(d.out), d
+
+
+def run_oracle(w: Workload, storage="same", threshold=None):
+    """Oracle over all layers.  storage='same': round at the storage points like the device
+    contract (mode B); storage=None: fp64 throughout (mode A)."""
+    st = w.dtype if storage == "same" else storage
+    thr = w.threshold if threshold is None else threshold
+    return O.infer(w.indptr, w.indices, w.edge_weights, w.x_as_f32(), w.layers, storage=st, threshold=thr,
+                   follow_reorder=True)
+
+
+def check_against_oracle(w: Workload, got: np.ndarray, tol=None, label=""):
+    ref = run_oracle(w)[-1]
+    err = compare.rel_error(got, ref)
+    tol = TOL[w.dtype] if tol is None else tol
+    assert err["finite"], label
+    assert err["max_rel"] <= tol, (label, err)
+    return err

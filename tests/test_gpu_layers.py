@@ -1,0 +1,195 @@
+"""Parity of the CUDA layer pass with the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import (TOL, check_against_oracle, make_gat_layer, make_sage_layer, run_device, run_oracle,
+                      small_workload, to_numpy)
+from paper_2307_00228_b200 import binding as B
+from paper_2307_00228_b200 import host
+from workloads import compare
+
+pytestmark = pytest.mark.gpu
+
+HUBS = (257, 300, 1000, 2500, 33, 32, 9, 8, 1)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("op", ["sum", "mean", "max"])
+@pytest.mark.parametrize("weights", [False, True])
+@pytest.mark.parametrize("threshold", [0, 64, 1000])
+def test_sage_layer_parity(dtype, op, weights, threshold):
+    # 1500 vertices: several 128-row GEMM tiles and a ragged tail; every degree bucket is populated
+    fi, fo = 64, 32
+    for reorder in ([False, True] if op != "max" else [False]):
+        layer = make_sage_layer(1, op, "relu", fi, fo, dtype, weights=weights, allow_reorder=reorder)
+        w = small_workload(2, 1500, 40, dtype, [layer], hubs=HUBS, weights=weights, threshold=threshold)
+        got, d = run_device(w)
+        if threshold:
+            assert d.n_split_owners > 0
+        check_against_oracle(w, got, label=(dtype, op, weights, threshold, reorder))
+
+
+@pytest.mark.parametrize("dtype,dims", [("f32", (4, 4)), ("f32", (8, 16)), ("f32", (16, 8)), ("f32", (32, 64)), ("f32", (128, 128)),
+                                        ("f32", (128, 64)), ("bf16", (8, 8)), ("bf16", (16, 64)), ("bf16", (64, 128)),
+                                        ("bf16", (128, 64)), ("bf16", (256, 32))])
+def test_every_supported_row_width(dtype, dims):
+    fi, fo = dims
+    for op in ("mean", "max"):
+        layer = make_sage_layer(3, op, "none", fi, fo, dtype)
+        w = small_workload(4, 700, 20, dtype, [layer], hubs=(400, 90), threshold=128)
+        got, _ = run_device(w)
+        check_against_oracle(w, got, label=(dtype, dims, op))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("act", ["none", "relu", "elu"])
+def test_gat_layer_parity(dtype, act):
+    layer = make_gat_layer(5, act, 64, 4, 32, dtype)
+    w = small_workload(6, 1300, 30, dtype, [layer], hubs=HUBS)
+    got, _ = run_device(w)
+    check_against_oracle(w, got, label=(dtype, act))
+
+
+@pytest.mark.parametrize("heads,hd", [(1, 8), (2, 16), (8, 8), (1, 128), (4, 32)])
+def test_gat_head_shapes(heads, hd):
+    layer = make_gat_layer(7, "elu", 32, heads, hd, "bf16")
+    w = small_workload(8, 500, 12, "bf16", [layer], hubs=(300, 40))
+    got, _ = run_device(w)
+    check_against_oracle(w, got, label=(heads, hd))
+
+
+def test_gat_large_scores_do_not_overflow():
+    layer = make_gat_layer(9, "none", 16, 2, 8, "f32")
+    layer.att_src *= 200.0
+    layer.att_dst *= 200.0
+    w = small_workload(10, 400, 25, "f32", [layer], hubs=(300,))
+    got, _ = run_device(w)
+    assert np.isfinite(got).all()
+    check_against_oracle(w, got, tol=1e-3)   # exp of large score differences: looser than the plain fp32 bound
+
+
+def test_gat_refuses_a_split_graph():
+    layer = make_gat_layer(9, "none", 16, 2, 8, "f32")
+    w = small_workload(10, 400, 25, "f32", [layer], hubs=(300,), threshold=16)
+    with pytest.raises(B.ItError) as ei:
+        run_device(w)
+    assert ei.value.status_name == "IT_ERR_UNSUPPORTED"
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_multi_layer_infer_matches_layer_by_layer_and_oracle(dtype):
+    layers = [make_sage_layer(11, "mean", "relu", 32, 64, dtype), make_sage_layer(12, "sum", "relu", 64, 32, dtype, weights=True),
+              make_sage_layer(13, "max", "none", 32, 16, dtype)]
+    w = small_workload(14, 2100, 16, dtype, layers, hubs=HUBS, weights=True, threshold=100)
+    got, d = run_device(w)
+    check_against_oracle(w, got)
+    # exactly the sequence of it_layer_forward calls: bit-identical
+    h = d.x
+    for lay, src in zip(d.layers, w.layers):
+        ws = torch.empty(B.it_workspace_bytes(d.graph, [lay]), dtype=torch.uint8, device="cuda")
+        o = torch.empty((w.n, src.out_dim), dtype=d.x.dtype, device="cuda")
+        B.it_layer_forward(d.graph, lay, h, o, ws)
+        h = o
+    torch.cuda.synchronize()
+    assert torch.equal(h, d.out)
+
+
+def test_run_to_run_results_are_bit_identical():
+    """The paper's consistency requirement: the same prediction at every run."""
+    layers = [make_sage_layer(15, "sum", "relu", 64, 64, "f32", weights=True), make_sage_layer(16, "mean", "none", 64, 16, "f32")]
+    w = small_workload(17, 3000, 30, "f32", layers, hubs=HUBS, weights=True, threshold=64)
+    d = host.upload(w)
+    outs = []
+    for _ in range(4):
+        d.out.zero_()
+        d.workspace.random_(0, 255)          # stale scratch must not matter
+        d.infer()
+        torch.cuda.synchronize()
+        outs.append(d.out.clone())
+    assert all(torch.equal(outs[0], o) for o in outs[1:])
+
+
+def test_split_does_not_change_max_and_integer_sums():
+    """Partial gather + combine: exact for max, and for sums of small integers."""
+    lay_max = make_sage_layer(18, "max", "none", 32, 32, "f32")
+    lay_sum = make_sage_layer(19, "sum", "none", 32, 32, "f32")
+    for lay in (lay_max, lay_sum):
+        lay.W[:] = 0
+        lay.W[32:] = np.eye(32, dtype=np.float32)   # output = the aggregate itself
+        lay.bias = None
+        w = small_workload(20, 900, 25, "f32", [lay], hubs=(2000, 513))
+        w.x = np.round(w.x * 4).astype(np.float32)
+        base, _ = run_device(w, threshold=0)
+        for T in (1, 7, 64, 512):
+            got, _ = run_device(w, threshold=T)
+            assert np.array_equal(got, base), (lay.op, T)
+        assert np.array_equal(base, run_oracle(w, storage=None)[-1])
+
+
+def test_int32_and_int64_indptr_agree():
+    layer = make_sage_layer(21, "mean", "relu", 64, 64, "bf16")
+    w = small_workload(22, 1000, 20, "bf16", [layer], hubs=(600,), threshold=128)
+    a, _ = run_device(w, int32_indptr=False)
+    b, _ = run_device(w, int32_indptr=True)
+    assert np.array_equal(a, b)
+
+
+def test_degenerate_inputs():
+    layer = make_sage_layer(23, "mean", "relu", 16, 16, "f32")
+    # no edges at all: output = act(x W_self + b)
+    w = small_workload(24, 300, 0, "f32", [layer])
+    assert w.e == 0
+    got, _ = run_device(w)
+    check_against_oracle(w, got)
+    # a single vertex with a self-loop and a multi-edge
+    w = small_workload(25, 1, 0, "f32", [layer])
+    w.indptr = np.array([0, 3], np.int64)
+    w.indices = np.zeros(3, np.int32)
+    w.e = 3
+    got, _ = run_device(w)
+    check_against_oracle(w, got)
+    # every vertex has exactly one in-edge
+    w = small_workload(26, 257, 1, "f32", [layer], p_zero=0.0)
+    got, _ = run_device(w)
+    check_against_oracle(w, got)
+
+
+def test_error_statuses():
+    layer = make_sage_layer(27, "sum", "relu", 16, 16, "f32", weights=True)
+    w = small_workload(28, 100, 5, "f32", [layer], weights=True)
+    d = host.upload(w)
+    out = torch.empty((w.n, 16), device="cuda")
+
+    def status_of(fn):
+        with pytest.raises(B.ItError) as ei:
+            fn()
+        return ei.value.status_name
+
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], d.x, out, small)) == "IT_ERR_WORKSPACE"
+    assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], d.x, d.x, d.workspace)) == "IT_ERR_INVALID_ARG"
+    misaligned = d.workspace[1:]
+    assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], d.x, out, misaligned)) == "IT_ERR_WORKSPACE"
+    bad = host.layer_to_device(make_sage_layer(29, "sum", "relu", 6, 16, "f32"), "f32")   # 24-byte rows
+    assert status_of(lambda: B.it_workspace_bytes(d.graph, [bad])) == "IT_ERR_INVALID_ARG"
+    mism = [d.layers[0], host.layer_to_device(make_sage_layer(30, "sum", "relu", 32, 16, "f32"), "f32")]
+    assert status_of(lambda: B.it_workspace_bytes(d.graph, mism)) == "IT_ERR_INVALID_ARG"
+    # edge weights requested from a graph that has none
+    w2 = small_workload(28, 100, 5, "f32", [layer], weights=False)
+    assert status_of(lambda: host.upload(w2)) == "IT_ERR_INVALID_ARG"
+    assert torch.ones(4, device="cuda").sum().item() == 4
+
+
+def test_mode_a_error_is_reported_and_bounded():
+    """Against the exact fp64 oracle (no rounding at storage points) the bf16 path stays within a few bf16 ulps per layer."""
+    layers = [make_sage_layer(31, "mean", "relu", 64, 64, "bf16"), make_sage_layer(32, "mean", "none", 64, 32, "bf16")]
+    w = small_workload(33, 2000, 20, "bf16", layers, hubs=(700,), threshold=256)
+    got, _ = run_device(w)
+    err = compare.rel_error(got, run_oracle(w, storage=None)[-1])
+    assert err["max_rel"] < 5e-2
+    # and the fp32 path is far tighter
+    layers = [make_sage_layer(31, "mean", "relu", 64, 64, "f32"), make_sage_layer(32, "mean", "none", 64, 32, "f32")]
+    w = small_workload(33, 2000, 20, "f32", layers, hubs=(700,), threshold=256)
+    got, _ = run_device(w)
+    assert compare.rel_error(got, run_oracle(w, storage=None)[-1])["max_rel"] < TOL["f32"]

@@ -476,3 +476,28 @@ def test_storage_mode_stays_close_to_exact_mode():
         b = O.infer(ip, ix, None, X, layers, storage=storage, threshold=7, follow_reorder=True)[-1]
         assert np.abs(a - b).max() / np.sqrt((a ** 2).mean()) < tol
         assert not np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "gat"])
+def test_infer_at_targets_equals_full_graph_inference(op):
+    """Evaluating only the L-hop in-neighbourhood of some targets gives the full-graph values
+    there (and reads nothing else: untouched rows are NaN)."""
+    rng = np.random.default_rng(21)
+    n = 400
+    ip, ix = random_graph(rng, n, 6)
+    w = rng.random(ix.shape[0])
+    X = rng.standard_normal((n, 8))
+    if op == "gat":
+        layers = [L("gat", "elu", rng.standard_normal((8, 8)) * .3, rng.standard_normal(8) * .1, 2,
+                    rng.standard_normal((2, 4)) * .3, rng.standard_normal((2, 4)) * .3) for _ in range(2)]
+    else:
+        layers = [L(op, "relu", rng.standard_normal((16, 8)) * .3, rng.standard_normal(8) * .1, use_edge_weights=True),
+                  L(op, "none", rng.standard_normal((16, 4)) * .3, rng.standard_normal(4) * .1, use_edge_weights=True)]
+    targets = rng.permutation(n)[:25]
+    for storage in (None, "bf16"):
+        for thr in (0, 3):
+            if op == "gat" and thr:
+                continue
+            full = O.infer(ip, ix, w, X, layers, storage=storage, threshold=thr, follow_reorder=True)[-1]
+            part = O.infer_at(ip, ix, w, X, layers, targets, storage=storage, threshold=thr, follow_reorder=True)
+            assert np.array_equal(part, full[targets])
