@@ -171,7 +171,7 @@ class _DevArray:
     """Minimal __cuda_array_interface__ holder so torch can view library-owned device memory."""
 
     def __init__(self, ptr, count, typestr):
-        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, True), "version": 2}
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, False), "version": 2}
 
 
 def _borrow(ptr, count, dtype, device):
