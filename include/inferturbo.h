@@ -160,6 +160,37 @@ it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const 
 it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, const void *x,
                    void *out, void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * it_layer_forward_static — it_layer_forward for callers that must not allocate device
+ * memory (the paper has no counterpart: its workers allocate freely on CPU hosts).
+ *
+ * Who needs it: code that runs where cudaMalloc is unavailable or forbidden — inside a
+ * latency-critical serving loop that has frozen its memory pool, inside a host callback, or in
+ * a process whose device memory is handed out entirely by another component — and that
+ * therefore cannot obtain the scratch `workspace` that it_layer_forward asks for.  Here the
+ * scratch is a fixed array of IT_STATIC_WORKSPACE_BYTES that is part of the library image:
+ * every GPU that loads the library holds those bytes until the process exits, whether or not
+ * this call is ever made, which is why the limit is modest.
+ *
+ * Same arguments, results and errors as it_layer_forward, minus the workspace.  A layer whose
+ * scratch need (it_workspace_bytes of that one layer) exceeds IT_STATIC_WORKSPACE_BYTES is
+ * rejected with IT_ERR_WORKSPACE and nothing is launched.  The call itself performs no
+ * cudaMalloc / cudaFree and calls no allocating routine; for that reason it refuses to run
+ * (IT_ERR_UNSUPPORTED) while it_profile_begin instrumentation is active, since that creates
+ * CUDA events on demand.  (it_graph_create / it_split_hubs do allocate: build the graph
+ * during set-up.)
+ *
+ * The first call on each device looks up the device address of the array (with that device
+ * current) and caches it; make that first call during set-up, before any stream capture.
+ * All calls on a device share the one array.  It keeps the previous call's contents; nothing
+ * in it needs to start at zero, because every kernel writes the part it later reads.  Two
+ * calls whose kernels can overlap on the GPU (different streams without an ordering between
+ * them) race on the array: serialise them.
+ */
+#define IT_STATIC_WORKSPACE_BYTES (32u << 20)
+it_status it_layer_forward_static(const it_graph *g, const it_layer_desc *layer, const void *h_in,
+                                  void *h_out, void *stream);
+
 /* Frees the library-owned arrays of the graph.  NULL is accepted. */
 it_status it_graph_destroy(it_graph *g);
 

@@ -24,7 +24,7 @@ ACTS = {"none": 0, "relu": 1, "elu": 2}
 IT_MAX_BUCKETS = 8
 EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspace_bytes", "it_layer_forward",
            "it_infer", "it_graph_destroy", "it_status_string", "it_last_error_message", "it_profile_begin",
-           "it_profile_end", "it_kernel_launch_count"]
+           "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static"]
 
 
 class ItError(RuntimeError):
@@ -214,6 +214,23 @@ def it_layer_forward(g: Graph, layer, h_in: torch.Tensor, h_out: torch.Tensor, w
     arr = _c_layers([layer])
     _check(lib().it_layer_forward(g.handle, arr, _ptr(h_in), _ptr(h_out), _ptr(workspace),
                                   workspace.numel() * workspace.element_size(), _stream(stream)))
+    return h_out
+
+
+STATIC_WORKSPACE_BYTES = 32 << 20
+
+
+def it_layer_forward_static(g: Graph, layer, h_in: torch.Tensor, h_out: torch.Tensor, stream=None):
+    """it_layer_forward without a caller workspace, for callers that cannot allocate device
+    memory: the scratch is a fixed STATIC_WORKSPACE_BYTES array inside the library, shared by
+    all calls on a device (so calls that could overlap on the GPU must be serialised).  Layers
+    that need more scratch raise ItError(IT_ERR_WORKSPACE).  Make the first call during set-up."""
+    assert h_in.is_contiguous() and h_out.is_contiguous()
+    L = lib()
+    L.it_layer_forward_static.restype = C.c_int
+    L.it_layer_forward_static.argtypes = [C.c_void_p, C.POINTER(it_layer_desc), C.c_void_p, C.c_void_p, C.c_void_p]
+    arr = _c_layers([layer])
+    _check(L.it_layer_forward_static(g.handle, arr, _ptr(h_in), _ptr(h_out), _stream(stream)))
     return h_out
 
 

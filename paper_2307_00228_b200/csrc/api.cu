@@ -1,5 +1,7 @@
 // it_layer_forward / it_infer / it_workspace_bytes: argument checks, workspace carving and the
 // launch sequence of one layer.  All arithmetic lives in the kernels of the other files.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -171,6 +173,52 @@ extern "C" it_status it_layer_forward(const it_graph *g, const it_layer_desc *la
   IT_REQUIRE(g->n == 0 || !overlaps(h_in, (size_t)g->n * layer->in_dim * s, h_out, (size_t)g->n * layer->out_dim * s),
              IT_ERR_INVALID_ARG, "h_in and h_out overlap");
   return layer_forward_impl(g, layer, h_in, h_out, (char *)workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+// ----------------------------------------------------------------------------- no-allocation variant
+// Scratch for it_layer_forward_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address; kernels receive the looked-up pointer.
+static __device__ __align__(256) unsigned char g_static_workspace[IT_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void *g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_workspace on the current device (looked up once per device).
+it_status static_workspace_ptr(void **out) {
+  int dev = -1;
+  IT_CUDA_TRY(cudaGetDevice(&dev));
+  IT_REQUIRE(dev >= 0 && dev < kMaxDevices, IT_ERR_UNSUPPORTED, "device ordinal %d is beyond %d", dev, kMaxDevices);
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void *p = nullptr;
+    IT_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_workspace));
+    IT_REQUIRE(p != nullptr && ((uintptr_t)p % 256) == 0, IT_ERR_CUDA, "built-in scratch has no usable device address");
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return IT_OK;
+}
+}  // namespace
+
+extern "C" it_status it_layer_forward_static(const it_graph *g, const it_layer_desc *layer, const void *h_in,
+                                             void *h_out, void *stream) {
+  IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
+  IT_TRY(check_layer(g, layer));
+  IT_REQUIRE((h_in && h_out) || g->n == 0, IT_ERR_INVALID_ARG, "h_in / h_out is NULL");
+  const size_t s = (size_t)it_dtype_size(layer->feat_dtype);
+  IT_REQUIRE(g->n == 0 || !overlaps(h_in, (size_t)g->n * layer->in_dim * s, h_out, (size_t)g->n * layer->out_dim * s),
+             IT_ERR_INVALID_ARG, "h_in and h_out overlap");
+  IT_REQUIRE(!it_profile_is_on(), IT_ERR_UNSUPPORTED,
+             "it_layer_forward_static does not run while instrumentation is on (it would create CUDA events)");
+  const size_t need = plan_layer(g, layer).bytes;
+  IT_REQUIRE(need <= (size_t)IT_STATIC_WORKSPACE_BYTES, IT_ERR_WORKSPACE,
+             "layer needs %zu bytes of scratch, the built-in array holds %zu; use it_layer_forward with a caller workspace",
+             need, (size_t)IT_STATIC_WORKSPACE_BYTES);
+  void *ws = nullptr;
+  IT_TRY(static_workspace_ptr(&ws));
+  return layer_forward_impl(g, layer, h_in, h_out, (char *)ws, (size_t)IT_STATIC_WORKSPACE_BYTES, (cudaStream_t)stream);
 }
 
 extern "C" it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, const void *x, void *out,

@@ -51,6 +51,7 @@ struct it_prof_scope {
   int slot_;
   cudaStream_t st_;
 };
+bool it_profile_is_on();
 #define IT_LAUNCH(kid, bytes, flops, st, ...) \
   do {                                        \
     it_prof_scope _scope((kid), (bytes), (flops), (st)); \

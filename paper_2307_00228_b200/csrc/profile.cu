@@ -38,6 +38,11 @@ it_prof_scope::~it_prof_scope() {
   if (slot_ < (int)g_slots.size()) cudaEventRecord(g_slots[slot_].b, st_);
 }
 
+bool it_profile_is_on() {
+  std::lock_guard<std::mutex> lk(g_mu);
+  return g_on;
+}
+
 extern "C" int64_t it_kernel_launch_count(void) {
   std::lock_guard<std::mutex> lk(g_mu);
   return g_launches;
