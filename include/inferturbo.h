@@ -191,6 +191,15 @@ it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_lay
 it_status it_layer_forward_static(const it_graph *g, const it_layer_desc *layer, const void *h_in,
                                   void *h_out, void *stream);
 
+/*
+ * it_graph_check — waits for `stream` and reports whether any kernel launched for this graph
+ * since the last check gave up one of its bounded device-side waits (the tensor-core apply
+ * waits on hardware barriers with an iteration limit instead of spinning for ever).
+ * Returns IT_ERR_TIMEOUT in that case (and clears the condition): outputs written since the
+ * last check are then not valid.  IT_OK otherwise.  No counterpart in the paper.
+ */
+it_status it_graph_check(it_graph *g, void *stream);
+
 /* Frees the library-owned arrays of the graph.  NULL is accepted. */
 it_status it_graph_destroy(it_graph *g);
 

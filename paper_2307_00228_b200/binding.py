@@ -12,7 +12,7 @@ from dataclasses import dataclass
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libinferturbo.so")
+LIB_PATH = os.environ.get("INFERTURBO_LIB") or os.path.join(_PKG, "libinferturbo.so")
 
 IT_OK = 0
 STATUS_NAMES = ["IT_OK", "IT_ERR_INVALID_ARG", "IT_ERR_BAD_GRAPH", "IT_ERR_UNSUPPORTED", "IT_ERR_WORKSPACE",
@@ -24,7 +24,7 @@ ACTS = {"none": 0, "relu": 1, "elu": 2}
 IT_MAX_BUCKETS = 8
 EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspace_bytes", "it_layer_forward",
            "it_infer", "it_graph_destroy", "it_status_string", "it_last_error_message", "it_profile_begin",
-           "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static"]
+           "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static", "it_graph_check"]
 
 
 class ItError(RuntimeError):
@@ -240,6 +240,14 @@ def it_infer(g: Graph, layers, x: torch.Tensor, out: torch.Tensor, workspace: to
     _check(lib().it_infer(g.handle, arr, len(layers), _ptr(x), _ptr(out), _ptr(workspace),
                           workspace.numel() * workspace.element_size(), _stream(stream)))
     return out
+
+
+def it_graph_check(g: Graph, stream=None):
+    """Synchronise the stream; raises ItError(IT_ERR_TIMEOUT) if a kernel gave up a bounded wait."""
+    L = lib()
+    L.it_graph_check.restype = C.c_int
+    L.it_graph_check.argtypes = [C.c_void_p, C.c_void_p]
+    _check(L.it_graph_check(g.handle, _stream(stream)))
 
 
 def it_graph_destroy(g: Graph):

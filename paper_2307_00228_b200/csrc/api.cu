@@ -46,25 +46,43 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
   auto take = [&](size_t bytes) { size_t o = off; off += it_align_up(bytes); return o; };
   if (L->op == IT_GATHER_GAT) {
     w.plan = PLAN_GAT;
-    w.off_B = take(fi * (fo + 2 * (size_t)L->heads) * 4);
+    w.off_B = take(fi * (fo + 2 * (size_t)L->heads) * 8);
     w.off_partials = off;
     w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
     w.off_b = take(n * fo * s);                    // Z
   } else if (reorders(L)) {
     w.plan = PLAN_SAGE_REORDER;
-    w.off_B = take(fi * 2 * fo * 4);
+    w.off_B = take(fi * 2 * fo * 8);
     w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
     w.off_a = take(n * fo * 4);  // S (fp32)
     w.off_b = take(n * fo * s);  // Z
   } else {
     w.plan = PLAN_SAGE;
-    w.off_B = take(2 * fi * fo * 4);
+    w.off_B = take(2 * fi * fo * 8);
     w.off_partials = take((size_t)g->n_partial_rows * fi * 4);
     w.off_a = take(n * fi * s);  // A
     w.off_b = off;
   }
   w.bytes = off;
   return w;
+}
+
+// The dense transform of a layer: on the tensor cores when the shape allows it, otherwise the
+// fp32 CUDA-core kernel.  `ga` is filled for the CUDA-core kernel (for GAT: NB includes the
+// 2*heads score columns and out2 = scores); the tensor-core kernel derives its own view.
+it_status run_apply(const it_graph *g, const it_layer_desc *L, it_prep_kind kind, it_gemm_args ga, float *B,
+                    float *scores, cudaStream_t st) {
+  const int K = ga.K1 + (ga.X2 ? ga.K2 : 0);
+  const bool want_scores = kind == IT_PREP_GAT;
+  const int heads = L->heads > 0 ? L->heads : 1, hd = L->out_dim / heads;
+  if (it_tc_supported(ga, heads, hd, want_scores)) {
+    IT_TRY(it_launch_prep_weights_tc(kind, L, ga.n0 + ga.n1, K, B, st));
+    return it_launch_gemm_tc(ga, B, L->att_src, L->att_dst, heads, hd, want_scores ? scores : nullptr, g->num_sms,
+                             g->d_status, st);
+  }
+  ga.B = B;
+  IT_TRY(it_launch_prep_weights(kind, L, B, st));
+  return it_launch_gemm(ga, st);
 }
 
 it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const void *h_in, void *h_out, char *ws,
@@ -80,13 +98,12 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
     IT_REQUIRE(L->att_src && L->att_dst, IT_ERR_INVALID_ARG, "GAT layer needs att_src and att_dst");
     float *scores = reinterpret_cast<float *>(ws + w.off_a);
     void *Z = ws + w.off_b;
-    IT_TRY(it_launch_prep_weights(IT_PREP_GAT, L, B, st));
     it_gemm_args ga{};
     ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
     ga.B = B; ga.NB = L->out_dim + 2 * L->heads;
     ga.n0 = 0; ga.out0 = nullptr; ga.dt0 = dt; ga.bias0 = nullptr; ga.act0 = IT_ACT_NONE;
     ga.n1 = L->out_dim; ga.out1 = Z; ga.dt1 = dt; ga.out2 = scores;
-    IT_TRY(it_launch_gemm(ga, st));
+    IT_TRY(run_apply(g, L, IT_PREP_GAT, ga, B, scores, st));
     it_gat_args aa{};
     aa.g = g; aa.dtype = dt; aa.heads = L->heads; aa.head_dim = L->out_dim / L->heads; aa.z = Z; aa.scores = scores;
     aa.slope = L->leaky_slope; aa.bias = L->bias; aa.act = L->act; aa.dst = h_out;
@@ -98,18 +115,16 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
   if (w.plan == PLAN_SAGE_REORDER) {
     float *S = reinterpret_cast<float *>(ws + w.off_a);
     void *Z = ws + w.off_b;
-    IT_TRY(it_launch_prep_weights(IT_PREP_SAGE_REORDER, L, B, st));
     it_gemm_args ga{};
     ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
     ga.B = B; ga.NB = 2 * L->out_dim;
     ga.n0 = L->out_dim; ga.out0 = S; ga.dt0 = IT_F32; ga.bias0 = L->bias; ga.act0 = IT_ACT_NONE;
     ga.n1 = L->out_dim; ga.out1 = Z; ga.dt1 = dt; ga.out2 = nullptr;
-    IT_TRY(it_launch_gemm(ga, st));
+    IT_TRY(run_apply(g, L, IT_PREP_SAGE_REORDER, ga, B, nullptr, st));
     gg.dim = L->out_dim; gg.src = Z; gg.dst = h_out; gg.epi = IT_EPI_ADD_ACT; gg.self_term = S; gg.act = L->act;
     return it_launch_gather(gg, st);
   }
   void *A = ws + w.off_a;
-  IT_TRY(it_launch_prep_weights(IT_PREP_SAGE, L, B, st));
   gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.act = IT_ACT_NONE;
   IT_TRY(it_launch_gather(gg, st));
   it_gemm_args ga{};
@@ -117,7 +132,7 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
   ga.B = B; ga.NB = L->out_dim;
   ga.n0 = L->out_dim; ga.out0 = h_out; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = L->act;
   ga.n1 = 0; ga.out1 = nullptr; ga.dt1 = dt; ga.out2 = nullptr;
-  return it_launch_gemm(ga, st);
+  return run_apply(g, L, IT_PREP_SAGE, ga, B, nullptr, st);
 }
 
 struct InferWs { size_t layer_bytes, buf_bytes, off_buf0, off_buf1, bytes; };

@@ -1,0 +1,542 @@
+// Apply on the 5th-generation tensor cores: a persistent, warp-specialised GEMM
+//   C[M, NB] = X1[M, K1] * B[0:K1, :] + X2[M, K2] * B[K1:, :]
+// with tcgen05.mma (accumulators in TMEM), operands staged in shared memory by TMA
+// (128-byte swizzle), the small weight matrix resident in shared memory for the life of the
+// CTA, two TMEM accumulator buffers so that the epilogue of one 128-row tile overlaps the
+// main loop of the next, and bias / activation / dtype routing / GAT scores in the epilogue.
+//
+// Two operand modes:
+//   bf16 : kind::f16 with bf16 inputs, fp32 accumulation.
+//   fp32 : three kind::tf32 products per step, A = A_hi + A_lo and B = B_hi + B_lo with
+//          A_hi*B_hi + A_lo*B_hi + A_hi*B_lo (the dropped A_lo*B_lo term is ~2^-22 relative);
+//          a single TF32 pass (10-bit mantissa) would miss the 1e-4 error bound.  A is split
+//          in shared memory by four dedicated warps, B is split once by the prep kernel.
+//
+// Every wait on an mbarrier is bounded: when one gives up, the CTA raises a flag that all
+// roles poll, drains, frees its TMEM and returns, and a status word in global memory is set.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int TC_BM = 128;          // rows per tile (UMMA M)
+constexpr int TC_KBLOCK_BYTES = 128;  // one swizzle row of K per k-block
+constexpr int TC_THREADS_BF16 = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 epilogue
+constexpr int TC_THREADS_TF32 = 320;  // ... plus warps 6-9 splitting A into hi / lo
+constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (or this wait ran out and started the abort).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+  for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols));
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols));
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+template <bool TF32>
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  if (TF32) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+  }
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128-byte swizzle rows:
+// start address, leading offset 16 B (unused for swizzled K-major), 1024 B between 8-row
+// groups, descriptor version 1, layout SWIZZLE_128B.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+
+__device__ __forceinline__ float act_apply(float x, int act) {
+  if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
+  if (act == IT_ACT_ELU) return x > 0.f ? x : expm1f(x);
+  return x;
+}
+
+// ----------------------------------------------------------------------------- kernel
+struct TcParams {
+  int64_t M;
+  int n_tiles_m, n_splits, nbc;   // row tiles, column splits, columns per CTA
+  int kb1, kb2;                   // k-blocks that come from X1 / X2
+  int NB;                         // total columns
+  int stages;
+  // epilogue routing (columns are global column ids)
+  int n0; void *out0; int out0_bf16; const float *bias0; int act0;
+  int n1; void *out1; int out1_bf16;
+  float *scores; const float *att_src; const float *att_dst; int heads, head_dim;  // GAT: scores [M, 2*heads]
+  int *status;                    // set to 1 if a bounded wait gave up
+};
+
+template <bool TF32>
+__global__ void __launch_bounds__(TF32 ? TC_THREADS_TF32 : TC_THREADS_BF16, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant__ CUtensorMap map_x2,
+               const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KB = p.kb1 + p.kb2;
+  const int b_tile_bytes = p.nbc * TC_KBLOCK_BYTES;              // one k-block of B (one part)
+  const int b_bytes = (TF32 ? 2 : 1) * KB * b_tile_bytes;
+  const int a_tile_bytes = TC_BM * TC_KBLOCK_BYTES;              // 16 KB
+  const int stage_bytes = (TF32 ? 2 : 1) * a_tile_bytes;
+
+  unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char *smem_b = base;
+  unsigned char *smem_a = base + b_bytes;   // b_bytes is a multiple of 1024 (nbc is a multiple of 16)
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_a + (size_t)p.stages * stage_bytes);
+  uint64_t *full = bars;                    // [stages]  TMA landed
+  uint64_t *empty = bars + p.stages;        // [stages]  MMAs that read the stage are done
+  uint64_t *ready = bars + 2 * p.stages;    // [stages]  (fp32 mode) hi / lo split written
+  uint64_t *b_full = bars + 3 * p.stages;   // [1]
+  uint64_t *acc_full = b_full + 1;          // [2]
+  uint64_t *acc_empty = acc_full + 2;       // [2]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const uint32_t acc_cols = (uint32_t)p.nbc;
+  uint32_t tmem_cols = 32;
+  while (tmem_cols < 2 * acc_cols) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+      mbar_init(&ready[s], 128);
+    }
+    mbar_init(b_full, 1);
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc_full[a], 1);
+      mbar_init(&acc_empty[a], 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_tiles = p.n_tiles_m * p.n_splits;
+  const int my_split = blockIdx.x % p.n_splits;   // gridDim.x is a multiple of n_splits: constant per CTA
+  const int col_base = my_split * p.nbc;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      // the weights of this CTA's columns, once
+      mbar_arrive_expect_tx(b_full, (uint32_t)b_bytes);
+      const int bk_elems = TF32 ? 32 : 64;
+      for (int part = 0; part < (TF32 ? 2 : 1); ++part)
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_2d(smem_b + (size_t)(part * KB + kb) * b_tile_bytes, &map_b, kb * bk_elems, part * p.NB + col_base, b_full);
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / p.n_splits) * TC_BM;
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full[stage], (uint32_t)a_tile_bytes);
+          if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * stage_bytes, &map_x1, kb * bk_elems, m0, &full[stage]);
+          else tma_load_2d(smem_a + (size_t)stage * stage_bytes, &map_x2, (kb - p.kb1) * bk_elems, m0, &full[stage]);
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // aborting: let the copies that were issued land before the CTA may exit (bounded)
+        for (int s = 0; s < p.stages; ++s)
+          for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it)
+            if (mbar_try_wait(&full[s], 0) || mbar_try_wait(&full[s], 1)) break;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: D = fp32, A/B = bf16 or tf32, both K-major, N = nbc, M = 128
+      const uint32_t fmt = TF32 ? 2u : 1u;
+      const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.nbc >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      bool ok = mbar_wait(b_full, 0, abort_flag);
+      uint32_t stage = 0, phase = 0;
+      uint32_t acc = 0, acc_phase = 0;
+      uint64_t *const wait_bar = TF32 ? ready : full;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * acc_cols;
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = mbar_wait(&wait_bar[stage], phase, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_hi = smem_u32(smem_a + (size_t)stage * stage_bytes);
+          const uint32_t b_hi = smem_u32(smem_b + (size_t)kb * b_tile_bytes);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {   // four 32-byte K steps inside the 128-byte swizzle row
+            const uint32_t first = (kb | k) != 0;
+            tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc, first);
+            if (TF32) {
+              const uint32_t a_lo = a_hi + a_tile_bytes;
+              const uint32_t b_lo = b_hi + (uint32_t)(KB * b_tile_bytes);
+              tc_mma<TF32>(d_tmem, make_desc(a_lo + k * 32), make_desc(b_hi + k * 32), idesc, 1u);
+              tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_lo + k * 32), idesc, 1u);
+            }
+          }
+          tc_commit(&empty[stage]);   // stage reusable once these MMAs have read it
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(&acc_full[acc]);    // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
+    const int quarter = warp & 3;   // a warp may only touch TMEM lanes [32 * (warp % 4), +32)
+    const int row_in_tile = quarter * 32 + lane;
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    const int n01 = p.n0 + p.n1;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int64_t m = (int64_t)(tile / p.n_splits) * TC_BM + row_in_tile;
+      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      float s_src[8], s_dst[8];
+#pragma unroll
+      for (int h = 0; h < 8; ++h) { s_src[h] = 0.f; s_dst[h] = 0.f; }
+      for (int c = 0; c < p.nbc; c += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * acc_cols + (uint32_t)c, r);
+        tmem_ld_wait();
+        const int gc = col_base + c;   // global column of r[0]; 16-column groups never straddle a segment
+        if (m < p.M) {
+          float v[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+          if (p.scores) {   // GAT: attention scores from the unrounded accumulators
+            const int h = gc / p.head_dim, d0 = gc % p.head_dim;
+            float a = 0.f, b = 0.f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              a = fmaf(v[i], __ldg(p.att_src + h * p.head_dim + d0 + i), a);
+              b = fmaf(v[i], __ldg(p.att_dst + h * p.head_dim + d0 + i), b);
+            }
+#pragma unroll
+            for (int hh = 0; hh < 8; ++hh)
+              if (hh == h) { s_src[hh] += a; s_dst[hh] += b; }
+          }
+          void *dst; int bf16; int64_t off;
+          if (gc < p.n0) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = act_apply(v[i] + (p.bias0 ? __ldg(p.bias0 + gc + i) : 0.f), p.act0);
+            dst = p.out0; bf16 = p.out0_bf16; off = m * p.n0 + gc;
+          } else {
+            dst = p.out1; bf16 = p.out1_bf16; off = m * p.n1 + (gc - p.n0);
+          }
+          if (gc < n01) {
+            if (bf16) {
+              uint32_t w[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                w[i] = *reinterpret_cast<uint32_t *>(&h2);
+              }
+              uint4 *q = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(dst) + off);
+              q[0] = make_uint4(w[0], w[1], w[2], w[3]);
+              q[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            } else {
+              float4 *q = reinterpret_cast<float4 *>(reinterpret_cast<float *>(dst) + off);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) q[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+          }
+        }
+      }
+      if (p.scores && m < p.M) {
+        for (int h = 0; h < p.heads; ++h) {
+          const int h_lo = col_base / p.head_dim, h_hi = (col_base + p.nbc) / p.head_dim;
+          if (h >= h_lo && h < h_hi) {
+            float a = 0.f, b = 0.f;
+#pragma unroll
+            for (int hh = 0; hh < 8; ++hh)
+              if (hh == h) { a = s_src[hh]; b = s_dst[hh]; }
+            p.scores[m * 2 * p.heads + h] = a;
+            p.scores[m * 2 * p.heads + p.heads + h] = b;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  } else {
+    // ------------------------------------------------------------------ fp32 mode: split A into hi + lo
+    if (TF32) {
+      const int tid = threadIdx.x - 192;   // 0..127
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        for (int kb = 0; kb < KB; ++kb) {
+          ok = mbar_wait(&full[stage], phase, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          float4 *hi = reinterpret_cast<float4 *>(smem_a + (size_t)stage * stage_bytes);
+          float4 *lo = reinterpret_cast<float4 *>(smem_a + (size_t)stage * stage_bytes + a_tile_bytes);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {   // 1024 float4 per tile, 128 threads
+            const int i = tid + j * 128;
+            const float4 x = hi[i];
+            float4 h, l;
+            h.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); l.x = x.x - h.x;
+            h.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u); l.y = x.y - h.y;
+            h.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); l.z = x.z - h.z;
+            h.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u); l.w = x.w - h.w;
+            hi[i] = h;
+            lo[i] = l;
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
+          mbar_arrive(&ready[stage]);
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, 1);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
+// ----------------------------------------------------------------------------- weight prep (K-major, split)
+struct PrepTcParams {
+  int kind, in_dim, out_dim, w_is_bf16, NB, K;
+  const void *W;
+  void *B;   // bf16 [NB, K]  or  fp32 [2, NB, K] (hi, lo)
+};
+
+__global__ void prep_weights_tc_kernel(PrepTcParams p) {
+  const int64_t total = (int64_t)p.NB * p.K;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int n = (int)(i / p.K), k = (int)(i % p.K);
+    int64_t src;   // element of W that is B[k, n]
+    if (p.kind == IT_PREP_SAGE_REORDER) src = n < p.out_dim ? (int64_t)k * p.out_dim + n : (int64_t)(p.in_dim + k) * p.out_dim + (n - p.out_dim);
+    else src = (int64_t)k * p.out_dim + n;
+    if (p.w_is_bf16) {
+      reinterpret_cast<__nv_bfloat16 *>(p.B)[i] = reinterpret_cast<const __nv_bfloat16 *>(p.W)[src];
+    } else {
+      const float w = reinterpret_cast<const float *>(p.W)[src];
+      // hi = w rounded to tf32 (nearest even on the 13 dropped bits), lo = the exact remainder
+      uint32_t u = __float_as_uint(w);
+      u += 0xfffu + ((u >> 13) & 1u);
+      u &= 0xffffe000u;
+      const float hi = __uint_as_float(u);
+      reinterpret_cast<float *>(p.B)[i] = hi;
+      reinterpret_cast<float *>(p.B)[total + i] = w - hi;
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D row-major matrix [rows, cols] of `elem` bytes; box = 128 bytes of a row x box_rows rows, 128-byte swizzle.
+it_status make_map(CUtensorMap *map, const void *ptr, int elem, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn enc = get_encode();
+  IT_REQUIRE(enc != nullptr, IT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * (cuuint64_t)elem};
+  const cuuint32_t box[2] = {(cuuint32_t)(TC_KBLOCK_BYTES / elem), (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapDataType dt = elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  CUresult r = enc(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  IT_REQUIRE(r == CUDA_SUCCESS, IT_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return IT_OK;
+}
+
+constexpr int kSmemBudget = 227 * 1024;
+constexpr int kSmemAux = 1024 /*alignment slack*/ + 512 /*barriers*/;
+
+}  // namespace
+
+size_t it_tc_weights_bytes(const it_layer_desc *L, int NB, int K) {
+  return (size_t)NB * K * (L->feat_dtype == IT_BF16 ? 2 : 8);
+}
+
+// Column split of the tensor-core path: the largest columns-per-CTA count (a multiple of 16
+// that divides NB, at most 256) whose resident weights fit in 128 KB of shared memory.
+static bool tc_split(bool tf32, int NB, int KB, int *n_splits, int *nbc) {
+  for (int s = 1; s <= 16; ++s) {
+    if (NB % s != 0) continue;
+    const int c = NB / s;
+    if (c % 16 != 0 || c > 256) continue;
+    if ((size_t)(tf32 ? 2 : 1) * KB * c * TC_KBLOCK_BYTES > 128 * 1024) continue;
+    *n_splits = s; *nbc = c;
+    return true;
+  }
+  return false;
+}
+
+bool it_tc_supported(const it_gemm_args &a, int heads, int head_dim, bool want_scores) {
+  const bool tf32 = a.x_dtype == IT_F32;
+  const int elem = tf32 ? 4 : 2;
+  const int bk = TC_KBLOCK_BYTES / elem;
+  if (a.M <= 0 || a.M > (int64_t)INT32_MAX) return false;
+  const int K2 = a.X2 ? a.K2 : 0;
+  if (a.K1 <= 0 || a.K1 % bk != 0 || K2 % bk != 0) return false;
+  const int NB = a.n0 + a.n1;   // score columns are not materialised on this path
+  if (NB <= 0 || NB % 16 != 0 || a.n0 % 16 != 0) return false;
+  int n_splits, nbc;
+  if (!tc_split(tf32, NB, (a.K1 + K2) / bk, &n_splits, &nbc)) return false;
+  if (want_scores && (heads > 8 || head_dim % 16 != 0 || nbc % head_dim != 0)) return false;
+  return true;
+}
+
+it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *L, int NB, int K, void *B, cudaStream_t st) {
+  PrepTcParams p;
+  p.kind = kind; p.in_dim = L->in_dim; p.out_dim = L->out_dim; p.w_is_bf16 = L->weight_dtype == IT_BF16;
+  p.NB = NB; p.K = K; p.W = L->W; p.B = B;
+  IT_LAUNCH(IT_K_PREP, 0, 0, st, prep_weights_tc_kernel<<<64, 256, 0, st>>>(p));
+  IT_CUDA_TRY(cudaGetLastError());
+  return IT_OK;
+}
+
+// B: weights prepared by it_launch_prep_weights_tc.  a.B / a.NB / a.out2 of the generic args are ignored:
+// the tensor-core path computes n0 + n1 columns and, for GAT, the scores in its epilogue.
+it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *att_src, const float *att_dst, int heads,
+                            int head_dim, float *scores, int num_sms, int *status, cudaStream_t st) {
+  if (a.M == 0) return IT_OK;
+  const bool tf32 = a.x_dtype == IT_F32;
+  const int elem = tf32 ? 4 : 2;
+  const int bk = TC_KBLOCK_BYTES / elem;
+  const int NB = a.n0 + a.n1;
+  const int K2 = a.X2 ? a.K2 : 0;
+  const int K = a.K1 + K2;
+  const int KB = K / bk;
+  int n_splits = 1, nbc = NB;
+  IT_REQUIRE(tc_split(tf32, NB, KB, &n_splits, &nbc), IT_ERR_UNSUPPORTED, "tensor-core apply: cannot tile %d columns with K = %d", NB, K);
+  const int b_bytes = (tf32 ? 2 : 1) * KB * nbc * TC_KBLOCK_BYTES;
+  const int stage_bytes = (tf32 ? 2 : 1) * TC_BM * TC_KBLOCK_BYTES;
+  int stages = (kSmemBudget - kSmemAux - b_bytes) / stage_bytes;
+  if (stages > 8) stages = 8;
+  IT_REQUIRE(stages >= 2, IT_ERR_UNSUPPORTED, "tensor-core apply: no room for two operand stages");
+  const int smem = b_bytes + stages * stage_bytes + kSmemAux;
+
+  CUtensorMap m1, m2, mb;
+  IT_TRY(make_map(&m1, a.X1, elem, a.M, a.K1, TC_BM));
+  if (a.X2) IT_TRY(make_map(&m2, a.X2, elem, a.M, K2, TC_BM));
+  else m2 = m1;
+  IT_TRY(make_map(&mb, B, elem, (int64_t)(tf32 ? 2 : 1) * NB, K, nbc));
+
+  TcParams p;
+  p.M = a.M; p.n_tiles_m = (int)((a.M + TC_BM - 1) / TC_BM); p.n_splits = n_splits; p.nbc = nbc;
+  p.kb1 = a.K1 / bk; p.kb2 = K2 / bk; p.NB = NB; p.stages = stages;
+  p.n0 = a.n0; p.out0 = a.out0; p.out0_bf16 = a.dt0 == IT_BF16; p.bias0 = a.bias0; p.act0 = a.act0;
+  p.n1 = a.n1; p.out1 = a.out1; p.out1_bf16 = a.dt1 == IT_BF16;
+  p.scores = scores; p.att_src = att_src; p.att_dst = att_dst; p.heads = heads; p.head_dim = head_dim > 0 ? head_dim : 1;
+  p.status = status;
+
+  const int64_t n_tiles = (int64_t)p.n_tiles_m * n_splits;
+  int64_t grid = (int64_t)(num_sms / n_splits) * n_splits;
+  if (grid > n_tiles) grid = n_tiles;   // n_tiles is a multiple of n_splits
+  const double xs = elem;
+  const double bytes = (double)a.M * (K * xs + a.n0 * (a.dt0 == IT_F32 ? 4.0 : 2.0) + a.n1 * (a.dt1 == IT_F32 ? 4.0 : 2.0) +
+                                     (scores ? 8.0 * heads : 0.0)) + (double)K * NB * xs;
+  const double flops = 2.0 * (double)a.M * K * NB;
+  if (tf32) {
+    IT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    IT_LAUNCH(IT_K_GEMM_TC, bytes, flops, st, gemm_tc_kernel<true><<<(unsigned)grid, TC_THREADS_TF32, smem, st>>>(m1, m2, mb, p));
+  } else {
+    IT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    IT_LAUNCH(IT_K_GEMM_TC, bytes, flops, st, gemm_tc_kernel<false><<<(unsigned)grid, TC_THREADS_BF16, smem, st>>>(m1, m2, mb, p));
+  }
+  IT_CUDA_TRY(cudaGetLastError());
+  return IT_OK;
+}

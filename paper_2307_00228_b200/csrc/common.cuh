@@ -40,8 +40,8 @@ void it_set_error(const char *fmt, ...);
 
 // ----------------------------------------------------------------------------- instrumentation
 enum it_kernel_id {
-  IT_K_VALIDATE = 0, IT_K_SPLIT_SCAN, IT_K_SPLIT_FILL, IT_K_BUCKET_SCAN, IT_K_PREP, IT_K_GATHER_CTA, IT_K_GATHER_WARP,
-  IT_K_GATHER_SUBWARP, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_WARP, IT_K_GAT_SUBWARP,
+  IT_K_VALIDATE = 0, IT_K_SPLIT_SCAN, IT_K_SPLIT_FILL, IT_K_BUCKET_SCAN, IT_K_PREP, IT_K_GATHER_CTA, IT_K_GATHER_FLAT,
+  IT_K_GATHER_EMPTY, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_WARP, IT_K_GAT_SUBWARP,
   IT_K_COUNT
 };
 // Wraps one kernel launch: counts it and, while profiling is on, brackets it with events on `st`.
@@ -59,6 +59,14 @@ bool it_profile_is_on();
   } while (0)
 
 // ----------------------------------------------------------------------------- graph handle
+// One shadow row as the gather kernels read it: first edge, edge count, and where the
+// aggregate goes (vertex id >= 0 for an unsplit row, ~slot in the partial buffer otherwise).
+struct __align__(16) it_row_meta {
+  int64_t j0;
+  int32_t len;
+  int32_t dest;
+};
+
 struct it_graph {
   int64_t n = 0, e = 0;
   const void *indptr = nullptr;
@@ -84,6 +92,8 @@ struct it_graph {
   int64_t h_bucket_edges[IT_MAX_BUCKETS] = {0};  // edges held by the rows of each bucket
   int64_t *bucket_offsets = nullptr;  // device [n_buckets+1]
   int32_t *bucket_rows = nullptr;     // [R]
+  int *d_status = nullptr;            // device word: set to 1 by a kernel whose bounded wait gave up
+  it_row_meta *bucket_meta = nullptr; // [R] in bucket order: what a gather needs to know about one row, in one 16-byte load
 };
 
 static inline size_t it_align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -149,3 +159,14 @@ enum it_prep_kind { IT_PREP_SAGE = 0, IT_PREP_SAGE_REORDER = 1, IT_PREP_GAT = 2 
 // [W_self | W_neigh]; GAT [in, out + 2*heads] = [W | W a_src | W a_dst].
 it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *layer, float *B,
                                  cudaStream_t stream);
+
+// ----------------------------------------------------------------------------- apply_tc.cu
+// The same product on the tensor cores (tcgen05 + TMEM + TMA).  Needs K1, K2 multiples of 128
+// bytes and n0, n0 + n1 multiples of 16; computes the n0 + n1 columns and, for GAT, the
+// attention scores [M, 2*heads] in its epilogue (a.B, a.NB and a.out2 are not used).  B is the
+// matrix written by it_launch_prep_weights_tc: bf16 [NB, K] or fp32 [2, NB, K] (hi, lo), K-major.
+bool it_tc_supported(const it_gemm_args &a, int heads, int head_dim, bool want_scores);
+it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *layer, int NB, int K, void *B,
+                                    cudaStream_t stream);
+it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *att_src, const float *att_dst,
+                            int heads, int head_dim, float *scores, int num_sms, int *status, cudaStream_t stream);

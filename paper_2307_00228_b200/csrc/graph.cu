@@ -247,6 +247,18 @@ struct EdgesInBucket {
     return bucket_of(len, B) == which ? len : 0;
   }
 };
+__global__ void fill_bucket_meta_kernel(int64_t n_rows, const int32_t *__restrict__ bucket_rows,
+                                       const int64_t *__restrict__ sp, const int32_t *__restrict__ row_dest,
+                                       it_row_meta *__restrict__ meta) {
+  int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n_rows) return;
+  const int32_t r = bucket_rows[i];
+  it_row_meta m;
+  m.j0 = sp[r];
+  m.len = (int32_t)(sp[r + 1] - sp[r]);
+  m.dest = row_dest[r];
+  meta[i] = m;
+}
 __global__ void set_next_bucket_offset_kernel(int64_t *bucket_offsets, int which, const int64_t *count) {
   if (which == 0) bucket_offsets[0] = 0;
   bucket_offsets[which + 1] = bucket_offsets[which] + *count;
@@ -256,6 +268,7 @@ __global__ void set_next_bucket_offset_kernel(int64_t *bucket_offsets, int which
 static void free_derived(it_graph *g) {
   cudaFree(g->shadow_indptr); cudaFree(g->shadow_owner); cudaFree(g->owner_indptr);
   cudaFree(g->row_dest); cudaFree(g->split_owners); cudaFree(g->bucket_offsets); cudaFree(g->bucket_rows);
+  cudaFree(g->bucket_meta); g->bucket_meta = nullptr;
   g->shadow_indptr = nullptr; g->shadow_owner = nullptr; g->owner_indptr = nullptr; g->row_dest = nullptr;
   g->split_owners = nullptr; g->bucket_offsets = nullptr; g->bucket_rows = nullptr;
   g->n_rows = g->n_split_owners = g->n_partial_rows = 0;
@@ -302,6 +315,7 @@ static it_status split_impl(it_graph *g, int64_t T, cudaStream_t st) {
   SPLIT_CUDA(cudaMalloc(&g->row_dest, (size_t)(R > 0 ? R : 1) * sizeof(int32_t)));
   SPLIT_CUDA(cudaMalloc(&g->split_owners, (size_t)(S > 0 ? S : 1) * sizeof(int32_t)));
   SPLIT_CUDA(cudaMalloc(&g->bucket_rows, (size_t)(R > 0 ? R : 1) * sizeof(int32_t)));
+  SPLIT_CUDA(cudaMalloc(&g->bucket_meta, (size_t)(R > 0 ? R : 1) * sizeof(it_row_meta)));
   SPLIT_CUDA(cudaMalloc(&g->bucket_offsets, (IT_MAX_BUCKETS + 1) * sizeof(int64_t)));
   if (S > 0)
     SPLIT_TRY(scan_and_emit(IT_K_SPLIT_SCAN, n, IsSplit{ip, T}, EmitSplitOwner{ip, T, g->split_owners}, d_scratch, d_total + 1, st));
@@ -347,6 +361,10 @@ static it_status split_impl(it_graph *g, int64_t T, cudaStream_t st) {
     SPLIT_TRY(scan_and_emit(IT_K_BUCKET_SCAN, R, EdgesInBucket{g->shadow_indptr, B, b}, EmitNothing{}, d_scratch,
                             d_edges + b, st));
   }
+  if (R > 0)
+    IT_LAUNCH(IT_K_BUCKET_SCAN, 0, 0, st,
+              fill_bucket_meta_kernel<<<(unsigned)((R + 255) / 256), 256, 0, st>>>(R, g->bucket_rows, g->shadow_indptr,
+                                                                                    g->row_dest, g->bucket_meta));
   SPLIT_CUDA(cudaGetLastError());
   SPLIT_CUDA(cudaMemcpyAsync(g->h_bucket_edges, d_edges, B.nb * sizeof(int64_t), cudaMemcpyDeviceToHost, st));
   SPLIT_CUDA(cudaMemcpyAsync(g->h_bucket_offsets, g->bucket_offsets, (B.nb + 1) * sizeof(int64_t),
@@ -407,8 +425,14 @@ extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, i
   cudaGetDevice(&g->device);
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, g->device) == cudaSuccess && sms > 0) g->num_sms = sms;
+  if (cudaMalloc(&g->d_status, sizeof(int)) != cudaSuccess || cudaMemsetAsync(g->d_status, 0, sizeof(int), st) != cudaSuccess) {
+    it_set_error("allocating the status word failed");
+    cudaFree(g->d_status);
+    delete g;
+    return IT_ERR_OOM;
+  }
   it_status rc = split_impl(g, 0, st);
-  if (rc != IT_OK) { delete g; return rc; }
+  if (rc != IT_OK) { cudaFree(g->d_status); delete g; return rc; }
   *out = g;
   return IT_OK;
 }
@@ -438,9 +462,24 @@ extern "C" it_status it_graph_get_split(const it_graph *g, int64_t *n_rows, cons
   return IT_OK;
 }
 
+extern "C" it_status it_graph_check(it_graph *g, void *stream) {
+  IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
+  cudaStream_t st = (cudaStream_t)stream;
+  int h = 0;
+  IT_CUDA_TRY(cudaMemcpyAsync(&h, g->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  IT_CUDA_TRY(cudaStreamSynchronize(st));
+  if (h != 0) {
+    IT_CUDA_TRY(cudaMemsetAsync(g->d_status, 0, sizeof(int), st));
+    it_set_error("a kernel gave up a bounded wait; its outputs are not valid");
+    return IT_ERR_TIMEOUT;
+  }
+  return IT_OK;
+}
+
 extern "C" it_status it_graph_destroy(it_graph *g) {
   if (!g) return IT_OK;
   free_derived(g);
+  cudaFree(g->d_status);
   delete g;
   return IT_OK;
 }

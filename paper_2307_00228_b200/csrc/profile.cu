@@ -15,7 +15,7 @@ std::vector<Slot> g_slots;       // slots in use since it_profile_begin
 std::vector<Slot> g_pool;        // recycled event pairs
 int64_t g_launches = 0;
 const char *const kNames[IT_K_COUNT] = {"validate", "split_scan", "split_fill", "bucket_scan", "prep_weights",
-                                        "gather_cta", "gather_warp", "gather_subwarp", "combine", "gemm_fp32",
+                                        "gather_cta", "gather_flat", "gather_empty", "combine", "gemm_fp32",
                                         "gemm_tc", "gat_cta", "gat_warp", "gat_subwarp"};
 }  // namespace
 

@@ -63,7 +63,7 @@ def run_device(w: Workload, int32_indptr=False, threshold=None):
     """it_infer through the C ABI; returns (final output as fp64 numpy, DeviceWorkload)."""
     d = host.upload(w, int32_indptr=int32_indptr, threshold=threshold)
     d.infer()
-    torch.cuda.synchronize()
+    B.it_graph_check(d.graph)     # synchronises; raises if a kernel gave up a bounded wait
     return to_numpy(d.out), d
 
 
