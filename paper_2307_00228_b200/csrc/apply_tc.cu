@@ -22,8 +22,9 @@ namespace {
 
 constexpr int TC_BM = 128;          // rows per tile (UMMA M)
 constexpr int TC_KBLOCK_BYTES = 128;  // one swizzle row of K per k-block
-constexpr int TC_THREADS_BF16 = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 epilogue
-constexpr int TC_THREADS_TF32 = 320;  // ... plus warps 6-9 splitting A into hi / lo
+constexpr int TC_EPI_WARPS = 16;      // four warps per TMEM lane quarter, each takes every fourth 16-column group
+constexpr int TC_THREADS_BF16 = 64 + 32 * TC_EPI_WARPS;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2-17 epilogue
+constexpr int TC_THREADS_TF32 = TC_THREADS_BF16 + 128;    // ... plus four warps splitting A into hi / lo
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -111,12 +112,6 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
          ((uint64_t)2 << 61);
 }
 
-__device__ __forceinline__ float act_apply(float x, int act) {
-  if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
-  if (act == IT_ACT_ELU) return x > 0.f ? x : expm1f(x);
-  return x;
-}
-
 // ----------------------------------------------------------------------------- kernel
 struct TcParams {
   int64_t M;
@@ -140,21 +135,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   const int KB = p.kb1 + p.kb2;
   const int b_tile_bytes = p.nbc * TC_KBLOCK_BYTES;              // one k-block of B (one part)
   const int b_bytes = (TF32 ? 2 : 1) * KB * b_tile_bytes;
-  const int a_tile_bytes = TC_BM * TC_KBLOCK_BYTES;              // 16 KB
-  const int stage_bytes = (TF32 ? 2 : 1) * a_tile_bytes;
+  constexpr int a_tile_bytes = TC_BM * TC_KBLOCK_BYTES;          // 16 KB
 
+  // shared memory: resident weights | operand stages (raw / hi tiles) | fp32 mode: two lo tiles | barriers
   unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char *smem_b = base;
   unsigned char *smem_a = base + b_bytes;   // b_bytes is a multiple of 1024 (nbc is a multiple of 16)
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_a + (size_t)p.stages * stage_bytes);
+  unsigned char *smem_lo = smem_a + (size_t)p.stages * a_tile_bytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_lo + (TF32 ? 2 * a_tile_bytes : 0));
   uint64_t *full = bars;                    // [stages]  TMA landed
   uint64_t *empty = bars + p.stages;        // [stages]  MMAs that read the stage are done
   uint64_t *ready = bars + 2 * p.stages;    // [stages]  (fp32 mode) hi / lo split written
   uint64_t *b_full = bars + 3 * p.stages;   // [1]
   uint64_t *acc_full = b_full + 1;          // [2]
   uint64_t *acc_empty = acc_full + 2;       // [2]
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+  uint64_t *lo_free = acc_empty + 2;        // [2]  (fp32 mode) MMAs that read a lo tile are done
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(lo_free + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  // per-column constants of this CTA's columns, 16-byte aligned: bias (0 where none applies), GAT attention vectors
+  float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // [nbc]
+  float *att_s = bias_s + p.nbc;   // [2][nbc]: source vector, destination vector (only with scores)
 
   const uint32_t acc_cols = (uint32_t)p.nbc;
   uint32_t tmem_cols = 32;
@@ -164,12 +164,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
-      mbar_init(&ready[s], 128);
+      mbar_init(&ready[s], 4);
     }
     mbar_init(b_full, 1);
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], 4);
+      mbar_init(&acc_empty[a], TC_EPI_WARPS);
+      mbar_init(&lo_free[a], 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -177,6 +178,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   if (warp == 1) {
     tmem_alloc(tmem_slot, tmem_cols);
     tmem_relinquish();
+  }
+  for (int c = threadIdx.x; c < p.nbc; c += blockDim.x) {
+    const int gc = (blockIdx.x % p.n_splits) * p.nbc + c;
+    bias_s[c] = (p.bias0 && gc < p.n0) ? p.bias0[gc] : 0.f;
+    if (p.scores) {
+      att_s[c] = p.att_src[gc];
+      att_s[p.nbc + c] = p.att_dst[gc];
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -204,13 +213,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
           ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[stage], (uint32_t)a_tile_bytes);
-          if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * stage_bytes, &map_x1, kb * bk_elems, m0, &full[stage]);
-          else tma_load_2d(smem_a + (size_t)stage * stage_bytes, &map_x2, (kb - p.kb1) * bk_elems, m0, &full[stage]);
+          if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x1, kb * bk_elems, m0, &full[stage]);
+          else tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x2, (kb - p.kb1) * bk_elems, m0, &full[stage]);
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
-        // aborting: let the copies that were issued land before the CTA may exit (bounded)
+        // aborting: give the copies that were issued time to land before the CTA may exit (bounded)
         for (int s = 0; s < p.stages; ++s)
           for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it)
             if (mbar_try_wait(&full[s], 0) || mbar_try_wait(&full[s], 1)) break;
@@ -225,6 +234,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       bool ok = mbar_wait(b_full, 0, abort_flag);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
+      uint32_t lo = 0;
       uint64_t *const wait_bar = TF32 ? ready : full;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag);
@@ -235,20 +245,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
           ok = mbar_wait(&wait_bar[stage], phase, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a_hi = smem_u32(smem_a + (size_t)stage * stage_bytes);
+          const uint32_t a_hi = smem_u32(smem_a + (size_t)stage * a_tile_bytes);
           const uint32_t b_hi = smem_u32(smem_b + (size_t)kb * b_tile_bytes);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {   // four 32-byte K steps inside the 128-byte swizzle row
             const uint32_t first = (kb | k) != 0;
             tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc, first);
             if (TF32) {
-              const uint32_t a_lo = a_hi + a_tile_bytes;
+              const uint32_t a_lo = smem_u32(smem_lo + (size_t)lo * a_tile_bytes);
               const uint32_t b_lo = b_hi + (uint32_t)(KB * b_tile_bytes);
               tc_mma<TF32>(d_tmem, make_desc(a_lo + k * 32), make_desc(b_hi + k * 32), idesc, 1u);
               tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_lo + k * 32), idesc, 1u);
             }
           }
           tc_commit(&empty[stage]);   // stage reusable once these MMAs have read it
+          if (TF32) { tc_commit(&lo_free[lo]); lo ^= 1u; }
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
@@ -256,52 +267,94 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
-  } else if (warp < 6) {
-    // ------------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
+  } else if (warp < 2 + TC_EPI_WARPS) {
+    // ------------------------------------------------------------------ epilogue
+    // 16 warps: 4 TMEM lane quarters x 4 column sub-sets.  Sub-set `sub` of a quarter takes the 16-column
+    // groups g with g % 4 == sub, or, when attention scores are accumulated, the heads h with h % 4 == sub
+    // (so that one warp sees every column of a head).
     const int quarter = warp & 3;   // a warp may only touch TMEM lanes [32 * (warp % 4), +32)
+    const int sub = (warp - 2) >> 2;
     const int row_in_tile = quarter * 32 + lane;
+    const bool odd = lane & 1;
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     const int n01 = p.n0 + p.n1;
+    const int gph = p.scores ? p.head_dim / 16 : 1;          // 16-column groups per ownership unit
+    const int n_units = (p.nbc / 16) / gph;                   // units in this CTA's columns
+    const int unit0 = p.scores ? col_base / p.head_dim : 0;   // global index of the first unit (head)
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const int64_t m = (int64_t)(tile / p.n_splits) * TC_BM + row_in_tile;
+      const int64_t m_even = m - (odd ? 1 : 0), m_odd = m_even + 1;   // the two rows a lane pair writes together
       ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      float s_src[8], s_dst[8];
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * acc_cols;
+      bool released = false;
+      auto release = [&]() {   // everything this warp needs is in registers: hand the accumulator back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        released = true;
+      };
+      // the last unit this warp owns (ownership: (unit0 + u) % 4 == sub)
+      int last_u = -1;
+      for (int u = n_units - 1; u >= 0; --u)
+        if (((unit0 + u) & 3) == sub) { last_u = u; break; }
+      for (int u = 0; u < n_units; ++u) {
+        if (((unit0 + u) & 3) != sub) continue;
+        float sc_a = 0.f, sc_b = 0.f;   // attention scores of this head
+        for (int j0 = 0; j0 < gph; j0 += 2) {
+          // up to two 16-column groups in flight from TMEM, one wait
+          uint32_t r[2][16];
+          const int c_first = (u * gph + j0) * 16;          // local column of the first group
+          const int n_g = (gph - j0) >= 2 ? 2 : 1;
+          tmem_ld16(taddr + (uint32_t)c_first, r[0]);
+          if (n_g == 2) tmem_ld16(taddr + (uint32_t)c_first + 16, r[1]);
+          tmem_ld_wait();
+          if (u == last_u && j0 + 2 >= gph) release();
 #pragma unroll
-      for (int h = 0; h < 8; ++h) { s_src[h] = 0.f; s_dst[h] = 0.f; }
-      for (int c = 0; c < p.nbc; c += 16) {
-        uint32_t r[16];
-        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * acc_cols + (uint32_t)c, r);
-        tmem_ld_wait();
-        const int gc = col_base + c;   // global column of r[0]; 16-column groups never straddle a segment
-        if (m < p.M) {
-          float v[16];
+          for (int k = 0; k < 2; ++k) {
+            if (k >= n_g) break;
+            const int c = c_first + 16 * k;   // local column of r[k][0]
+            const int gc = col_base + c;      // global column; a group never straddles an output segment
+            float v[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-          if (p.scores) {   // GAT: attention scores from the unrounded accumulators
-            const int h = gc / p.head_dim, d0 = gc % p.head_dim;
-            float a = 0.f, b = 0.f;
+            for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[k][i]);
+            if (p.scores) {   // GAT: attention scores from the unrounded accumulators
+              const float4 *as4 = reinterpret_cast<const float4 *>(att_s + c);
+              const float4 *ad4 = reinterpret_cast<const float4 *>(att_s + p.nbc + c);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              a = fmaf(v[i], __ldg(p.att_src + h * p.head_dim + d0 + i), a);
-              b = fmaf(v[i], __ldg(p.att_dst + h * p.head_dim + d0 + i), b);
+              for (int i = 0; i < 4; ++i) {
+                const float4 a4 = as4[i], d4 = ad4[i];
+                sc_a = fmaf(v[4 * i], a4.x, sc_a); sc_a = fmaf(v[4 * i + 1], a4.y, sc_a);
+                sc_a = fmaf(v[4 * i + 2], a4.z, sc_a); sc_a = fmaf(v[4 * i + 3], a4.w, sc_a);
+                sc_b = fmaf(v[4 * i], d4.x, sc_b); sc_b = fmaf(v[4 * i + 1], d4.y, sc_b);
+                sc_b = fmaf(v[4 * i + 2], d4.z, sc_b); sc_b = fmaf(v[4 * i + 3], d4.w, sc_b);
+              }
             }
+            if (gc >= n01) continue;
+            void *dst; int bf16; int ld; int lc;
+            if (gc < p.n0) {
+              const float4 *bs = reinterpret_cast<const float4 *>(bias_s + c);
 #pragma unroll
-            for (int hh = 0; hh < 8; ++hh)
-              if (hh == h) { s_src[hh] += a; s_dst[hh] += b; }
-          }
-          void *dst; int bf16; int64_t off;
-          if (gc < p.n0) {
+              for (int i = 0; i < 4; ++i) {
+                const float4 b4 = bs[i];
+                v[4 * i] += b4.x; v[4 * i + 1] += b4.y; v[4 * i + 2] += b4.z; v[4 * i + 3] += b4.w;
+              }
+              if (p.act0 == IT_ACT_RELU) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = act_apply(v[i] + (p.bias0 ? __ldg(p.bias0 + gc + i) : 0.f), p.act0);
-            dst = p.out0; bf16 = p.out0_bf16; off = m * p.n0 + gc;
-          } else {
-            dst = p.out1; bf16 = p.out1_bf16; off = m * p.n1 + (gc - p.n0);
-          }
-          if (gc < n01) {
+                for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+              } else if (p.act0 == IT_ACT_ELU) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = v[i] > 0.f ? v[i] : expm1f(v[i]);
+              }
+              dst = p.out0; bf16 = p.out0_bf16; ld = p.n0; lc = gc;
+            } else {
+              dst = p.out1; bf16 = p.out1_bf16; ld = p.n1; lc = gc - p.n0;
+            }
+            // A lane pair (rows m_even, m_odd) swaps halves so that every store instruction writes whole
+            // 32-byte sectors: the even lane takes the low 16 bytes of each 32-byte piece, the odd lane the high.
             if (bf16) {
               uint32_t w[8];
 #pragma unroll
@@ -309,63 +362,85 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
                 __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
                 w[i] = *reinterpret_cast<uint32_t *>(&h2);
               }
-              uint4 *q = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(dst) + off);
-              q[0] = make_uint4(w[0], w[1], w[2], w[3]);
-              q[1] = make_uint4(w[4], w[5], w[6], w[7]);
-            } else {
-              float4 *q = reinterpret_cast<float4 *>(reinterpret_cast<float *>(dst) + off);
+              uint32_t got[4];
 #pragma unroll
-              for (int i = 0; i < 4; ++i) q[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+              for (int i = 0; i < 4; ++i) got[i] = __shfl_xor_sync(0xffffffffu, odd ? w[i] : w[4 + i], 1);
+              // even lane: row_even bytes 0-15 (own w0-3), row_odd bytes 0-15 (partner's w0-3)
+              // odd lane : row_even bytes 16-31 (partner's w4-7), row_odd bytes 16-31 (own w4-7)
+              __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + lc + (odd ? 8 : 0);
+              const uint4 first = odd ? make_uint4(got[0], got[1], got[2], got[3]) : make_uint4(w[0], w[1], w[2], w[3]);
+              const uint4 second = odd ? make_uint4(w[4], w[5], w[6], w[7]) : make_uint4(got[0], got[1], got[2], got[3]);
+              if (m_even < p.M) *reinterpret_cast<uint4 *>(o + m_even * ld) = first;
+              if (m_odd < p.M) *reinterpret_cast<uint4 *>(o + m_odd * ld) = second;
+            } else {
+              float got[8];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                got[i] = __shfl_xor_sync(0xffffffffu, odd ? v[i] : v[4 + i], 1);           // columns 0-3 <-> 4-7
+                got[4 + i] = __shfl_xor_sync(0xffffffffu, odd ? v[8 + i] : v[12 + i], 1);  // columns 8-11 <-> 12-15
+              }
+              // even lane: row_even cols 0-3, 8-11 (own); row_odd cols 0-3, 8-11 (partner's)
+              // odd lane : row_even cols 4-7, 12-15 (partner's); row_odd cols 4-7, 12-15 (own)
+              float *o = reinterpret_cast<float *>(dst) + lc + (odd ? 4 : 0);
+              float4 e0, e1, o0, o1;
+              if (!odd) {
+                e0 = make_float4(v[0], v[1], v[2], v[3]); e1 = make_float4(v[8], v[9], v[10], v[11]);
+                o0 = make_float4(got[0], got[1], got[2], got[3]); o1 = make_float4(got[4], got[5], got[6], got[7]);
+              } else {
+                e0 = make_float4(got[0], got[1], got[2], got[3]); e1 = make_float4(got[4], got[5], got[6], got[7]);
+                o0 = make_float4(v[4], v[5], v[6], v[7]); o1 = make_float4(v[12], v[13], v[14], v[15]);
+              }
+              if (m_even < p.M) {
+                *reinterpret_cast<float4 *>(o + m_even * ld) = e0;
+                *reinterpret_cast<float4 *>(o + m_even * ld + 8) = e1;
+              }
+              if (m_odd < p.M) {
+                *reinterpret_cast<float4 *>(o + m_odd * ld) = o0;
+                *reinterpret_cast<float4 *>(o + m_odd * ld + 8) = o1;
+              }
             }
           }
         }
-      }
-      if (p.scores && m < p.M) {
-        for (int h = 0; h < p.heads; ++h) {
-          const int h_lo = col_base / p.head_dim, h_hi = (col_base + p.nbc) / p.head_dim;
-          if (h >= h_lo && h < h_hi) {
-            float a = 0.f, b = 0.f;
-#pragma unroll
-            for (int hh = 0; hh < 8; ++hh)
-              if (hh == h) { a = s_src[hh]; b = s_dst[hh]; }
-            p.scores[m * 2 * p.heads + h] = a;
-            p.scores[m * 2 * p.heads + p.heads + h] = b;
-          }
+        if (p.scores && m < p.M) {
+          const int h = unit0 + u;
+          p.scores[m * 2 * p.heads + h] = sc_a;
+          p.scores[m * 2 * p.heads + p.heads + h] = sc_b;
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      if (!released) release();   // a warp that owns no columns of this CTA still has to sign off
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   } else {
     // ------------------------------------------------------------------ fp32 mode: split A into hi + lo
     if (TF32) {
-      const int tid = threadIdx.x - 192;   // 0..127
+      const int tid = threadIdx.x - TC_THREADS_BF16;   // 0..127
       uint32_t stage = 0, phase = 0;
+      uint32_t lo = 0, lo_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(&full[stage], phase, abort_flag);
+          ok = mbar_wait(&full[stage], phase, abort_flag) && mbar_wait(&lo_free[lo], lo_phase ^ 1u, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          float4 *hi = reinterpret_cast<float4 *>(smem_a + (size_t)stage * stage_bytes);
-          float4 *lo = reinterpret_cast<float4 *>(smem_a + (size_t)stage * stage_bytes + a_tile_bytes);
+          float4 *hi_t = reinterpret_cast<float4 *>(smem_a + (size_t)stage * a_tile_bytes);
+          float4 *lo_t = reinterpret_cast<float4 *>(smem_lo + (size_t)lo * a_tile_bytes);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {   // 1024 float4 per tile, 128 threads
             const int i = tid + j * 128;
-            const float4 x = hi[i];
+            const float4 x = hi_t[i];
             float4 h, l;
             h.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); l.x = x.x - h.x;
             h.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u); l.y = x.y - h.y;
             h.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); l.z = x.z - h.z;
             h.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u); l.w = x.w - h.w;
-            hi[i] = h;
-            lo[i] = l;
+            hi_t[i] = h;
+            lo_t[i] = l;
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
-          mbar_arrive(&ready[stage]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&ready[stage]);
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+          if (++lo == 2) { lo = 0; lo_phase ^= 1u; }
         }
       }
     }
@@ -442,7 +517,7 @@ it_status make_map(CUtensorMap *map, const void *ptr, int elem, int64_t rows, in
 }
 
 constexpr int kSmemBudget = 227 * 1024;
-constexpr int kSmemAux = 1024 /*alignment slack*/ + 512 /*barriers*/;
+constexpr int kSmemAux = 1024 /*alignment slack*/ + 288 /*barriers, TMEM slot, abort flag, alignment*/;
 
 }  // namespace
 
@@ -503,11 +578,13 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   int n_splits = 1, nbc = NB;
   IT_REQUIRE(tc_split(tf32, NB, KB, &n_splits, &nbc), IT_ERR_UNSUPPORTED, "tensor-core apply: cannot tile %d columns with K = %d", NB, K);
   const int b_bytes = (tf32 ? 2 : 1) * KB * nbc * TC_KBLOCK_BYTES;
-  const int stage_bytes = (tf32 ? 2 : 1) * TC_BM * TC_KBLOCK_BYTES;
-  int stages = (kSmemBudget - kSmemAux - b_bytes) / stage_bytes;
+  const int stage_bytes = TC_BM * TC_KBLOCK_BYTES;             // one raw / hi operand tile
+  const int lo_bytes = tf32 ? 2 * stage_bytes : 0;             // fp32 mode: two lo tiles shared by all stages
+  const int const_bytes = nbc * 4 * (scores ? 3 : 1);          // bias (+ attention vectors) of this CTA's columns
+  int stages = (kSmemBudget - kSmemAux - const_bytes - b_bytes - lo_bytes) / stage_bytes;
   if (stages > 8) stages = 8;
   IT_REQUIRE(stages >= 2, IT_ERR_UNSUPPORTED, "tensor-core apply: no room for two operand stages");
-  const int smem = b_bytes + stages * stage_bytes + kSmemAux;
+  const int smem = b_bytes + stages * stage_bytes + lo_bytes + kSmemAux + const_bytes;
 
   CUtensorMap m1, m2, mb;
   IT_TRY(make_map(&m1, a.X1, elem, a.M, a.K1, TC_BM));
