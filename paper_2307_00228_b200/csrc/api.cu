@@ -47,7 +47,7 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
   if (L->op == IT_GATHER_GAT) {
     w.plan = PLAN_GAT;
     w.off_B = take(fi * (fo + 2 * (size_t)L->heads) * 8);
-    w.off_partials = off;
+    w.off_partials = take(it_gat_partial_bytes(g, L->out_dim, L->heads));
     w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
     w.off_b = take(n * fo * s);                    // Z
   } else if (reorders(L)) {
@@ -105,7 +105,7 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
     ga.n1 = L->out_dim; ga.out1 = Z; ga.dt1 = dt; ga.out2 = scores;
     IT_TRY(run_apply(g, L, IT_PREP_GAT, ga, B, scores, st));
     it_gat_args aa{};
-    aa.g = g; aa.dtype = dt; aa.heads = L->heads; aa.head_dim = L->out_dim / L->heads; aa.z = Z; aa.scores = scores;
+    aa.g = g; aa.dtype = dt; aa.heads = L->heads; aa.head_dim = L->out_dim / L->heads; aa.z = Z; aa.scores = scores; aa.partials = partials;
     aa.slope = L->leaky_slope; aa.bias = L->bias; aa.act = L->act; aa.dst = h_out;
     return it_launch_gat(aa, st);
   }

@@ -41,7 +41,7 @@ void it_set_error(const char *fmt, ...);
 // ----------------------------------------------------------------------------- instrumentation
 enum it_kernel_id {
   IT_K_VALIDATE = 0, IT_K_SPLIT_SCAN, IT_K_SPLIT_FILL, IT_K_BUCKET_SCAN, IT_K_PREP, IT_K_GATHER_CTA, IT_K_GATHER_FLAT,
-  IT_K_GATHER_EMPTY, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_WARP, IT_K_GAT_SUBWARP,
+  IT_K_GATHER_EMPTY, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY,
   IT_K_COUNT
 };
 // Wraps one kernel launch: counts it and, while profiling is on, brackets it with events on `st`.
@@ -93,6 +93,7 @@ struct it_graph {
   int64_t *bucket_offsets = nullptr;  // device [n_buckets+1]
   int32_t *bucket_rows = nullptr;     // [R]
   int *d_status = nullptr;            // device word: set to 1 by a kernel whose bounded wait gave up
+  int32_t *bucket_owner = nullptr;    // [R] in bucket order: the vertex each row belongs to
   it_row_meta *bucket_meta = nullptr; // [R] in bucket order: what a gather needs to know about one row, in one 16-byte load
 };
 
@@ -128,12 +129,14 @@ struct it_gat_args {
   int heads, head_dim;
   const void *z;          // [n, heads*head_dim] messages
   const float *scores;    // [n, 2*heads]: source scores of the vertex, then its destination scores
+  float *partials;        // it_gat_partial_bytes() of fp32 scratch for the groups of split vertices (may be NULL if none)
   float slope;
   const float *bias;      // may be NULL
   it_act act;
   void *dst;              // [n, heads*head_dim]
 };
 it_status it_launch_gat(const it_gat_args &a, cudaStream_t stream);
+size_t it_gat_partial_bytes(const it_graph *g, int dim, int heads);
 
 // ----------------------------------------------------------------------------- apply.cu
 // C[M, NB] = X1[M, K1] * B[0:K1, :] + X2[M, K2] * B[K1:K1+K2, :]   (X2 may be NULL, K2 = 0)

@@ -1,269 +1,162 @@
 // GAT reduce: per destination and head, e = LeakyReLU(s_src[u] + s_dst[v]), softmax over the
 // in-edges, attention-weighted sum of the source rows z_u, then bias and activation.
 // One pass over the edges with a running (max, sum, weighted accumulator) state per lane
-// ("online" softmax); states of different edge slots / warps are merged in a fixed order.
-// HBM-bound like the plain gather: one 16-byte row slice + one 4-byte score per lane per edge.
-#include "common.cuh"
+// ("online" softmax).  Such states merge associatively — (m, l, acc) and (m', l', acc') give
+// M = max(m, m'), l e^(m-M) + l' e^(m'-M), acc e^(m-M) + acc' e^(m'-M) — so the groups of a split
+// hub are reduced independently into partial states and merged in group order, exactly like
+// the partial sums of the plain gather.  The edge streaming lives in stream.cuh.
+#include "stream.cuh"
 
 namespace {
 
-constexpr int GAT_THREADS = 256;
-constexpr int GAT_UNROLL = 4;
+using namespace it_stream;
 
-template <typename T> struct Vec16;
-template <> struct Vec16<float> {
-  static constexpr int VEC = 4;
-  __device__ static __forceinline__ void load(const float *p, float (&v)[4]) {
-    float4 x = __ldg(reinterpret_cast<const float4 *>(p));
-    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
-  }
-  __device__ static __forceinline__ void store(float *p, const float (&v)[4]) {
-    *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
-  }
-};
-template <> struct Vec16<__nv_bfloat16> {
-  static constexpr int VEC = 8;
-  __device__ static __forceinline__ void load(const __nv_bfloat16 *p, float (&v)[8]) {
-    uint4 x = __ldg(reinterpret_cast<const uint4 *>(p));
-    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(w[i] << 16);
-      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  }
-  __device__ static __forceinline__ void store(__nv_bfloat16 *p, const float (&v)[8]) {
-    uint32_t w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-      w[i] = *reinterpret_cast<uint32_t *>(&h);
-    }
-    *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
-  }
-};
+__host__ __device__ inline int gat_partial_stride(int dim, int heads) { return dim + ((2 * heads + 3) / 4) * 4; }
 
-__device__ __forceinline__ float act_apply(float x, int act) {
-  if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
-  if (act == IT_ACT_ELU) return x > 0.f ? x : expm1f(x);
-  return x;
-}
-
-struct GatParams {
-  const int64_t *__restrict__ shadow_indptr;
-  const int32_t *__restrict__ indices;
-  const int32_t *__restrict__ bucket_rows;
-  const int32_t *__restrict__ row_dest;
-  const void *__restrict__ z;
-  const float *__restrict__ scores;  // [n, 2*heads]: source scores, then destination scores
+template <typename T>
+struct GatPolicy {
+  static constexpr int VEC = Row16<T>::VEC;
+  static constexpr int NS = VEC + 2;   // accumulators, running max, running sum
+  static constexpr bool WEIGHTED = false, HAS_EXTRA = true, NEEDS_OWNER = true;
+  const float *__restrict__ scores;    // [n, 2*heads]: source scores of the vertex, then its destination scores
   const float *__restrict__ bias;
   void *__restrict__ dst;
-  int64_t row_lo, row_hi;
+  float *__restrict__ partials;        // [n_partial_rows, stride]: acc[dim], m[heads], l[heads]
   int dim, heads, head_dim, act;
   float slope;
-};
+  // per-thread
+  int col, head;
+  float s_dst;
 
-template <int VEC> struct SoftState {
-  float m, l, acc[VEC];
-  __device__ __forceinline__ void init() {
-    m = -INFINITY; l = 0.f;
+  __device__ __forceinline__ void setup(int t) { col = t * VEC; head = col / head_dim; s_dst = 0.f; }
+  __device__ __forceinline__ void init(float (&st)[NS]) const {
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+    for (int k = 0; k < VEC; ++k) st[k] = 0.f;
+    st[VEC] = -INFINITY;
+    st[VEC + 1] = 0.f;
   }
-  // merge another state (m2, l2, acc2) into this one
-  __device__ __forceinline__ void merge(float m2, float l2, const float (&a2)[VEC]) {
-    const float mn = fmaxf(m, m2);
-    const float f1 = (m == -INFINITY) ? 0.f : __expf(m - mn);
-    const float f2 = (m2 == -INFINITY) ? 0.f : __expf(m2 - mn);
-    l = l * f1 + l2 * f2;
+  __device__ __forceinline__ float extra(uint32_t s) const { return __ldg(scores + (uint64_t)s * (2 * heads) + head); }
+  __device__ __forceinline__ void edge(float (&st)[NS], const uint4 &raw, float, float x) const {
+    float e = x + s_dst;
+    e = e > 0.f ? e : slope * e;
+    const float m_new = fmaxf(st[VEC], e);
+    const float scale = __expf(st[VEC] - m_new);   // exp(-inf) = 0 for the first edge; m_new is finite
+    const float pw = __expf(e - m_new);
+    float f[VEC];
+    Row16<T>::unpack(raw, f);
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) acc[i] = acc[i] * f1 + a2[i] * f2;
-    m = mn;
+    for (int k = 0; k < VEC; ++k) st[k] = fmaf(pw, f[k], st[k] * scale);
+    st[VEC + 1] = fmaf(st[VEC + 1], scale, pw);
+    st[VEC] = m_new;
   }
-};
-
-template <typename T, int LPR, int GROUP>
-__device__ __forceinline__ void gat_edges(const GatParams &p, int64_t j0, int64_t j1, unsigned group_mask, int t,
-                                          float s_dst, SoftState<Vec16<T>::VEC> &st) {
-  constexpr int VEC = Vec16<T>::VEC;
-  constexpr int SLOTS = GROUP / LPR;
-  const int slot = t / LPR;
-  const int col = (t % LPR) * VEC;
-  const int head = col / p.head_dim;
-  const int sstride = 2 * p.heads;
-  const T *__restrict__ z = reinterpret_cast<const T *>(p.z);
-  for (int64_t base = j0; base < j1; base += GROUP) {
-    const int64_t mine = base + t;
-    const int32_t my_idx = mine < j1 ? __ldg(p.indices + mine) : 0;
-    const int cnt = (int)((j1 - base) < (int64_t)GROUP ? (j1 - base) : (int64_t)GROUP);
-    for (int k0 = 0; k0 < cnt; k0 += SLOTS * GAT_UNROLL) {
-      float v[GAT_UNROLL][VEC];
-      float e[GAT_UNROLL];
-      float mx = st.m;
+  __device__ __forceinline__ void merge(float (&st)[NS], const float (&o)[NS]) const {
+    const float m_new = fmaxf(st[VEC], o[VEC]);
+    const float f1 = st[VEC] == -INFINITY ? 0.f : __expf(st[VEC] - m_new);
+    const float f2 = o[VEC] == -INFINITY ? 0.f : __expf(o[VEC] - m_new);
 #pragma unroll
-      for (int u = 0; u < GAT_UNROLL; ++u) {
-        const int ei = k0 + u * SLOTS + slot;
-        const int32_t s = __shfl_sync(group_mask, my_idx, ei & (GROUP - 1), GROUP);
-        e[u] = -INFINITY;
-        if (ei < cnt) {
-          Vec16<T>::load(z + (int64_t)s * p.dim + col, v[u]);
-          const float x = __ldg(p.scores + (int64_t)s * sstride + head) + s_dst;
-          e[u] = x > 0.f ? x : p.slope * x;
-        }
+    for (int k = 0; k < VEC; ++k) st[k] = st[k] * f1 + o[k] * f2;
+    st[VEC + 1] = st[VEC + 1] * f1 + o[VEC + 1] * f2;
+    st[VEC] = m_new;
+  }
+  __device__ __forceinline__ void begin_row(int32_t, int32_t owner) {
+    s_dst = __ldg(scores + (int64_t)owner * (2 * heads) + heads + head);
+  }
+  __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t) const {
+    if (dest < 0) {   // a group of a split vertex: its state goes to the partial buffer
+      float *q = partials + (int64_t)(~dest) * gat_partial_stride(dim, heads);
+#pragma unroll
+      for (int i = 0; i < VEC; i += 4)
+        *reinterpret_cast<float4 *>(q + col + i) = make_float4(st[i], st[i + 1], st[i + 2], st[i + 3]);
+      if (col % head_dim == 0) {
+        q[dim + head] = st[VEC];
+        q[dim + heads + head] = st[VEC + 1];
       }
-#pragma unroll
-      for (int u = 0; u < GAT_UNROLL; ++u) mx = fmaxf(mx, e[u]);
-      if (mx == -INFINITY) continue;  // this slot saw no edge yet
-      const float scale = (st.m == -INFINITY) ? 0.f : __expf(st.m - mx);
-      st.l *= scale;
-#pragma unroll
-      for (int i = 0; i < VEC; ++i) st.acc[i] *= scale;
-      st.m = mx;
-#pragma unroll
-      for (int u = 0; u < GAT_UNROLL; ++u) {
-        if (e[u] != -INFINITY) {
-          const float pw = __expf(e[u] - mx);
-          st.l += pw;
-#pragma unroll
-          for (int i = 0; i < VEC; ++i) st.acc[i] = fmaf(pw, v[u][i], st.acc[i]);
-        }
-      }
+      return;
     }
+    const float inv = st[VEC + 1] > 0.f ? 1.f / st[VEC + 1] : 0.f;
+    float o[VEC];
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) o[i] = act_apply(st[i] * inv + (bias ? __ldg(bias + col + i) : 0.f), act);
+    Row16<T>::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, o);
   }
-}
+};
 
-template <int LPR, int GROUP, int VEC>
-__device__ __forceinline__ void fold_states(unsigned group_mask, SoftState<VEC> &st) {
-#pragma unroll
-  for (int o = GROUP / 2; o >= LPR; o >>= 1) {
-    const float m2 = __shfl_xor_sync(group_mask, st.m, o, GROUP);
-    const float l2 = __shfl_xor_sync(group_mask, st.l, o, GROUP);
-    float a2[VEC];
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) a2[i] = __shfl_xor_sync(group_mask, st.acc[i], o, GROUP);
-    // only slot 0 is read at the end, and it is always the first operand: the order is fixed
-    st.merge(m2, l2, a2);
-  }
-}
+// Merge the partial states of every split vertex in group order; one warp per vertex.
+struct GatCombineParams {
+  const int32_t *__restrict__ split_owners;
+  const int64_t *__restrict__ owner_indptr;
+  const float *__restrict__ partials;
+  const float *__restrict__ bias;
+  void *__restrict__ dst;
+  int64_t n_split_owners;
+  int dim, heads, head_dim, act;
+};
 
 template <typename T>
-__device__ __forceinline__ void gat_finish(const GatParams &p, int64_t v, int col, SoftState<Vec16<T>::VEC> &st) {
-  constexpr int VEC = Vec16<T>::VEC;
-  const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
-  float o[VEC];
-#pragma unroll
-  for (int i = 0; i < VEC; ++i) {
-    float x = st.acc[i] * inv;
-    if (p.bias) x += __ldg(p.bias + col + i);
-    o[i] = act_apply(x, p.act);
-  }
-  Vec16<T>::store(reinterpret_cast<T *>(p.dst) + v * p.dim + col, o);
-}
-
-template <typename T, int LPR, int GROUP>
-__global__ void __launch_bounds__(GAT_THREADS) gat_group_kernel(GatParams p) {
-  constexpr int VEC = Vec16<T>::VEC;
+__global__ void __launch_bounds__(THREADS) gat_combine_kernel(GatCombineParams p) {
   const int lane = threadIdx.x & 31;
-  const int t = lane % GROUP;
-  const unsigned group_mask = (GROUP == 32) ? 0xffffffffu : (((1u << (GROUP & 31)) - 1u) << (lane - t));
-  const int64_t groups_total = (int64_t)gridDim.x * (GAT_THREADS / GROUP);
-  const int64_t group_id = (int64_t)blockIdx.x * (GAT_THREADS / GROUP) + threadIdx.x / GROUP;
-  const int col = (t % LPR) * VEC;
-  const int head = col / p.head_dim;
-  for (int64_t i = p.row_lo + group_id; i < p.row_hi; i += groups_total) {
-    const int32_t r = __ldg(p.bucket_rows + i);
-    const int64_t v = __ldg(p.row_dest + r);  // graph is unsplit: row == vertex
-    const int64_t j0 = __ldg(p.shadow_indptr + r), j1 = __ldg(p.shadow_indptr + r + 1);
-    const float s_dst = __ldg(p.scores + v * 2 * p.heads + p.heads + head);
-    SoftState<VEC> st;
-    st.init();
-    gat_edges<T, LPR, GROUP>(p, j0, j1, group_mask, t, s_dst, st);
-    fold_states<LPR, GROUP, VEC>(group_mask, st);
-    if (t < LPR) gat_finish<T>(p, v, col, st);
-  }
-}
-
-template <typename T, int LPR>
-__global__ void __launch_bounds__(GAT_THREADS) gat_cta_kernel(GatParams p) {
-  constexpr int VEC = Vec16<T>::VEC;
-  constexpr int WARPS = GAT_THREADS / 32;
-  __shared__ float red[WARPS][LPR][VEC + 2];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col = (lane % LPR) * VEC;
-  const int head = col / p.head_dim;
-  for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {
-    const int32_t r = __ldg(p.bucket_rows + i);
-    const int64_t v = __ldg(p.row_dest + r);
-    const int64_t j0 = __ldg(p.shadow_indptr + r), j1 = __ldg(p.shadow_indptr + r + 1);
-    const float s_dst = __ldg(p.scores + v * 2 * p.heads + p.heads + head);
-    int64_t chunk = (j1 - j0 + WARPS - 1) / WARPS;
-    chunk = (chunk + 31) / 32 * 32;
-    int64_t a = j0 + warp * chunk, b = a + chunk;
-    if (a > j1) a = j1;
-    if (b > j1) b = j1;
-    SoftState<VEC> st;
-    st.init();
-    gat_edges<T, LPR, 32>(p, a, b, 0xffffffffu, lane, s_dst, st);
-    fold_states<LPR, 32, VEC>(0xffffffffu, st);
-    __syncthreads();
-    if (lane < LPR) {
-      red[warp][lane][0] = st.m; red[warp][lane][1] = st.l;
-#pragma unroll
-      for (int k = 0; k < VEC; ++k) red[warp][lane][2 + k] = st.acc[k];
-    }
-    __syncthreads();
-    if (warp == 0 && lane < LPR) {
-      for (int w = 1; w < WARPS; ++w) {
-        float a2[VEC];
-#pragma unroll
-        for (int k = 0; k < VEC; ++k) a2[k] = red[w][lane][2 + k];
-        st.merge(red[w][lane][0], red[w][lane][1], a2);
+  const int stride = gat_partial_stride(p.dim, p.heads);
+  const int64_t warps_total = (int64_t)gridDim.x * (THREADS / 32);
+  for (int64_t k = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); k < p.n_split_owners; k += warps_total) {
+    const int64_t v = __ldg(p.split_owners + k);
+    const int64_t r0 = __ldg(p.owner_indptr + v), r1 = __ldg(p.owner_indptr + v + 1);
+    const float *P = p.partials + (r0 - v + k) * stride;   // first partial row of this vertex
+    const int n = (int)(r1 - r0);
+    for (int c = lane * 4; c < p.dim; c += 128) {
+      const int head = c / p.head_dim;
+      float M = -INFINITY;
+      for (int g = 0; g < n; ++g) M = fmaxf(M, __ldg(P + (int64_t)g * stride + p.dim + head));
+      float l = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int g = 0; g < n; ++g) {
+        const float mg = __ldg(P + (int64_t)g * stride + p.dim + head);
+        const float f = mg == -INFINITY ? 0.f : __expf(mg - M);
+        l = fmaf(__ldg(P + (int64_t)g * stride + p.dim + p.heads + head), f, l);
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(P + (int64_t)g * stride + c));
+        acc.x = fmaf(a.x, f, acc.x); acc.y = fmaf(a.y, f, acc.y); acc.z = fmaf(a.z, f, acc.z); acc.w = fmaf(a.w, f, acc.w);
       }
-      gat_finish<T>(p, v, col, st);
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      float o[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) o[i] = act_apply(o[i] + (p.bias ? __ldg(p.bias + c + i) : 0.f), p.act);
+      T *d = reinterpret_cast<T *>(p.dst) + v * p.dim + c;
+      if (sizeof(T) == 4) {
+        *reinterpret_cast<float4 *>(d) = make_float4(o[0], o[1], o[2], o[3]);
+      } else {
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(o[0], o[1]), h1 = __floats2bfloat162_rn(o[2], o[3]);
+        *reinterpret_cast<uint2 *>(d) = make_uint2(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1));
+      }
     }
   }
 }
 
 template <typename T, int LPR>
-it_status launch_buckets(const it_graph *g, GatParams p, cudaStream_t st) {
-  for (int b = g->n_buckets - 1; b >= 0; --b) {
-    const int64_t lo = g->h_bucket_offsets[b], hi = g->h_bucket_offsets[b + 1];
-    if (hi <= lo) continue;
-    p.row_lo = lo; p.row_hi = hi;
-    const int64_t bound = g->bucket_bounds[b], rows = hi - lo;
-    const int64_t max_blocks = (int64_t)g->num_sms * 8;
-    // algorithmic bytes: per edge the index, one source score per head and one source row; per
-    // row its bounds, id, destination scores and one output row
-    const double row_bytes = (double)p.dim * sizeof(T);
-    const double bytes = (double)g->h_bucket_edges[b] * (4.0 + 4.0 * p.heads + row_bytes) +
-                         (double)rows * (16.0 + 8.0 + 4.0 * p.heads + row_bytes);
-    if (bound > 256) {
-      unsigned blocks = (unsigned)(rows < max_blocks ? rows : max_blocks);
-      IT_LAUNCH(IT_K_GAT_CTA, bytes, 0, st, gat_cta_kernel<T, LPR><<<blocks, GAT_THREADS, 0, st>>>(p));
-    } else if (bound > 8 || LPR == 32) {
-      int64_t want = (rows + (GAT_THREADS / 32) - 1) / (GAT_THREADS / 32);
-      unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
-      IT_LAUNCH(IT_K_GAT_WARP, bytes, 0, st, gat_group_kernel<T, LPR, 32><<<blocks, GAT_THREADS, 0, st>>>(p));
-    } else {
-      int64_t want = (rows + (GAT_THREADS / LPR) - 1) / (GAT_THREADS / LPR);
-      unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
-      IT_LAUNCH(IT_K_GAT_SUBWARP, bytes, 0, st, gat_group_kernel<T, LPR, LPR><<<blocks, GAT_THREADS, 0, st>>>(p));
-    }
-  }
-  IT_CUDA_TRY(cudaGetLastError());
-  return IT_OK;
+it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, cudaStream_t st) {
+  GatPolicy<T> pol;
+  pol.scores = a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
+  pol.dim = a.heads * a.head_dim; pol.heads = a.heads; pol.head_dim = a.head_dim; pol.act = a.act; pol.slope = a.slope;
+  pol.col = 0; pol.head = 0; pol.s_dst = 0.f;
+  const it_graph *g = a.g;
+  // algorithmic bytes: per edge the index, one source score per head and one source row; per row
+  // its metadata, owner, destination scores and one output row
+  const double row_bytes = (double)pol.dim * sizeof(T);
+  const int heads = a.heads;
+  auto bytes_of = [=](int b, int64_t rows) {
+    return (double)g->h_bucket_edges[b] * (4.0 + 4.0 * heads + row_bytes) + (double)rows * (20.0 + 4.0 * heads + row_bytes);
+  };
+  return launch_buckets<T, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, st);
 }
 
 template <typename T>
-it_status launch_lpr(const it_gat_args &a, GatParams p, cudaStream_t st) {
+it_status launch_gat(const it_gat_args &a, StreamParams sp, cudaStream_t st) {
   const int lpr = a.heads * a.head_dim * (int)sizeof(T) / 16;
   switch (lpr) {
-    case 1: return launch_buckets<T, 1>(a.g, p, st);
-    case 2: return launch_buckets<T, 2>(a.g, p, st);
-    case 4: return launch_buckets<T, 4>(a.g, p, st);
-    case 8: return launch_buckets<T, 8>(a.g, p, st);
-    case 16: return launch_buckets<T, 16>(a.g, p, st);
-    case 32: return launch_buckets<T, 32>(a.g, p, st);
+    case 1: return launch_gat_lpr<T, 1>(a, sp, st);
+    case 2: return launch_gat_lpr<T, 2>(a, sp, st);
+    case 4: return launch_gat_lpr<T, 4>(a, sp, st);
+    case 8: return launch_gat_lpr<T, 8>(a, sp, st);
+    case 16: return launch_gat_lpr<T, 16>(a, sp, st);
+    case 32: return launch_gat_lpr<T, 32>(a, sp, st);
   }
   it_set_error("gat: row of %d bytes is not 16, 32, 64, 128, 256 or 512 bytes", a.heads * a.head_dim * (int)sizeof(T));
   return IT_ERR_UNSUPPORTED;
@@ -271,16 +164,34 @@ it_status launch_lpr(const it_gat_args &a, GatParams p, cudaStream_t st) {
 
 }  // namespace
 
+size_t it_gat_partial_bytes(const it_graph *g, int dim, int heads) {
+  return (size_t)g->n_partial_rows * gat_partial_stride(dim, heads) * sizeof(float);
+}
+
 it_status it_launch_gat(const it_gat_args &a, cudaStream_t st) {
   const it_graph *g = a.g;
-  IT_REQUIRE(g->n_split_owners == 0, IT_ERR_UNSUPPORTED,
-             "GAT layers run on an unsplit graph (attention is reduced in apply_node, not by partial gather)");
   const int vec = a.dtype == IT_F32 ? 4 : 8;
   IT_REQUIRE(a.head_dim % vec == 0, IT_ERR_UNSUPPORTED, "gat: head_dim must be a multiple of %d", vec);
+  IT_REQUIRE(g->n_partial_rows == 0 || a.partials, IT_ERR_WORKSPACE, "gat: no partial buffer");
   if (g->n == 0) return IT_OK;
-  GatParams p;
-  p.shadow_indptr = g->shadow_indptr; p.indices = g->indices; p.bucket_rows = g->bucket_rows; p.row_dest = g->row_dest;
-  p.z = a.z; p.scores = a.scores; p.bias = a.bias; p.dst = a.dst; p.row_lo = p.row_hi = 0;
-  p.dim = a.heads * a.head_dim; p.heads = a.heads; p.head_dim = a.head_dim; p.act = a.act; p.slope = a.slope;
-  return a.dtype == IT_F32 ? launch_lpr<float>(a, p, st) : launch_lpr<__nv_bfloat16>(a, p, st);
+  StreamParams sp;
+  sp.meta = g->bucket_meta; sp.owner = g->bucket_owner; sp.indices = g->indices; sp.weights = nullptr;
+  sp.src = a.z; sp.row_lo = sp.row_hi = 0; sp.dim = a.heads * a.head_dim; sp.batch_rows = 1;
+  if (a.dtype == IT_F32) IT_TRY(launch_gat<float>(a, sp, st));
+  else IT_TRY(launch_gat<__nv_bfloat16>(a, sp, st));
+  if (g->n_split_owners > 0) {
+    GatCombineParams c;
+    c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.partials = a.partials; c.bias = a.bias;
+    c.dst = a.dst; c.n_split_owners = g->n_split_owners; c.dim = a.heads * a.head_dim; c.heads = a.heads;
+    c.head_dim = a.head_dim; c.act = a.act;
+    int64_t want = (g->n_split_owners + 7) / 8;
+    int64_t cap = (int64_t)g->num_sms * 8;
+    unsigned blocks = (unsigned)(want < cap ? want : cap);
+    const double cbytes = (double)it_gat_partial_bytes(g, c.dim, c.heads) +
+                          (double)g->n_split_owners * c.dim * (a.dtype == IT_F32 ? 4.0 : 2.0);
+    if (a.dtype == IT_F32) IT_LAUNCH(IT_K_COMBINE, cbytes, 0, st, gat_combine_kernel<float><<<blocks, THREADS, 0, st>>>(c));
+    else IT_LAUNCH(IT_K_COMBINE, cbytes, 0, st, gat_combine_kernel<__nv_bfloat16><<<blocks, THREADS, 0, st>>>(c));
+    IT_CUDA_TRY(cudaGetLastError());
+  }
+  return IT_OK;
 }

@@ -249,7 +249,8 @@ struct EdgesInBucket {
 };
 __global__ void fill_bucket_meta_kernel(int64_t n_rows, const int32_t *__restrict__ bucket_rows,
                                        const int64_t *__restrict__ sp, const int32_t *__restrict__ row_dest,
-                                       it_row_meta *__restrict__ meta) {
+                                       const int32_t *__restrict__ shadow_owner, it_row_meta *__restrict__ meta,
+                                       int32_t *__restrict__ bucket_owner) {
   int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (i >= n_rows) return;
   const int32_t r = bucket_rows[i];
@@ -258,6 +259,7 @@ __global__ void fill_bucket_meta_kernel(int64_t n_rows, const int32_t *__restric
   m.len = (int32_t)(sp[r + 1] - sp[r]);
   m.dest = row_dest[r];
   meta[i] = m;
+  bucket_owner[i] = shadow_owner[r];
 }
 __global__ void set_next_bucket_offset_kernel(int64_t *bucket_offsets, int which, const int64_t *count) {
   if (which == 0) bucket_offsets[0] = 0;
@@ -269,6 +271,7 @@ static void free_derived(it_graph *g) {
   cudaFree(g->shadow_indptr); cudaFree(g->shadow_owner); cudaFree(g->owner_indptr);
   cudaFree(g->row_dest); cudaFree(g->split_owners); cudaFree(g->bucket_offsets); cudaFree(g->bucket_rows);
   cudaFree(g->bucket_meta); g->bucket_meta = nullptr;
+  cudaFree(g->bucket_owner); g->bucket_owner = nullptr;
   g->shadow_indptr = nullptr; g->shadow_owner = nullptr; g->owner_indptr = nullptr; g->row_dest = nullptr;
   g->split_owners = nullptr; g->bucket_offsets = nullptr; g->bucket_rows = nullptr;
   g->n_rows = g->n_split_owners = g->n_partial_rows = 0;
@@ -316,6 +319,7 @@ static it_status split_impl(it_graph *g, int64_t T, cudaStream_t st) {
   SPLIT_CUDA(cudaMalloc(&g->split_owners, (size_t)(S > 0 ? S : 1) * sizeof(int32_t)));
   SPLIT_CUDA(cudaMalloc(&g->bucket_rows, (size_t)(R > 0 ? R : 1) * sizeof(int32_t)));
   SPLIT_CUDA(cudaMalloc(&g->bucket_meta, (size_t)(R > 0 ? R : 1) * sizeof(it_row_meta)));
+  SPLIT_CUDA(cudaMalloc(&g->bucket_owner, (size_t)(R > 0 ? R : 1) * sizeof(int32_t)));
   SPLIT_CUDA(cudaMalloc(&g->bucket_offsets, (IT_MAX_BUCKETS + 1) * sizeof(int64_t)));
   if (S > 0)
     SPLIT_TRY(scan_and_emit(IT_K_SPLIT_SCAN, n, IsSplit{ip, T}, EmitSplitOwner{ip, T, g->split_owners}, d_scratch, d_total + 1, st));
@@ -364,7 +368,7 @@ static it_status split_impl(it_graph *g, int64_t T, cudaStream_t st) {
   if (R > 0)
     IT_LAUNCH(IT_K_BUCKET_SCAN, 0, 0, st,
               fill_bucket_meta_kernel<<<(unsigned)((R + 255) / 256), 256, 0, st>>>(R, g->bucket_rows, g->shadow_indptr,
-                                                                                    g->row_dest, g->bucket_meta));
+                                                                                    g->row_dest, g->shadow_owner, g->bucket_meta, g->bucket_owner));
   SPLIT_CUDA(cudaGetLastError());
   SPLIT_CUDA(cudaMemcpyAsync(g->h_bucket_edges, d_edges, B.nb * sizeof(int64_t), cudaMemcpyDeviceToHost, st));
   SPLIT_CUDA(cudaMemcpyAsync(g->h_bucket_offsets, g->bucket_offsets, (B.nb + 1) * sizeof(int64_t),

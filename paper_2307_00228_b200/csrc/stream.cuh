@@ -1,0 +1,367 @@
+// Row-streaming machinery shared by the plain gather (sum / mean / max) and the GAT reduce.
+//
+// Both walk the in-edges of shadow rows and fold one 16-byte slice of every source row per
+// lane into a small per-lane state; they differ only in that state and its update (a Policy).
+// HBM-bound: one 16-byte load per lane per edge, several edges in flight per lane, a fixed
+// order of operations (results are bit-reproducible; no floating-point atomics anywhere).
+//
+// Work decomposition.  A feature row of `dim` elements is LPR = dim * sizeof(T) / 16 lanes wide.
+//   * stream_rows_kernel: a *group* of LPR lanes takes a batch of rows of its bucket (one coalesced
+//     16-byte metadata load per row) and walks the batch's edges as one flat stream: the lanes
+//     load LPR source ids at a time (the next chunk is prefetched while the current one is
+//     consumed), every id is broadcast by shuffle, all lanes load their slice of that source
+//     row, UNROLL rows in flight, and a row is finished when the stream crosses its end.
+//     Short rows therefore cost no dependent-load round trip of their own.
+//   * stream_cta_kernel: one CTA per very long row, each warp a contiguous chunk, SLOTS = 32 / LPR
+//     edges at once per warp; slot and warp states are merged in a fixed order.
+//
+// Policy interface (all __device__):
+//   static constexpr int NS;                 // floats of per-lane state
+//   static constexpr bool WEIGHTED, HAS_EXTRA, NEEDS_OWNER;
+//   void init(float (&st)[NS]);
+//   float extra(uint32_t src_row);           // per-edge scalar that is loaded with the row (HAS_EXTRA)
+//   void edge(float (&st)[NS], const uint4 &raw, float w, float x);
+//   void merge(float (&st)[NS], const float (&other)[NS]);     // other comes later in edge order
+//   void begin_row(int32_t dest, int32_t owner);               // prefetch what end_row needs
+//   void end_row(float (&st)[NS], int32_t dest, int32_t owner, int64_t len);
+#pragma once
+
+#include "common.cuh"
+
+#ifndef IT_GATHER_UNROLL
+#define IT_GATHER_UNROLL 4   // source rows in flight per lane
+#endif
+#ifndef IT_GATHER_MIN_BLOCKS
+#define IT_GATHER_MIN_BLOCKS 4   // resident CTAs per SM the register budget is set for
+#endif
+#ifndef IT_GATHER_CTA_ABOVE
+#define IT_GATHER_CTA_ABOVE 2048   // rows longer than this get a whole CTA; shorter ones a lane group
+#endif
+
+namespace it_stream {
+
+constexpr int THREADS = 256;
+constexpr int UNROLL = IT_GATHER_UNROLL;
+
+template <typename T> struct Row16;
+template <> struct Row16<float> {
+  static constexpr int VEC = 4;
+  __device__ static __forceinline__ void unpack(const uint4 &x, float (&v)[4]) {
+    v[0] = __uint_as_float(x.x); v[1] = __uint_as_float(x.y); v[2] = __uint_as_float(x.z); v[3] = __uint_as_float(x.w);
+  }
+  __device__ static __forceinline__ void store(float *p, const float (&v)[4]) {
+    __stcs(reinterpret_cast<float4 *>(p), make_float4(v[0], v[1], v[2], v[3]));
+  }
+};
+template <> struct Row16<__nv_bfloat16> {
+  static constexpr int VEC = 8;
+  __device__ static __forceinline__ void unpack(const uint4 &x, float (&v)[8]) {
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static __forceinline__ void store(__nv_bfloat16 *p, const float (&v)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t *>(&h);
+    }
+    __stcs(reinterpret_cast<uint4 *>(p), make_uint4(w[0], w[1], w[2], w[3]));
+  }
+};
+
+__device__ __forceinline__ float act_apply(float x, int act) {
+  if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
+  if (act == IT_ACT_ELU) return x > 0.f ? x : expm1f(x);
+  return x;
+}
+
+// What every streaming kernel needs besides its policy.
+struct StreamParams {
+  const it_row_meta *__restrict__ meta;   // bucket order
+  const int32_t *__restrict__ owner;      // bucket order: vertex a row belongs to (policies with NEEDS_OWNER)
+  const int32_t *__restrict__ indices;
+  const float *__restrict__ weights;
+  const void *__restrict__ src;           // [n, dim] rows that are gathered
+  int64_t row_lo, row_hi;                 // range inside the bucket-ordered row list
+  int dim;
+  int batch_rows;                         // rows a lane group takes at a time (<= LPR)
+};
+
+__device__ __forceinline__ it_row_meta load_meta(const it_row_meta *p) {
+  const int4 raw = __ldcs(reinterpret_cast<const int4 *>(p));
+  it_row_meta m;
+  m.j0 = (int64_t)(((uint64_t)(uint32_t)raw.y << 32) | (uint32_t)raw.x);
+  m.len = raw.z;
+  m.dest = raw.w;
+  return m;
+}
+
+// ----------------------------------------------------------------------------- batches of rows per lane group
+// Rows handled here have at least one edge: empty rows live in their own bucket.
+template <typename T, int LPR, class Policy>
+__global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_kernel(StreamParams p, Policy pol) {
+  constexpr int G = LPR;
+  constexpr int U = UNROLL < G ? UNROLL : G;
+  constexpr int NS = Policy::NS;
+  const int lane = threadIdx.x & 31;
+  const int t = lane % G;
+  const unsigned gbits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
+  const unsigned gmask = gbits << (lane - t);
+  pol.setup(t);
+  const int64_t n_rows = p.row_hi - p.row_lo;
+  const int BR = p.batch_rows;  // rows per batch, <= G: lanes t < BR hold their metadata
+  const int64_t n_batches = (n_rows + BR - 1) / BR;
+  const int64_t groups_total = (int64_t)gridDim.x * (THREADS / G);
+  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * 16;
+  const uint32_t row_bytes = (uint32_t)p.dim * (uint32_t)sizeof(T);
+
+  for (int64_t b = (int64_t)blockIdx.x * (THREADS / G) + threadIdx.x / G; b < n_batches; b += groups_total) {
+    // ---- batch metadata: lane t owns row t of the batch
+    const int64_t i = p.row_lo + b * BR + t;
+    int64_t my_j0 = 0;
+    int my_len = 0, my_dest = 0, my_owner = 0;
+    if (t < BR && i < p.row_hi) {
+      const it_row_meta m = load_meta(p.meta + i);
+      my_j0 = m.j0; my_len = m.len; my_dest = m.dest;
+      if (Policy::NEEDS_OWNER) my_owner = __ldcs(p.owner + i);
+    }
+    int my_end = my_len;  // inclusive prefix sum of the row lengths
+#pragma unroll
+    for (int o = 1; o < G; o <<= 1) {
+      const int y = __shfl_up_sync(gmask, my_end, o, G);
+      if (t >= o) my_end += y;
+    }
+    const int total = __shfl_sync(gmask, my_end, G - 1, G);
+    const int my_start = my_end - my_len;
+
+    // ---- one chunk of the flat edge stream: lane t fetches edge (base + t) and learns whether it
+    // is the last edge of its row; `ends` collects those flags for the whole chunk.
+    auto load_chunk = [&](int base, int32_t &idx, float &w, unsigned &ends) {
+      const int q = base + t;
+      int lo = 0;
+#pragma unroll
+      for (int step = G / 2; step >= 1; step >>= 1) {
+        const int e = __shfl_sync(gmask, my_end, lo + step - 1, G);
+        if (e <= q) lo += step;
+      }
+      const int row_end = __shfl_sync(gmask, my_end, lo, G);
+      const int64_t j = __shfl_sync(gmask, my_j0, lo, G) + (q - __shfl_sync(gmask, my_start, lo, G));
+      idx = 0;
+      w = 1.f;
+      if (q < total) {
+        idx = __ldcs(p.indices + j);
+        if (Policy::WEIGHTED) w = __ldcs(p.weights + j);
+      }
+      ends = (__ballot_sync(gmask, q < total && q + 1 == row_end) >> (lane - t)) & gbits;
+    };
+
+    float st[NS];
+    pol.init(st);
+    int cur = 0;  // row of the batch that st belongs to
+    pol.begin_row(__shfl_sync(gmask, my_dest, 0, G), __shfl_sync(gmask, my_owner, 0, G));
+    auto next_row = [&]() {
+      pol.end_row(st, __shfl_sync(gmask, my_dest, cur, G), __shfl_sync(gmask, my_owner, cur, G),
+                  __shfl_sync(gmask, my_len, cur, G));
+      ++cur;
+      pol.init(st);
+      const int32_t nd = __shfl_sync(gmask, my_dest, cur & (G - 1), G);
+      const int32_t no = __shfl_sync(gmask, my_owner, cur & (G - 1), G);
+      if (cur < BR && __shfl_sync(gmask, my_len, cur & (G - 1), G) > 0) pol.begin_row(nd, no);
+    };
+
+    int32_t idx_c, idx_n;
+    float w_c, w_n;
+    unsigned ends_c, ends_n;
+    load_chunk(0, idx_c, w_c, ends_c);
+    for (int base = 0; base < total; base += G) {
+      load_chunk(base + G, idx_n, w_n, ends_n);  // in flight while this chunk is consumed
+      const int cnt = (total - base) < G ? (total - base) : G;
+      int k0 = 0;
+      for (; k0 + U <= cnt; k0 += U) {  // full groups of U edges: no predicates
+        uint4 v[U];
+        float w[U], x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const uint32_t s = (uint32_t)__shfl_sync(gmask, idx_c, k0 + u, G);
+          w[u] = Policy::WEIGHTED ? __shfl_sync(gmask, w_c, k0 + u, G) : 1.f;
+          v[u] = __ldg(reinterpret_cast<const uint4 *>(my_src + (uint64_t)s * row_bytes));
+          x[u] = Policy::HAS_EXTRA ? pol.extra(s) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          pol.edge(st, v[u], w[u], x[u]);
+          if ((ends_c >> (k0 + u)) & 1u) next_row();  // group-uniform
+        }
+      }
+      if (k0 < cnt) {  // tail of the chunk
+        uint4 v[U];
+        float w[U], x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int e = k0 + u;
+          const uint32_t s = (uint32_t)__shfl_sync(gmask, idx_c, e & (G - 1), G);
+          w[u] = Policy::WEIGHTED ? __shfl_sync(gmask, w_c, e & (G - 1), G) : 1.f;
+          x[u] = 0.f;
+          if (e < cnt) {
+            v[u] = __ldg(reinterpret_cast<const uint4 *>(my_src + (uint64_t)s * row_bytes));
+            if (Policy::HAS_EXTRA) x[u] = pol.extra(s);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (k0 + u < cnt) {
+            pol.edge(st, v[u], w[u], x[u]);
+            if ((ends_c >> (k0 + u)) & 1u) next_row();
+          }
+        }
+      }
+      idx_c = idx_n; w_c = w_n; ends_c = ends_n;
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- very long rows: one CTA each
+template <typename T, int LPR, class Policy>
+__global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kernel(StreamParams p, Policy pol) {
+  constexpr int NS = Policy::NS;
+  constexpr int WARPS = THREADS / 32;
+  constexpr int SLOTS = 32 / LPR;
+  constexpr int U = UNROLL;
+  __shared__ float red[WARPS][LPR][NS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int slot = lane / LPR, t = lane % LPR;
+  pol.setup(t);
+  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * 16;
+  const uint32_t row_bytes = (uint32_t)p.dim * (uint32_t)sizeof(T);
+  for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {
+    const it_row_meta m = load_meta(p.meta + i);
+    const int32_t owner = Policy::NEEDS_OWNER ? __ldcs(p.owner + i) : 0;
+    const int64_t j0 = m.j0, j1 = m.j0 + m.len;
+    const int64_t chunk = ((int64_t)m.len + WARPS - 1) / WARPS;
+    int64_t a = j0 + warp * chunk, b = a + chunk;
+    if (a > j1) a = j1;
+    if (b > j1) b = j1;
+    float st[NS];
+    pol.init(st);
+    pol.begin_row(m.dest, owner);
+    // edges [a, b) with the whole warp: SLOTS edges at once, index chunk of 32 prefetched one step ahead
+    auto load_chunk = [&](int64_t base, int32_t &idx, float &w) {
+      idx = 0; w = 1.f;
+      if (base + lane < b) {
+        idx = __ldcs(p.indices + base + lane);
+        if (Policy::WEIGHTED) w = __ldcs(p.weights + base + lane);
+      }
+    };
+    int32_t idx_c, idx_n;
+    float w_c, w_n;
+    load_chunk(a, idx_c, w_c);
+    for (int64_t base = a; base < b; base += 32) {
+      load_chunk(base + 32, idx_n, w_n);
+      const int cnt = (int)((b - base) < 32 ? (b - base) : 32);
+      for (int k0 = 0; k0 < cnt; k0 += SLOTS * U) {
+        uint4 v[U];
+        float w[U], x[U];
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int e = k0 + u * SLOTS + slot;
+          const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idx_c, e & 31);
+          w[u] = Policy::WEIGHTED ? __shfl_sync(0xffffffffu, w_c, e & 31) : 1.f;
+          ok[u] = e < cnt;
+          x[u] = 0.f;
+          if (ok[u]) {
+            v[u] = __ldg(reinterpret_cast<const uint4 *>(my_src + (uint64_t)s * row_bytes));
+            if (Policy::HAS_EXTRA) x[u] = pol.extra(s);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+          if (ok[u]) pol.edge(st, v[u], w[u], x[u]);
+      }
+      idx_c = idx_n; w_c = w_n;
+    }
+    // fold the SLOTS edge slots into slot 0, lower slot first
+#pragma unroll
+    for (int o = 16; o >= LPR; o >>= 1) {
+      float other[NS];
+#pragma unroll
+      for (int k = 0; k < NS; ++k) other[k] = __shfl_xor_sync(0xffffffffu, st[k], o);
+      pol.merge(st, other);   // only slot 0 is read at the end, and it is always the first operand
+    }
+    __syncthreads();  // red[] free again
+    if (lane < LPR) {
+#pragma unroll
+      for (int k = 0; k < NS; ++k) red[warp][lane][k] = st[k];
+    }
+    __syncthreads();
+    if (warp == 0 && lane < LPR) {
+      for (int w = 1; w < WARPS; ++w) {
+        float other[NS];
+#pragma unroll
+        for (int k = 0; k < NS; ++k) other[k] = red[w][lane][k];
+        pol.merge(st, other);
+      }
+      pol.end_row(st, m.dest, owner, m.len);
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- empty rows
+template <typename T, int LPR, class Policy>
+__global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, Policy pol) {
+  constexpr int NS = Policy::NS;
+  const int t = threadIdx.x % LPR;
+  pol.setup(t);
+  const int64_t groups_total = (int64_t)gridDim.x * (THREADS / LPR);
+  for (int64_t i = p.row_lo + (int64_t)blockIdx.x * (THREADS / LPR) + threadIdx.x / LPR; i < p.row_hi; i += groups_total) {
+    const it_row_meta m = load_meta(p.meta + i);
+    const int32_t owner = Policy::NEEDS_OWNER ? __ldcs(p.owner + i) : 0;
+    float st[NS];
+    pol.init(st);
+    pol.begin_row(m.dest, owner);
+    pol.end_row(st, m.dest, owner, 0);
+  }
+}
+
+// ----------------------------------------------------------------------------- bucket dispatch
+// Longest rows first so that the tail of the launch sequence is made of short rows.
+// bytes_of(bucket, rows) gives the algorithmic bytes of a launch; kid_* the instrumentation ids.
+template <typename T, int LPR, class Policy, class BytesF>
+it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, BytesF bytes_of, int kid_cta, int kid_rows,
+                         int kid_empty, cudaStream_t st) {
+  for (int b = g->n_buckets - 1; b >= 0; --b) {
+    const int64_t lo = g->h_bucket_offsets[b], hi = g->h_bucket_offsets[b + 1];
+    if (hi <= lo) continue;
+    p.row_lo = lo; p.row_hi = hi;
+    const int64_t bound = g->bucket_bounds[b];
+    const int64_t rows = hi - lo;
+    const int64_t max_blocks = (int64_t)g->num_sms * IT_GATHER_MIN_BLOCKS * 2;
+    const double bytes = bytes_of(b, rows);
+    if (bound == 0) {
+      int64_t want = (rows + (THREADS / LPR) - 1) / (THREADS / LPR);
+      unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
+      IT_LAUNCH(kid_empty, bytes, 0, st, stream_empty_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+    } else if (bound > IT_GATHER_CTA_ABOVE) {
+      unsigned blocks = (unsigned)(rows < max_blocks ? rows : max_blocks);
+      IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+    } else {
+      // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
+      int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
+      if (br > LPR) br = LPR;
+      p.batch_rows = br;
+      const int64_t batches = (rows + br - 1) / br;
+      int64_t want = (batches + (THREADS / LPR) - 1) / (THREADS / LPR);
+      unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
+      IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+    }
+  }
+  IT_CUDA_TRY(cudaGetLastError());
+  return IT_OK;
+}
+
+}  // namespace it_stream
