@@ -13,9 +13,10 @@ using namespace it_stream;
 
 __host__ __device__ inline int gat_partial_stride(int dim, int heads) { return dim + ((2 * heads + 3) / 4) * 4; }
 
-template <typename T>
+template <typename T, int SB>
 struct GatPolicy {
-  static constexpr int VEC = Row16<T>::VEC;
+  using Slice = RowSlice<T, SB>;
+  static constexpr int VEC = Slice::VEC;
   static constexpr int NS = VEC + 2;   // accumulators, running max, running sum
   static constexpr bool WEIGHTED = false, HAS_EXTRA = true, NEEDS_OWNER = true;
   const float *__restrict__ scores;    // [n, 2*heads]: source scores of the vertex, then its destination scores
@@ -36,14 +37,14 @@ struct GatPolicy {
     st[VEC + 1] = 0.f;
   }
   __device__ __forceinline__ float extra(uint32_t s) const { return __ldg(scores + (uint64_t)s * (2 * heads) + head); }
-  __device__ __forceinline__ void edge(float (&st)[NS], const uint4 &raw, float, float x) const {
+  __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float, float x) const {
     float e = x + s_dst;
     e = e > 0.f ? e : slope * e;
     const float m_new = fmaxf(st[VEC], e);
     const float scale = __expf(st[VEC] - m_new);   // exp(-inf) = 0 for the first edge; m_new is finite
     const float pw = __expf(e - m_new);
     float f[VEC];
-    Row16<T>::unpack(raw, f);
+    Slice::unpack(raw, f);
 #pragma unroll
     for (int k = 0; k < VEC; ++k) st[k] = fmaf(pw, f[k], st[k] * scale);
     st[VEC + 1] = fmaf(st[VEC + 1], scale, pw);
@@ -64,9 +65,10 @@ struct GatPolicy {
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t) const {
     if (dest < 0) {   // a group of a split vertex: its state goes to the partial buffer
       float *q = partials + (int64_t)(~dest) * gat_partial_stride(dim, heads);
+      float a[VEC];
 #pragma unroll
-      for (int i = 0; i < VEC; i += 4)
-        *reinterpret_cast<float4 *>(q + col + i) = make_float4(st[i], st[i + 1], st[i + 2], st[i + 3]);
+      for (int i = 0; i < VEC; ++i) a[i] = st[i];
+      store_floats<VEC>(q + col, a);
       if (col % head_dim == 0) {
         q[dim + head] = st[VEC];
         q[dim + heads + head] = st[VEC + 1];
@@ -77,7 +79,7 @@ struct GatPolicy {
     float o[VEC];
 #pragma unroll
     for (int i = 0; i < VEC; ++i) o[i] = act_apply(st[i] * inv + (bias ? __ldg(bias + col + i) : 0.f), act);
-    Row16<T>::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, o);
+    Slice::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, o);
   }
 };
 
@@ -130,9 +132,9 @@ __global__ void __launch_bounds__(THREADS) gat_combine_kernel(GatCombineParams p
   }
 }
 
-template <typename T, int LPR>
+template <typename T, int SB, int LPR>
 it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, cudaStream_t st) {
-  GatPolicy<T> pol;
+  GatPolicy<T, SB> pol;
   pol.scores = a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
   pol.dim = a.heads * a.head_dim; pol.heads = a.heads; pol.head_dim = a.head_dim; pol.act = a.act; pol.slope = a.slope;
   pol.col = 0; pol.head = 0; pol.s_dst = 0.f;
@@ -144,22 +146,18 @@ it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, cudaStream_t st)
   auto bytes_of = [=](int b, int64_t rows) {
     return (double)g->h_bucket_edges[b] * (4.0 + 4.0 * heads + row_bytes) + (double)rows * (20.0 + 4.0 * heads + row_bytes);
   };
-  return launch_buckets<T, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, st);
+  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, st);
 }
 
 template <typename T>
 it_status launch_gat(const it_gat_args &a, StreamParams sp, cudaStream_t st) {
-  const int lpr = a.heads * a.head_dim * (int)sizeof(T) / 16;
-  switch (lpr) {
-    case 1: return launch_gat_lpr<T, 1>(a, sp, st);
-    case 2: return launch_gat_lpr<T, 2>(a, sp, st);
-    case 4: return launch_gat_lpr<T, 4>(a, sp, st);
-    case 8: return launch_gat_lpr<T, 8>(a, sp, st);
-    case 16: return launch_gat_lpr<T, 16>(a, sp, st);
-    case 32: return launch_gat_lpr<T, 32>(a, sp, st);
-  }
-  it_set_error("gat: row of %d bytes is not 16, 32, 64, 128, 256 or 512 bytes", a.heads * a.head_dim * (int)sizeof(T));
-  return IT_ERR_UNSUPPORTED;
+  return dispatch_row_bytes(a.heads * a.head_dim * (int)sizeof(T), [&]<int SB, int LPR>() {
+    if ((a.head_dim * (int)sizeof(T)) % SB != 0) {
+      it_set_error("gat: a %d-byte lane slice would straddle two heads (head_dim %d)", SB, a.head_dim);
+      return IT_ERR_UNSUPPORTED;
+    }
+    return launch_gat_lpr<T, SB, LPR>(a, sp, st);
+  });
 }
 
 }  // namespace
@@ -170,9 +168,8 @@ size_t it_gat_partial_bytes(const it_graph *g, int dim, int heads) {
 
 it_status it_launch_gat(const it_gat_args &a, cudaStream_t st) {
   const it_graph *g = a.g;
-  const int vec = a.dtype == IT_F32 ? 4 : 8;
-  IT_REQUIRE(a.head_dim % vec == 0, IT_ERR_UNSUPPORTED, "gat: head_dim must be a multiple of %d", vec);
   IT_REQUIRE(g->n_partial_rows == 0 || a.partials, IT_ERR_WORKSPACE, "gat: no partial buffer");
+  IT_REQUIRE(g->n_split_owners == 0 || a.head_dim % 4 == 0, IT_ERR_UNSUPPORTED, "gat on a split graph needs head_dim to be a multiple of 4");
   if (g->n == 0) return IT_OK;
   StreamParams sp;
   sp.meta = g->bucket_meta; sp.owner = g->bucket_owner; sp.indices = g->indices; sp.weights = nullptr;

@@ -8,10 +8,11 @@ namespace {
 using namespace it_stream;
 constexpr int GATHER_THREADS = THREADS;
 
-// Per lane: VEC fp32 accumulators for its 16-byte slice of the row.
-template <typename T, bool IS_MAX, bool WEIGHTED_>
+// Per lane: VEC fp32 accumulators for its slice of the row.
+template <typename T, int SB, bool IS_MAX, bool WEIGHTED_>
 struct SagePolicy {
-  static constexpr int VEC = Row16<T>::VEC;
+  using Slice = RowSlice<T, SB>;
+  static constexpr int VEC = Slice::VEC;
   static constexpr int NS = VEC;
   static constexpr bool WEIGHTED = WEIGHTED_, HAS_EXTRA = false, NEEDS_OWNER = false;
   float *__restrict__ partials;
@@ -28,9 +29,9 @@ struct SagePolicy {
     for (int k = 0; k < NS; ++k) st[k] = IS_MAX ? -INFINITY : 0.f;
   }
   __device__ __forceinline__ float extra(uint32_t) const { return 0.f; }
-  __device__ __forceinline__ void edge(float (&st)[NS], const uint4 &raw, float w, float) const {
+  __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float w, float) const {
     float f[VEC];
-    Row16<T>::unpack(raw, f);
+    Slice::unpack(raw, f);
 #pragma unroll
     for (int k = 0; k < VEC; ++k) {
       if (IS_MAX) st[k] = fmaxf(st[k], WEIGHTED ? w * f[k] : f[k]);
@@ -43,13 +44,7 @@ struct SagePolicy {
   }
   // the matching slice of the self term is fetched when the row starts, so that end_row does not wait for it
   __device__ __forceinline__ void begin_row(int32_t dest, int32_t) {
-    if (epi == IT_EPI_ADD_ACT && dest >= 0) {
-#pragma unroll
-      for (int i = 0; i < VEC; i += 4) {
-        const float4 s4 = __ldcs(reinterpret_cast<const float4 *>(self_term + (int64_t)dest * dim + col + i));
-        self[i] = s4.x; self[i + 1] = s4.y; self[i + 2] = s4.z; self[i + 3] = s4.w;
-      }
-    }
+    if (epi == IT_EPI_ADD_ACT && dest >= 0) load_floats_stream<VEC>(self_term + (int64_t)dest * dim + col, self);
   }
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t len) const {
     if (IS_MAX && len == 0) {
@@ -57,10 +52,7 @@ struct SagePolicy {
       for (int i = 0; i < VEC; ++i) st[i] = 0.f;
     }
     if (dest < 0) {  // a group of a split vertex: raw partial, finished by the combine kernel
-      float *q = partials + (int64_t)(~dest) * dim + col;
-#pragma unroll
-      for (int i = 0; i < VEC; i += 4)
-        *reinterpret_cast<float4 *>(q + i) = make_float4(st[i], st[i + 1], st[i + 2], st[i + 3]);
+      store_floats<VEC>(partials + (int64_t)(~dest) * dim + col, st);
       return;
     }
     if (is_mean && len > 0) {
@@ -72,7 +64,7 @@ struct SagePolicy {
 #pragma unroll
       for (int i = 0; i < VEC; ++i) st[i] = act_apply(st[i] + self[i], act);
     }
-    Row16<T>::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, st);
+    Slice::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, st);
   }
 };
 
@@ -130,9 +122,9 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 }
 
 // ----------------------------------------------------------------------------- dispatch
-template <typename T, int LPR, bool IS_MAX, bool WEIGHTED>
+template <typename T, int SB, int LPR, bool IS_MAX, bool WEIGHTED>
 it_status launch_policy(const it_gather_args &a, StreamParams sp, cudaStream_t st) {
-  SagePolicy<T, IS_MAX, WEIGHTED> pol;
+  SagePolicy<T, SB, IS_MAX, WEIGHTED> pol;
   pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.dim = a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
   const it_graph *g = a.g;
@@ -143,29 +135,16 @@ it_status launch_policy(const it_gather_args &a, StreamParams sp, cudaStream_t s
     return (double)g->h_bucket_edges[b] * (4.0 + (WEIGHTED ? 4.0 : 0.0) + row_bytes) +
            (double)rows * (16.0 + row_bytes + (a.epi == IT_EPI_ADD_ACT ? 4.0 * a.dim : 0.0));
   };
-  return launch_buckets<T, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, st);
-}
-
-template <typename T, int LPR>
-it_status launch_ops(const it_gather_args &a, StreamParams sp, cudaStream_t st) {
-  const bool mx = a.op == IT_GATHER_MAX, w = a.use_edge_weights != 0;
-  if (mx) return w ? launch_policy<T, LPR, true, true>(a, sp, st) : launch_policy<T, LPR, true, false>(a, sp, st);
-  return w ? launch_policy<T, LPR, false, true>(a, sp, st) : launch_policy<T, LPR, false, false>(a, sp, st);
+  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, st);
 }
 
 template <typename T>
 it_status launch_lpr(const it_gather_args &a, StreamParams sp, cudaStream_t st) {
-  const int lpr = a.dim * (int)sizeof(T) / 16;
-  switch (lpr) {
-    case 1: return launch_ops<T, 1>(a, sp, st);
-    case 2: return launch_ops<T, 2>(a, sp, st);
-    case 4: return launch_ops<T, 4>(a, sp, st);
-    case 8: return launch_ops<T, 8>(a, sp, st);
-    case 16: return launch_ops<T, 16>(a, sp, st);
-    case 32: return launch_ops<T, 32>(a, sp, st);
-  }
-  it_set_error("gather: row of %d x %d bytes is not 16, 32, 64, 128, 256 or 512 bytes", a.dim, (int)sizeof(T));
-  return IT_ERR_UNSUPPORTED;
+  const bool mx = a.op == IT_GATHER_MAX, w = a.use_edge_weights != 0;
+  return dispatch_row_bytes(a.dim * (int)sizeof(T), [&]<int SB, int LPR>() {
+    if (mx) return w ? launch_policy<T, SB, LPR, true, true>(a, sp, st) : launch_policy<T, SB, LPR, true, false>(a, sp, st);
+    return w ? launch_policy<T, SB, LPR, false, true>(a, sp, st) : launch_policy<T, SB, LPR, false, false>(a, sp, st);
+  });
 }
 
 }  // namespace

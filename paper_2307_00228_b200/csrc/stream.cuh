@@ -1,11 +1,11 @@
 // Row-streaming machinery shared by the plain gather (sum / mean / max) and the GAT reduce.
 //
-// Both walk the in-edges of shadow rows and fold one 16-byte slice of every source row per
+// Both walk the in-edges of shadow rows and fold one slice of every source row per
 // lane into a small per-lane state; they differ only in that state and its update (a Policy).
-// HBM-bound: one 16-byte load per lane per edge, several edges in flight per lane, a fixed
+// HBM-bound: one 4- to 16-byte load per lane per edge, several edges in flight per lane, a fixed
 // order of operations (results are bit-reproducible; no floating-point atomics anywhere).
 //
-// Work decomposition.  A feature row of `dim` elements is LPR = dim * sizeof(T) / 16 lanes wide.
+// Work decomposition.  A feature row is LPR lanes wide (32 for rows of 128 bytes and more).
 //   * stream_rows_kernel: a *group* of LPR lanes takes a batch of rows of its bucket (one coalesced
 //     16-byte metadata load per row) and walks the batch's edges as one flat stream: the lanes
 //     load LPR source ids at a time (the next chunk is prefetched while the current one is
@@ -20,7 +20,7 @@
 //   static constexpr bool WEIGHTED, HAS_EXTRA, NEEDS_OWNER;
 //   void init(float (&st)[NS]);
 //   float extra(uint32_t src_row);           // per-edge scalar that is loaded with the row (HAS_EXTRA)
-//   void edge(float (&st)[NS], const uint4 &raw, float w, float x);
+//   void edge(float (&st)[NS], const Raw &raw, float w, float x);   // Raw = the packed slice
 //   void merge(float (&st)[NS], const float (&other)[NS]);     // other comes later in edge order
 //   void begin_row(int32_t dest, int32_t owner);               // prefetch what end_row needs
 //   void end_row(float (&st)[NS], int32_t dest, int32_t owner, int64_t len);
@@ -43,36 +43,85 @@ namespace it_stream {
 constexpr int THREADS = 256;
 constexpr int UNROLL = IT_GATHER_UNROLL;
 
-template <typename T> struct Row16;
-template <> struct Row16<float> {
-  static constexpr int VEC = 4;
-  __device__ static __forceinline__ void unpack(const uint4 &x, float (&v)[4]) {
-    v[0] = __uint_as_float(x.x); v[1] = __uint_as_float(x.y); v[2] = __uint_as_float(x.z); v[3] = __uint_as_float(x.w);
-  }
-  __device__ static __forceinline__ void store(float *p, const float (&v)[4]) {
-    __stcs(reinterpret_cast<float4 *>(p), make_float4(v[0], v[1], v[2], v[3]));
-  }
-};
-template <> struct Row16<__nv_bfloat16> {
-  static constexpr int VEC = 8;
-  __device__ static __forceinline__ void unpack(const uint4 &x, float (&v)[8]) {
-    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+// One lane's slice of a feature row: SB = 4, 8 or 16 bytes.  Rows of 128 bytes and more are spread
+// over all 32 lanes of a warp (SB = row bytes / 32), so that every load instruction fetches one whole
+// row and a warp never has to split into independently running lane groups; narrower rows use 4-byte
+// slices and a group of LPR = row bytes / 4 lanes.  A slice stays packed in registers while it is in
+// flight and is widened to fp32 only when it is consumed.
+template <int SB> struct SliceRaw;
+template <> struct SliceRaw<4> { using type = uint32_t; };
+template <> struct SliceRaw<8> { using type = uint2; };
+template <> struct SliceRaw<16> { using type = uint4; };
+
+template <int SB>
+__device__ __forceinline__ void raw_words(const typename SliceRaw<SB>::type &x, uint32_t (&w)[SB / 4]) {
+  if constexpr (SB == 4) { w[0] = x; }
+  else if constexpr (SB == 8) { w[0] = x.x; w[1] = x.y; }
+  else { w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
+}
+template <int SB>
+__device__ __forceinline__ typename SliceRaw<SB>::type words_raw(const uint32_t (&w)[SB / 4]) {
+  if constexpr (SB == 4) return w[0];
+  else if constexpr (SB == 8) return make_uint2(w[0], w[1]);
+  else return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <typename T, int SB> struct RowSlice {
+  static constexpr int VEC = SB / (int)sizeof(T);
+  using Raw = typename SliceRaw<SB>::type;
+  __device__ static __forceinline__ Raw load(const char *p) { return __ldg(reinterpret_cast<const Raw *>(p)); }
+  __device__ static __forceinline__ void unpack(const Raw &x, float (&v)[VEC]) {
+    uint32_t w[SB / 4];
+    raw_words<SB>(x, w);
+    if constexpr (sizeof(T) == 4) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(w[i] << 16);
-      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+      for (int i = 0; i < VEC; ++i) v[i] = __uint_as_float(w[i]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < SB / 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+      }
     }
   }
-  __device__ static __forceinline__ void store(__nv_bfloat16 *p, const float (&v)[8]) {
-    uint32_t w[4];
+  __device__ static __forceinline__ void store(T *p, const float (&v)[VEC]) {
+    uint32_t w[SB / 4];
+    if constexpr (sizeof(T) == 4) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-      w[i] = *reinterpret_cast<uint32_t *>(&h);
+      for (int i = 0; i < VEC; ++i) w[i] = __float_as_uint(v[i]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < SB / 4; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t *>(&h);
+      }
     }
-    __stcs(reinterpret_cast<uint4 *>(p), make_uint4(w[0], w[1], w[2], w[3]));
+    __stcs(reinterpret_cast<Raw *>(p), words_raw<SB>(w));
   }
 };
+
+// VEC consecutive fp32 values (VEC = 1, 2, 4 or 8), vectorised
+template <int VEC>
+__device__ __forceinline__ void store_floats(float *p, const float (&v)[VEC]) {
+  if constexpr (VEC == 1) { *p = v[0]; }
+  else if constexpr (VEC == 2) { *reinterpret_cast<float2 *>(p) = make_float2(v[0], v[1]); }
+  else {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 4) *reinterpret_cast<float4 *>(p + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+  }
+}
+template <int VEC>
+__device__ __forceinline__ void load_floats_stream(const float *p, float (&v)[VEC]) {
+  if constexpr (VEC == 1) { v[0] = __ldcs(p); }
+  else if constexpr (VEC == 2) { const float2 x = __ldcs(reinterpret_cast<const float2 *>(p)); v[0] = x.x; v[1] = x.y; }
+  else {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 4) {
+      const float4 x = __ldcs(reinterpret_cast<const float4 *>(p + i));
+      v[i] = x.x; v[i + 1] = x.y; v[i + 2] = x.z; v[i + 3] = x.w;
+    }
+  }
+}
 
 __device__ __forceinline__ float act_apply(float x, int act) {
   if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
@@ -103,10 +152,13 @@ __device__ __forceinline__ it_row_meta load_meta(const it_row_meta *p) {
 
 // ----------------------------------------------------------------------------- batches of rows per lane group
 // Rows handled here have at least one edge: empty rows live in their own bucket.
-template <typename T, int LPR, class Policy>
+template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_kernel(StreamParams p, Policy pol) {
   constexpr int G = LPR;
-  constexpr int U = UNROLL < G ? UNROLL : G;
+  // more rows in flight for narrower slices, as far as the register budget and the size of the unrolled
+  // consume loop (which carries a copy of the end-of-row code per edge) allow
+  constexpr int UW = Policy::HAS_EXTRA ? UNROLL : (UNROLL * (16 / SB) < 2 * UNROLL ? UNROLL * (16 / SB) : 2 * UNROLL);
+  constexpr int U = UW < G ? UW : G;
   constexpr int NS = Policy::NS;
   const int lane = threadIdx.x & 31;
   const int t = lane % G;
@@ -117,7 +169,8 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
   const int BR = p.batch_rows;  // rows per batch, <= G: lanes t < BR hold their metadata
   const int64_t n_batches = (n_rows + BR - 1) / BR;
   const int64_t groups_total = (int64_t)gridDim.x * (THREADS / G);
-  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * 16;
+  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * SB;
+  using Slice = RowSlice<T, SB>;
   const uint32_t row_bytes = (uint32_t)p.dim * (uint32_t)sizeof(T);
 
   for (int64_t b = (int64_t)blockIdx.x * (THREADS / G) + threadIdx.x / G; b < n_batches; b += groups_total) {
@@ -183,13 +236,13 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
       const int cnt = (total - base) < G ? (total - base) : G;
       int k0 = 0;
       for (; k0 + U <= cnt; k0 += U) {  // full groups of U edges: no predicates
-        uint4 v[U];
+        typename Slice::Raw v[U];
         float w[U], x[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           const uint32_t s = (uint32_t)__shfl_sync(gmask, idx_c, k0 + u, G);
           w[u] = Policy::WEIGHTED ? __shfl_sync(gmask, w_c, k0 + u, G) : 1.f;
-          v[u] = __ldg(reinterpret_cast<const uint4 *>(my_src + (uint64_t)s * row_bytes));
+          v[u] = Slice::load(my_src + (uint64_t)s * row_bytes);
           x[u] = Policy::HAS_EXTRA ? pol.extra(s) : 0.f;
         }
 #pragma unroll
@@ -199,7 +252,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
         }
       }
       if (k0 < cnt) {  // tail of the chunk
-        uint4 v[U];
+        typename Slice::Raw v[U];
         float w[U], x[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -208,7 +261,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
           w[u] = Policy::WEIGHTED ? __shfl_sync(gmask, w_c, e & (G - 1), G) : 1.f;
           x[u] = 0.f;
           if (e < cnt) {
-            v[u] = __ldg(reinterpret_cast<const uint4 *>(my_src + (uint64_t)s * row_bytes));
+            v[u] = Slice::load(my_src + (uint64_t)s * row_bytes);
             if (Policy::HAS_EXTRA) x[u] = pol.extra(s);
           }
         }
@@ -226,17 +279,18 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
 }
 
 // ----------------------------------------------------------------------------- very long rows: one CTA each
-template <typename T, int LPR, class Policy>
+template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kernel(StreamParams p, Policy pol) {
   constexpr int NS = Policy::NS;
   constexpr int WARPS = THREADS / 32;
   constexpr int SLOTS = 32 / LPR;
-  constexpr int U = UNROLL;
+  constexpr int U = UNROLL * (16 / SB);   // the same bytes in flight per lane whatever the slice width
   __shared__ float red[WARPS][LPR][NS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int slot = lane / LPR, t = lane % LPR;
   pol.setup(t);
-  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * 16;
+  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * SB;
+  using Slice = RowSlice<T, SB>;
   const uint32_t row_bytes = (uint32_t)p.dim * (uint32_t)sizeof(T);
   for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {
     const it_row_meta m = load_meta(p.meta + i);
@@ -264,7 +318,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
       load_chunk(base + 32, idx_n, w_n);
       const int cnt = (int)((b - base) < 32 ? (b - base) : 32);
       for (int k0 = 0; k0 < cnt; k0 += SLOTS * U) {
-        uint4 v[U];
+        typename Slice::Raw v[U];
         float w[U], x[U];
         bool ok[U];
 #pragma unroll
@@ -275,7 +329,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
           ok[u] = e < cnt;
           x[u] = 0.f;
           if (ok[u]) {
-            v[u] = __ldg(reinterpret_cast<const uint4 *>(my_src + (uint64_t)s * row_bytes));
+            v[u] = Slice::load(my_src + (uint64_t)s * row_bytes);
             if (Policy::HAS_EXTRA) x[u] = pol.extra(s);
           }
         }
@@ -312,7 +366,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
 }
 
 // ----------------------------------------------------------------------------- empty rows
-template <typename T, int LPR, class Policy>
+template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, Policy pol) {
   constexpr int NS = Policy::NS;
   const int t = threadIdx.x % LPR;
@@ -331,7 +385,7 @@ __global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, P
 // ----------------------------------------------------------------------------- bucket dispatch
 // Longest rows first so that the tail of the launch sequence is made of short rows.
 // bytes_of(bucket, rows) gives the algorithmic bytes of a launch; kid_* the instrumentation ids.
-template <typename T, int LPR, class Policy, class BytesF>
+template <typename T, int SB, int LPR, class Policy, class BytesF>
 it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, BytesF bytes_of, int kid_cta, int kid_rows,
                          int kid_empty, cudaStream_t st) {
   for (int b = g->n_buckets - 1; b >= 0; --b) {
@@ -345,10 +399,10 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
     if (bound == 0) {
       int64_t want = (rows + (THREADS / LPR) - 1) / (THREADS / LPR);
       unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
-      IT_LAUNCH(kid_empty, bytes, 0, st, stream_empty_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+      IT_LAUNCH(kid_empty, bytes, 0, st, stream_empty_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
     } else if (bound > IT_GATHER_CTA_ABOVE) {
       unsigned blocks = (unsigned)(rows < max_blocks ? rows : max_blocks);
-      IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+      IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
     } else {
       // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
       int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
@@ -357,11 +411,26 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
       const int64_t batches = (rows + br - 1) / br;
       int64_t want = (batches + (THREADS / LPR) - 1) / (THREADS / LPR);
       unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
-      IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+      IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
     }
   }
   IT_CUDA_TRY(cudaGetLastError());
   return IT_OK;
+}
+
+// Pick the slice width and group size for a row of `row_bytes` bytes and call f.template operator()<SB, LPR>().
+template <class F>
+it_status dispatch_row_bytes(int row_bytes, F f) {
+  switch (row_bytes) {
+    case 512: return f.template operator()<16, 32>();
+    case 256: return f.template operator()<8, 32>();
+    case 128: return f.template operator()<4, 32>();
+    case 64: return f.template operator()<4, 16>();
+    case 32: return f.template operator()<4, 8>();
+    case 16: return f.template operator()<4, 4>();
+  }
+  it_set_error("feature row of %d bytes is not 16, 32, 64, 128, 256 or 512 bytes", row_bytes);
+  return IT_ERR_UNSUPPORTED;
 }
 
 }  // namespace it_stream

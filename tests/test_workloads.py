@@ -37,7 +37,7 @@ def test_scaled_configs_have_the_right_models():
     assert m.x.shape == (m.n, 128) and m.layers[0].use_edge_weights and m.layers[1].out_dim == 64
     g = make("gat", 0.002)
     assert g.dtype == "bf16" and g.x.dtype == np.uint16 and g.layers[0].heads == 4 and g.layers[0].act == "elu"
-    assert g.layers[0].att_src.shape == (4, 32) and g.threshold == 0
+    assert g.layers[0].att_src.shape == (4, 32) and g.threshold == 4096
     # bf16 parameters are exactly representable
     W = g.layers[0].W
     assert np.array_equal(wrng.bf16_bits_to_f32(wrng.f32_to_bf16_bits(W)), W)

@@ -115,7 +115,7 @@ def make(name: str, scale: float = 1.0) -> Workload:
         n, e = s(5_000_000), s(100_000_000)
         indptr, indices = graphs.power_law_graph(g, n, e, 2.0, s(200_000))
         return Workload(name, n, e, indptr, indices, None, "bf16", _features(n, 128, "bf16"),
-                        gat_layers([128, 128, 128], 4, ["elu", "none"], "bf16"), 0)
+                        gat_layers([128, 128, 128], 4, ["elu", "none"], "bf16"), 4096)
     if name == "extreme":
         n, e = s(20_000_000), s(200_000_000)
         n_hubs = 100 if scale >= 0.01 else 4
