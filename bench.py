@@ -299,10 +299,14 @@ def run_ours(args):
                       for s in stats), key=lambda r: -r["share"])
     top = max(stats, key=lambda s: s["total_ms"])
     achieved = (top["algo_bytes"] / 1e9) / (top["total_ms"] * 1e-3)
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    # DRAM bytes per launch of that kernel from the committed ncu capture (lines "traffic <workload>:<kernel> <bytes>")
     traffic = None
-    if os.path.exists(traffic_path):
-        traffic = json.load(open(traffic_path)).get(f"{w.name}:{top['name']}")
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.md")
+    if os.path.exists(traffic_path) and args.scale == 1.0:
+        for line in open(traffic_path):
+            parts = line.split()
+            if len(parts) == 3 and parts[0] == "traffic" and parts[1] == f"{w.name}:{top['name']}":
+                traffic = float(parts[2])
     roofline = {"bound": "hbm", "kernel": top["name"], "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                 "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": traffic,
                 "algo_bytes_per_launch": top["algo_bytes"] / max(1, top["launches"]),
