@@ -332,3 +332,25 @@ def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, th
         H = np.full((n, layer.out_dim), np.nan)
         H[need[l]] = out_rows
     return H[targets]
+
+
+def compact_neighbourhood(indptr, indices, edge_weights, targets, n_layers):
+    """The part of the graph an n_layers-layer model reads to produce `targets`, relabelled to
+    consecutive ids so that huge graphs can be checked without full-size fp64 arrays.
+    Returns (vertex_ids, c_indptr, c_indices, c_weights, c_targets): vertex_ids are the global
+    ids (sorted) of the compact vertices; a compact vertex keeps its in-edges only if some layer
+    output of it is needed (the others are read as layer-0 inputs only)."""
+    targets = _i64(targets)
+    need = np.unique(targets)
+    for _ in range(n_layers - 1):
+        need = _sources_of(indptr, indices, need)          # where layer 1 .. L-1 outputs are needed
+    ids = _sources_of(indptr, indices, need)               # plus the layer-0 inputs they read
+    sub, idx, w = _sub_csr(indptr, indices, edge_weights, need)
+    deg = np.zeros(ids.shape[0], np.int64)
+    pos_need = np.searchsorted(ids, need)
+    deg[pos_need] = np.diff(sub)
+    c_indptr = np.zeros(ids.shape[0] + 1, np.int64)
+    np.cumsum(deg, out=c_indptr[1:])
+    # rows of `need` are ascending in both numberings, so the concatenated edge lists keep their order
+    c_indices = np.searchsorted(ids, idx.astype(np.int64)).astype(np.int32)
+    return ids, c_indptr, c_indices, w, np.searchsorted(ids, targets)

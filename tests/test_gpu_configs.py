@@ -5,14 +5,18 @@ oracle, and (b) where they fit the test budget, at full size in the launch confi
 benchmark times, checked on sampled vertices that the oracle evaluates from their L-hop
 in-neighbourhood.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
 
 from gpu_util import TOL, check_against_oracle, run_device, to_numpy
 from oracle import oracle as O
+from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
 from workloads import compare, make
+from workloads import rng as wrng
 
 pytestmark = pytest.mark.gpu
 
@@ -79,3 +83,21 @@ def test_extreme_hub_rows_at_scale():
     d.infer()
     torch.cuda.synchronize()
     check_sampled(w, d, sampled_targets(w, 3, 200), "extreme")
+
+
+@pytest.mark.skipif(not os.environ.get("IT_RUN_LARGE"), reason="set IT_RUN_LARGE=1: needs ~100 GB of HBM, ~60 GB of host RAM and ~10 minutes")
+def test_large_full_size_sampled():
+    """100M vertices, 1.5B edges, int32 CSR, bf16: sampled vertices against the oracle evaluated on
+    their 2-hop in-neighbourhood (relabelled to a compact graph)."""
+    w = make("large")
+    d = host.upload(w, int32_indptr=True)
+    d.infer()
+    B.it_graph_check(d.graph)
+    targets = sampled_targets(w, 2, 150)
+    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, None, targets, len(w.layers))
+    xc = wrng.bf16_bits_to_f32(w.x[ids])
+    ref = O.infer_at(cip, cix, cw, xc, w.layers, ct, storage=w.dtype, threshold=w.threshold, follow_reorder=True)
+    got = to_numpy(d.out[torch.from_numpy(targets).cuda()])
+    err = compare.rel_error(got, ref)
+    print("large full size:", err, "rows", d.n_rows, "split owners", d.n_split_owners)
+    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], err

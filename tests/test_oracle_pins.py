@@ -501,3 +501,19 @@ def test_infer_at_targets_equals_full_graph_inference(op):
             full = O.infer(ip, ix, w, X, layers, storage=storage, threshold=thr, follow_reorder=True)[-1]
             part = O.infer_at(ip, ix, w, X, layers, targets, storage=storage, threshold=thr, follow_reorder=True)
             assert np.array_equal(part, full[targets])
+
+
+def test_compact_neighbourhood_gives_the_same_values():
+    rng = np.random.default_rng(23)
+    n = 500
+    ip, ix = random_graph(rng, n, 5)
+    w = rng.random(ix.shape[0])
+    X = rng.standard_normal((n, 6))
+    layers = [L("sum", "relu", rng.standard_normal((12, 6)) * .3, rng.standard_normal(6) * .1, use_edge_weights=True),
+              L("mean", "none", rng.standard_normal((12, 4)) * .3, rng.standard_normal(4) * .1)]
+    targets = rng.permutation(n)[:20]
+    full = O.infer(ip, ix, w, X, layers, threshold=3)[-1]
+    ids, cip, cix, cw, ct = O.compact_neighbourhood(ip, ix, w, targets, len(layers))
+    assert ids.shape[0] < n and np.all(np.diff(ids) > 0)
+    part = O.infer_at(cip, cix, cw, X[ids], layers, ct, threshold=3)
+    assert np.array_equal(part, full[targets])
