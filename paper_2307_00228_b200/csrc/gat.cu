@@ -37,6 +37,7 @@ struct GatPolicy {
     st[VEC + 1] = 0.f;
   }
   __device__ __forceinline__ float extra(uint32_t s) const { return __ldg(scores + (uint64_t)s * (2 * heads) + head); }
+  __device__ __forceinline__ const float *extra_ptr(uint32_t s) const { return scores + (uint64_t)s * (2 * heads) + head; }
   __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float, float x) const {
     float e = x + s_dst;
     e = e > 0.f ? e : slope * e;

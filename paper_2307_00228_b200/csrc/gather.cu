@@ -29,6 +29,7 @@ struct SagePolicy {
     for (int k = 0; k < NS; ++k) st[k] = IS_MAX ? -INFINITY : 0.f;
   }
   __device__ __forceinline__ float extra(uint32_t) const { return 0.f; }
+  __device__ __forceinline__ const float *extra_ptr(uint32_t) const { return nullptr; }
   __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float w, float) const {
     float f[VEC];
     Slice::unpack(raw, f);
