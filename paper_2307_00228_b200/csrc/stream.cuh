@@ -582,6 +582,125 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
   }
 }
 
+// The same for rows that span all 32 lanes, each warp streaming its part of the row through its
+// shared-memory ring (see stream_rows_ring_kernel): no ends of rows inside a part, so every full stage
+// takes the unrolled path.
+template <typename T, int SB, class Policy>
+__global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_cta_ring_kernel(StreamParams p, Policy pol) {
+  constexpr int NS = Policy::NS;
+  constexpr int WARPS = THREADS / 32;
+  constexpr int R = ring_stage_rows<SB>();
+  constexpr int S = IT_RING_STAGES;
+  constexpr int AHEAD = (S - 1) * R;
+  constexpr int ROWB = 32 * SB;
+  static_assert(32 % R == 0 && AHEAD <= 32, "a chunk is a whole number of stages and the fill reaches at most into the next chunk");
+  extern __shared__ uint4 ring_raw[];
+  __shared__ float red[WARPS][32][NS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_raw) + (uint32_t)warp * (uint32_t)ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
+  const uint32_t my_ring = ring + lane * SB;
+  const uint32_t my_xring = ring + S * R * ROWB + lane * 4;
+  pol.setup(lane);
+  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)lane * SB;
+
+  auto fill = [&](int stage, int32_t idxreg, int k0, int n) {
+    const uint32_t d = my_ring + stage * (R * ROWB);
+    const uint32_t dx = my_xring + stage * (R * 128);
+    if (n == R) {
+#pragma unroll
+      for (int u = 0; u < R; ++u) {
+        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u);
+        cp_async_slice<SB>(d + u * ROWB, my_src + (uint64_t)s * ROWB);
+        if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
+      }
+    } else {
+      for (int u = 0; u < n; ++u) {
+        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u);
+        cp_async_slice<SB>(d + u * ROWB, my_src + (uint64_t)s * ROWB);
+        if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
+      }
+    }
+  };
+
+  for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {
+    const it_row_meta m = load_meta(p.meta + i);
+    const int32_t owner = Policy::NEEDS_OWNER ? __ldcs(p.owner + i) : 0;
+    // this warp's part of the row: edges [a, a + total)
+    const int part = (m.len + WARPS - 1) / WARPS;
+    const int first = warp * part < m.len ? warp * part : m.len;
+    const int total = (m.len - first) < part ? (m.len - first) : part;
+    const int64_t a = m.j0 + first;
+    float st[NS];
+    pol.init(st);
+    pol.begin_row(m.dest, owner);
+    auto load_chunk = [&](int base, int32_t &idx, float &w) {
+      idx = 0; w = 1.f;
+      if (base + lane < total) {
+        idx = __ldcs(p.indices + a + base + lane);
+        if (Policy::WEIGHTED) w = __ldcs(p.weights + a + base + lane);
+      }
+    };
+    int32_t idx_c, idx_n;
+    float w_c, w_n;
+    load_chunk(0, idx_c, w_c);
+    int fs = 0, cs = 0;
+#pragma unroll
+    for (int k = 0; k < AHEAD; k += R) {
+      if (k < total) fill(fs, idx_c, k, (total - k) < R ? (total - k) : R);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      fs = fs + 1 == S ? 0 : fs + 1;
+    }
+    for (int base = 0; base < total; base += 32) {
+      load_chunk(base + 32, idx_n, w_n);
+      const int cnt = (total - base) < 32 ? (total - base) : 32;
+      for (int k0 = 0; k0 < cnt; k0 += R) {
+        const int f = k0 + AHEAD;
+        if (f < 32) {
+          const int left = cnt - f;
+          if (left > 0) fill(fs, idx_c, f, left < R ? left : R);
+        } else {
+          const int left = total - (base + f);
+          if (left > 0) fill(fs, idx_n, f - 32, left < R ? left : R);
+        }
+        fs = fs + 1 == S ? 0 : fs + 1;
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");
+        const int n = (cnt - k0) < R ? (cnt - k0) : R;
+        const uint32_t sr = my_ring + cs * (R * ROWB);
+        const uint32_t sx = my_xring + cs * (R * 128);
+        cs = cs + 1 == S ? 0 : cs + 1;
+        auto consume = [&](int u) {
+          const typename RowSlice<T, SB>::Raw raw = lds_slice<SB>(sr + u * ROWB);
+          const float w = Policy::WEIGHTED ? __shfl_sync(0xffffffffu, w_c, k0 + u) : 1.f;
+          const float x = Policy::HAS_EXTRA ? lds_f32(sx + u * 128) : 0.f;
+          pol.edge(st, raw, w, x);
+        };
+        if (n == R) {
+#pragma unroll
+          for (int u = 0; u < R; ++u) consume(u);
+        } else {
+          for (int u = 0; u < n; ++u) consume(u);
+        }
+      }
+      idx_c = idx_n; w_c = w_n;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // red[] free again
+#pragma unroll
+    for (int k = 0; k < NS; ++k) red[warp][lane][k] = st[k];
+    __syncthreads();
+    if (warp == 0) {
+      for (int w = 1; w < WARPS; ++w) {
+        float other[NS];
+#pragma unroll
+        for (int k = 0; k < NS; ++k) other[k] = red[w][lane][k];
+        pol.merge(st, other);
+      }
+      pol.end_row(st, m.dest, owner, m.len);
+    }
+  }
+}
+
 // ----------------------------------------------------------------------------- empty rows
 template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, Policy pol) {
@@ -618,8 +737,20 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
       unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
       IT_LAUNCH(kid_empty, bytes, 0, st, stream_empty_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
     } else if (bound > IT_GATHER_CTA_ABOVE) {
-      unsigned blocks = (unsigned)(rows < max_blocks ? rows : max_blocks);
-      IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+      if constexpr (LPR == 32 && SB >= IT_RING_MIN_SB) {
+        constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
+        static bool configured = false;   // per template instance
+        if (!configured) {
+          IT_CUDA_TRY(cudaFuncSetAttribute(stream_cta_ring_kernel<T, SB, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+          configured = true;
+        }
+        // one CTA per row as far as the grid allows: the hardware hands out rows as CTAs retire
+        unsigned blocks = (unsigned)(rows < (1 << 20) ? rows : (1 << 20));
+        IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_ring_kernel<T, SB, Policy><<<blocks, THREADS, smem, st>>>(p, pol));
+      } else {
+        unsigned blocks = (unsigned)(rows < max_blocks ? rows : max_blocks);
+        IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+      }
     } else {
       // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
       int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
