@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(THREADS) gat_combine_kernel(GatCombineParams p
 }
 
 template <typename T, int SB, int LPR>
-it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, cudaStream_t st) {
+it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   GatPolicy<T, SB> pol;
   pol.scores = a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
   pol.dim = a.heads * a.head_dim; pol.heads = a.heads; pol.head_dim = a.head_dim; pol.act = a.act; pol.slope = a.slope;
@@ -147,17 +147,19 @@ it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, cudaStream_t st)
   auto bytes_of = [=](int b, int64_t rows) {
     return (double)g->h_bucket_edges[b] * (4.0 + 4.0 * heads + row_bytes) + (double)rows * (20.0 + 4.0 * heads + row_bytes);
   };
-  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, st);
+  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, bound_lo, bound_hi, st);
 }
 
 template <typename T>
 it_status launch_gat(const it_gat_args &a, StreamParams sp, cudaStream_t st) {
-  return dispatch_row_bytes(a.heads * a.head_dim * (int)sizeof(T), [&]<int SB, int LPR>() {
+  // 16-byte slices as long as one never straddles two heads
+  const bool wide = (a.head_dim * (int)sizeof(T)) % 16 == 0;
+  return dispatch_row_bytes(a.heads * a.head_dim * (int)sizeof(T), wide, [&]<int SB, int LPR>(int64_t lo, int64_t hi) {
     if ((a.head_dim * (int)sizeof(T)) % SB != 0) {
       it_set_error("gat: a %d-byte lane slice would straddle two heads (head_dim %d)", SB, a.head_dim);
       return IT_ERR_UNSUPPORTED;
     }
-    return launch_gat_lpr<T, SB, LPR>(a, sp, st);
+    return launch_gat_lpr<T, SB, LPR>(a, sp, lo, hi, st);
   });
 }
 

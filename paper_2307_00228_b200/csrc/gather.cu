@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 
 // ----------------------------------------------------------------------------- dispatch
 template <typename T, int SB, int LPR, bool IS_MAX, bool WEIGHTED>
-it_status launch_policy(const it_gather_args &a, StreamParams sp, cudaStream_t st) {
+it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   SagePolicy<T, SB, IS_MAX, WEIGHTED> pol;
   pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.dim = a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
@@ -136,15 +136,15 @@ it_status launch_policy(const it_gather_args &a, StreamParams sp, cudaStream_t s
     return (double)g->h_bucket_edges[b] * (4.0 + (WEIGHTED ? 4.0 : 0.0) + row_bytes) +
            (double)rows * (16.0 + row_bytes + (a.epi == IT_EPI_ADD_ACT ? 4.0 * a.dim : 0.0));
   };
-  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, st);
+  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, bound_lo, bound_hi, st);
 }
 
 template <typename T>
 it_status launch_lpr(const it_gather_args &a, StreamParams sp, cudaStream_t st) {
   const bool mx = a.op == IT_GATHER_MAX, w = a.use_edge_weights != 0;
-  return dispatch_row_bytes(a.dim * (int)sizeof(T), [&]<int SB, int LPR>() {
-    if (mx) return w ? launch_policy<T, SB, LPR, true, true>(a, sp, st) : launch_policy<T, SB, LPR, true, false>(a, sp, st);
-    return w ? launch_policy<T, SB, LPR, false, true>(a, sp, st) : launch_policy<T, SB, LPR, false, false>(a, sp, st);
+  return dispatch_row_bytes(a.dim * (int)sizeof(T), true, [&]<int SB, int LPR>(int64_t lo, int64_t hi) {
+    if (mx) return w ? launch_policy<T, SB, LPR, true, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, true, false>(a, sp, lo, hi, st);
+    return w ? launch_policy<T, SB, LPR, false, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, false, false>(a, sp, lo, hi, st);
   });
 }
 

@@ -336,11 +336,11 @@ static it_status split_impl(it_graph *g, int64_t T, cudaStream_t st) {
     SPLIT_CUDA(cudaGetLastError());
   }
 
-  // degree buckets: {0, 8, 32, 256, everything longer}
+  // degree buckets: {0, 8, 32, 256, 1024, everything longer}
   Bounds B;
-  const int64_t fixed[4] = {0, 8, 32, 256};
+  const int64_t fixed[5] = {0, 8, 32, 256, 1024};
   B.nb = 0;
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 5; ++i)
     if (T <= 0 || fixed[i] < T) B.b[B.nb++] = fixed[i];
   B.b[B.nb++] = T > 0 ? T : INT64_MAX;
   g->n_buckets = B.nb;

@@ -38,16 +38,13 @@
 #define IT_RING_MIN_BLOCKS 4   // resident CTAs per SM of the shared-memory-ring kernel
 #endif
 #ifndef IT_RING_STAGE_ROWS
-#define IT_RING_STAGE_ROWS 4   // 512-byte rows per stage of the ring
+#define IT_RING_STAGE_ROWS 4   // 512-byte groups of rows per stage of the ring
 #endif
 #ifndef IT_RING_STAGES
 #define IT_RING_STAGES 2
 #endif
-#ifndef IT_RING_MIN_SB
-#define IT_RING_MIN_SB 4       // narrowest lane slice (bytes) that goes through the shared-memory ring
-#endif
 #ifndef IT_GATHER_CTA_ABOVE
-#define IT_GATHER_CTA_ABOVE 2048   // rows longer than this get a whole CTA; shorter ones a lane group
+#define IT_GATHER_CTA_ABOVE 1024   // rows longer than this get a whole CTA; shorter ones a lane group or a warp
 #endif
 
 namespace it_stream {
@@ -290,211 +287,6 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
   }
 }
 
-// ----------------------------------------------------------------------------- batches of rows per warp, rows staged in shared memory
-// The same walk as stream_rows_kernel for rows that span all 32 lanes, but the source rows are copied
-// asynchronously (cp.async) into a per-warp ring in shared memory instead of into registers: up to RING_ROWS
-// rows (8 KB) are in flight per warp whatever the slice width, the consume loop is a plain rolled loop
-// with one copy of the end-of-row code, and the register budget allows more resident warps.
-// Each lane copies and later reads only its own slice of every row, so no warp synchronisation is needed
-// between the copy and the read; cp.async.wait_group orders them.
-template <int SB>
-__device__ __forceinline__ void cp_async_slice(uint32_t smem_dst, const void *gmem_src) {   // smem_dst: shared-window address
-  if constexpr (SB == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-  else if constexpr (SB == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-}
-template <int SB>
-__device__ __forceinline__ typename SliceRaw<SB>::type lds_slice(uint32_t a) {
-  if constexpr (SB == 16) {
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
-    return v;
-  } else if constexpr (SB == 8) {
-    uint2 v;
-    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a) : "memory");
-    return v;
-  } else {
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-  }
-}
-__device__ __forceinline__ float lds_f32(uint32_t a) {
-  float v;
-  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
-  return v;
-}
-
-// The ring of a warp holds IT_RING_STAGES stages of ring_stage_rows() rows each: while one stage is consumed
-// the copies of the others are in flight.
-template <int SB> constexpr int ring_stage_rows() { return IT_RING_STAGE_ROWS * (16 / SB) < 16 ? IT_RING_STAGE_ROWS * (16 / SB) : 16; }
-template <int SB, bool HAS_EXTRA> constexpr int ring_bytes_per_warp() {
-  return IT_RING_STAGES * ring_stage_rows<SB>() * (32 * SB + (HAS_EXTRA ? 128 : 0));
-}
-
-template <typename T, int SB, class Policy>
-__global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_kernel(StreamParams p, Policy pol) {
-  constexpr int G = 32;
-  constexpr int NS = Policy::NS;
-  constexpr int R = ring_stage_rows<SB>();   // edges per stage
-  constexpr int S = IT_RING_STAGES;
-  constexpr int AHEAD = (S - 1) * R;         // the stage being filled is this many edges ahead of the one consumed
-  constexpr int ROWB = 32 * SB;
-  static_assert(32 % R == 0 && AHEAD <= 32, "a chunk is a whole number of stages and the fill reaches at most into the next chunk");
-  using Slice = RowSlice<T, SB>;
-  extern __shared__ uint4 ring_raw[];
-  const int lane = threadIdx.x & 31;
-  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_raw) +
-                        (uint32_t)(threadIdx.x >> 5) * (uint32_t)ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
-  const uint32_t my_ring = ring + lane * SB;                  // my slice of ring row 0
-  const uint32_t my_xring = ring + S * R * ROWB + lane * 4;   // my per-edge scalar of ring row 0 (HAS_EXTRA)
-  pol.setup(lane);
-  const int64_t n_rows = p.row_hi - p.row_lo;
-  const int BR = p.batch_rows;  // rows per batch, <= 32: lanes t < BR hold their metadata
-  const int64_t n_batches = (n_rows + BR - 1) / BR;
-  const int64_t warps_total = (int64_t)gridDim.x * (THREADS / 32);
-  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)lane * SB;
-  const uint32_t row_bytes = (uint32_t)ROWB;
-
-  // copy the rows of edges [k0, k0 + n) of the chunk whose indices sit in idxreg into a stage
-  auto fill = [&](int stage, int32_t idxreg, int k0, int n) {
-    const uint32_t d = my_ring + stage * (R * ROWB);
-    const uint32_t dx = my_xring + stage * (R * 128);
-    if (n == R) {
-#pragma unroll
-      for (int u = 0; u < R; ++u) {
-        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u);
-        cp_async_slice<SB>(d + u * ROWB, my_src + (uint64_t)s * row_bytes);
-        if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
-      }
-    } else {
-      for (int u = 0; u < n; ++u) {
-        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u);
-        cp_async_slice<SB>(d + u * ROWB, my_src + (uint64_t)s * row_bytes);
-        if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
-      }
-    }
-  };
-
-  for (int64_t b = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); b < n_batches; b += warps_total) {
-    // ---- batch metadata: lane t owns row t of the batch
-    const int64_t i = p.row_lo + b * BR + lane;
-    int64_t my_j0 = 0;
-    int my_len = 0, my_dest = 0, my_owner = 0;
-    if (lane < BR && i < p.row_hi) {
-      const it_row_meta m = load_meta(p.meta + i);
-      my_j0 = m.j0; my_len = m.len; my_dest = m.dest;
-      if (Policy::NEEDS_OWNER) my_owner = __ldcs(p.owner + i);
-    }
-    int my_end = my_len;  // inclusive prefix sum of the row lengths
-#pragma unroll
-    for (int o = 1; o < G; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, my_end, o);
-      if (lane >= o) my_end += y;
-    }
-    const int total = __shfl_sync(0xffffffffu, my_end, G - 1);
-    const int my_start = my_end - my_len;
-    const int64_t j_first = __shfl_sync(0xffffffffu, my_j0, 0);
-
-    auto load_chunk = [&](int base, int32_t &idx, float &w, unsigned &ends) {
-      const int q = base + lane;
-      int row_end = total;
-      int64_t j = j_first + q;
-      if (BR > 1) {   // which row of the batch edge q belongs to
-        int lo = 0;
-#pragma unroll
-        for (int step = G / 2; step >= 1; step >>= 1) {
-          const int e = __shfl_sync(0xffffffffu, my_end, lo + step - 1);
-          if (e <= q) lo += step;
-        }
-        row_end = __shfl_sync(0xffffffffu, my_end, lo);
-        j = __shfl_sync(0xffffffffu, my_j0, lo) + (q - __shfl_sync(0xffffffffu, my_start, lo));
-      }
-      idx = 0;
-      w = 1.f;
-      if (q < total) {
-        idx = __ldcs(p.indices + j);
-        if (Policy::WEIGHTED) w = __ldcs(p.weights + j);
-      }
-      ends = __ballot_sync(0xffffffffu, q < total && q + 1 == row_end);
-    };
-
-    float st[NS];
-    pol.init(st);
-    int cur = 0;  // row of the batch that st belongs to
-    pol.begin_row(__shfl_sync(0xffffffffu, my_dest, 0), __shfl_sync(0xffffffffu, my_owner, 0));
-    auto next_row = [&]() {
-      pol.end_row(st, __shfl_sync(0xffffffffu, my_dest, cur), Policy::NEEDS_OWNER ? __shfl_sync(0xffffffffu, my_owner, cur) : 0,
-                  __shfl_sync(0xffffffffu, my_len, cur));
-      ++cur;
-      pol.init(st);
-      const int32_t nd = __shfl_sync(0xffffffffu, my_dest, cur & 31);
-      const int32_t no = Policy::NEEDS_OWNER ? __shfl_sync(0xffffffffu, my_owner, cur & 31) : 0;
-      if (cur < BR && __shfl_sync(0xffffffffu, my_len, cur & 31) > 0) pol.begin_row(nd, no);
-    };
-
-    int32_t idx_c, idx_n;
-    float w_c, w_n;
-    unsigned ends_c, ends_n;
-    load_chunk(0, idx_c, w_c, ends_c);
-    int fs = 0, cs = 0;   // stage to fill next, stage to consume next
-#pragma unroll
-    for (int k = 0; k < AHEAD; k += R) {   // total >= 1: empty rows live in their own bucket
-      if (k < total) fill(fs, idx_c, k, (total - k) < R ? (total - k) : R);
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      fs = fs + 1 == S ? 0 : fs + 1;
-    }
-    for (int base = 0; base < total; base += G) {
-      load_chunk(base + G, idx_n, w_n, ends_n);  // in flight while this chunk is consumed
-      const int cnt = (total - base) < G ? (total - base) : G;
-      for (int k0 = 0; k0 < cnt; k0 += R) {
-        // the stage AHEAD edges further on: in this chunk, or at the head of the next one
-        const int f = k0 + AHEAD;
-        if (f < G) {
-          const int left = cnt - f;
-          if (left > 0) fill(fs, idx_c, f, left < R ? left : R);
-        } else {
-          const int left = total - (base + f);
-          if (left > 0) fill(fs, idx_n, f - G, left < R ? left : R);
-        }
-        fs = fs + 1 == S ? 0 : fs + 1;
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");   // the oldest stage has landed
-        const int n = (cnt - k0) < R ? (cnt - k0) : R;
-        const uint32_t sr = my_ring + cs * (R * ROWB);
-        const uint32_t sx = my_xring + cs * (R * 128);
-        cs = cs + 1 == S ? 0 : cs + 1;
-        auto consume = [&](int u) {
-          const typename Slice::Raw raw = lds_slice<SB>(sr + u * ROWB);
-          const float w = Policy::WEIGHTED ? __shfl_sync(0xffffffffu, w_c, k0 + u) : 1.f;
-          const float x = Policy::HAS_EXTRA ? lds_f32(sx + u * 128) : 0.f;
-          pol.edge(st, raw, w, x);
-        };
-        unsigned e = (ends_c >> k0) & ((1u << R) - 1u);   // rows that end inside this stage
-        if (n == R && e == 0) {
-#pragma unroll
-          for (int u = 0; u < R; ++u) consume(u);
-        } else {   // segment by segment: the edges up to the next end of a row, then the row's epilogue
-          int u = 0;
-          while (u < n) {
-            const int last = e ? __ffs(e) - 1 : n - 1;
-            for (; u + 4 <= last + 1; u += 4) {
-              consume(u); consume(u + 1); consume(u + 2); consume(u + 3);
-            }
-            for (; u <= last; ++u) consume(u);
-            if (e) {
-              next_row();
-              e &= e - 1;
-            }
-          }
-        }
-      }
-      idx_c = idx_n; w_c = w_n; ends_c = ends_n;
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");   // only empty groups are left
-  }
-}
-
 // ----------------------------------------------------------------------------- very long rows: one CTA each
 template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kernel(StreamParams p, Policy pol) {
@@ -582,125 +374,6 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
   }
 }
 
-// The same for rows that span all 32 lanes, each warp streaming its part of the row through its
-// shared-memory ring (see stream_rows_ring_kernel): no ends of rows inside a part, so every full stage
-// takes the unrolled path.
-template <typename T, int SB, class Policy>
-__global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_cta_ring_kernel(StreamParams p, Policy pol) {
-  constexpr int NS = Policy::NS;
-  constexpr int WARPS = THREADS / 32;
-  constexpr int R = ring_stage_rows<SB>();
-  constexpr int S = IT_RING_STAGES;
-  constexpr int AHEAD = (S - 1) * R;
-  constexpr int ROWB = 32 * SB;
-  static_assert(32 % R == 0 && AHEAD <= 32, "a chunk is a whole number of stages and the fill reaches at most into the next chunk");
-  extern __shared__ uint4 ring_raw[];
-  __shared__ float red[WARPS][32][NS];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_raw) + (uint32_t)warp * (uint32_t)ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
-  const uint32_t my_ring = ring + lane * SB;
-  const uint32_t my_xring = ring + S * R * ROWB + lane * 4;
-  pol.setup(lane);
-  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)lane * SB;
-
-  auto fill = [&](int stage, int32_t idxreg, int k0, int n) {
-    const uint32_t d = my_ring + stage * (R * ROWB);
-    const uint32_t dx = my_xring + stage * (R * 128);
-    if (n == R) {
-#pragma unroll
-      for (int u = 0; u < R; ++u) {
-        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u);
-        cp_async_slice<SB>(d + u * ROWB, my_src + (uint64_t)s * ROWB);
-        if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
-      }
-    } else {
-      for (int u = 0; u < n; ++u) {
-        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u);
-        cp_async_slice<SB>(d + u * ROWB, my_src + (uint64_t)s * ROWB);
-        if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
-      }
-    }
-  };
-
-  for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {
-    const it_row_meta m = load_meta(p.meta + i);
-    const int32_t owner = Policy::NEEDS_OWNER ? __ldcs(p.owner + i) : 0;
-    // this warp's part of the row: edges [a, a + total)
-    const int part = (m.len + WARPS - 1) / WARPS;
-    const int first = warp * part < m.len ? warp * part : m.len;
-    const int total = (m.len - first) < part ? (m.len - first) : part;
-    const int64_t a = m.j0 + first;
-    float st[NS];
-    pol.init(st);
-    pol.begin_row(m.dest, owner);
-    auto load_chunk = [&](int base, int32_t &idx, float &w) {
-      idx = 0; w = 1.f;
-      if (base + lane < total) {
-        idx = __ldcs(p.indices + a + base + lane);
-        if (Policy::WEIGHTED) w = __ldcs(p.weights + a + base + lane);
-      }
-    };
-    int32_t idx_c, idx_n;
-    float w_c, w_n;
-    load_chunk(0, idx_c, w_c);
-    int fs = 0, cs = 0;
-#pragma unroll
-    for (int k = 0; k < AHEAD; k += R) {
-      if (k < total) fill(fs, idx_c, k, (total - k) < R ? (total - k) : R);
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      fs = fs + 1 == S ? 0 : fs + 1;
-    }
-    for (int base = 0; base < total; base += 32) {
-      load_chunk(base + 32, idx_n, w_n);
-      const int cnt = (total - base) < 32 ? (total - base) : 32;
-      for (int k0 = 0; k0 < cnt; k0 += R) {
-        const int f = k0 + AHEAD;
-        if (f < 32) {
-          const int left = cnt - f;
-          if (left > 0) fill(fs, idx_c, f, left < R ? left : R);
-        } else {
-          const int left = total - (base + f);
-          if (left > 0) fill(fs, idx_n, f - 32, left < R ? left : R);
-        }
-        fs = fs + 1 == S ? 0 : fs + 1;
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");
-        const int n = (cnt - k0) < R ? (cnt - k0) : R;
-        const uint32_t sr = my_ring + cs * (R * ROWB);
-        const uint32_t sx = my_xring + cs * (R * 128);
-        cs = cs + 1 == S ? 0 : cs + 1;
-        auto consume = [&](int u) {
-          const typename RowSlice<T, SB>::Raw raw = lds_slice<SB>(sr + u * ROWB);
-          const float w = Policy::WEIGHTED ? __shfl_sync(0xffffffffu, w_c, k0 + u) : 1.f;
-          const float x = Policy::HAS_EXTRA ? lds_f32(sx + u * 128) : 0.f;
-          pol.edge(st, raw, w, x);
-        };
-        if (n == R) {
-#pragma unroll
-          for (int u = 0; u < R; ++u) consume(u);
-        } else {
-          for (int u = 0; u < n; ++u) consume(u);
-        }
-      }
-      idx_c = idx_n; w_c = w_n;
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();  // red[] free again
-#pragma unroll
-    for (int k = 0; k < NS; ++k) red[warp][lane][k] = st[k];
-    __syncthreads();
-    if (warp == 0) {
-      for (int w = 1; w < WARPS; ++w) {
-        float other[NS];
-#pragma unroll
-        for (int k = 0; k < NS; ++k) other[k] = red[w][lane][k];
-        pol.merge(st, other);
-      }
-      pol.end_row(st, m.dest, owner, m.len);
-    }
-  }
-}
-
 // ----------------------------------------------------------------------------- empty rows
 template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, Policy pol) {
@@ -718,15 +391,24 @@ __global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, P
   }
 }
 
+}  // namespace it_stream
+
+#include "stream_ring.cuh"
+
+namespace it_stream {
+
 // ----------------------------------------------------------------------------- bucket dispatch
 // Longest rows first so that the tail of the launch sequence is made of short rows.
 // bytes_of(bucket, rows) gives the algorithmic bytes of a launch; kid_* the instrumentation ids.
+// Only the buckets whose bound lies in (bound_lo, bound_hi] are launched: callers may give long and short
+// rows different slice widths.
 template <typename T, int SB, int LPR, class Policy, class BytesF>
 it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, BytesF bytes_of, int kid_cta, int kid_rows,
-                         int kid_empty, cudaStream_t st) {
+                         int kid_empty, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
+  constexpr bool RING = SB * LPR >= 128;   // rows of 128 bytes and more are staged through shared memory
   for (int b = g->n_buckets - 1; b >= 0; --b) {
     const int64_t lo = g->h_bucket_offsets[b], hi = g->h_bucket_offsets[b + 1];
-    if (hi <= lo) continue;
+    if (hi <= lo || g->bucket_bounds[b] <= bound_lo || g->bucket_bounds[b] > bound_hi) continue;
     p.row_lo = lo; p.row_hi = hi;
     const int64_t bound = g->bucket_bounds[b];
     const int64_t rows = hi - lo;
@@ -737,16 +419,16 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
       unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
       IT_LAUNCH(kid_empty, bytes, 0, st, stream_empty_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
     } else if (bound > IT_GATHER_CTA_ABOVE) {
-      if constexpr (LPR == 32 && SB >= IT_RING_MIN_SB) {
+      if constexpr (RING) {
         constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
         static bool configured = false;   // per template instance
         if (!configured) {
-          IT_CUDA_TRY(cudaFuncSetAttribute(stream_cta_ring_kernel<T, SB, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+          IT_CUDA_TRY(cudaFuncSetAttribute(stream_cta_ring_kernel<T, SB, LPR, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
           configured = true;
         }
         // one CTA per row as far as the grid allows: the hardware hands out rows as CTAs retire
         unsigned blocks = (unsigned)(rows < (1 << 20) ? rows : (1 << 20));
-        IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_ring_kernel<T, SB, Policy><<<blocks, THREADS, smem, st>>>(p, pol));
+        IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_ring_kernel<T, SB, LPR, Policy><<<blocks, THREADS, smem, st>>>(p, pol));
       } else {
         unsigned blocks = (unsigned)(rows < max_blocks ? rows : max_blocks);
         IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
@@ -754,23 +436,25 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
     } else {
       // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
       int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
-      if (br > LPR) br = LPR;
-      p.batch_rows = br;
-      const int64_t batches = (rows + br - 1) / br;
-      int64_t want = (batches + (THREADS / LPR) - 1) / (THREADS / LPR);
-      unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
-      if constexpr (LPR == 32 && SB >= IT_RING_MIN_SB) {
+      if constexpr (RING) {   // a whole warp per batch
         constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
         static bool configured = false;   // per template instance
         if (!configured) {
-          IT_CUDA_TRY(cudaFuncSetAttribute(stream_rows_ring_kernel<T, SB, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+          IT_CUDA_TRY(cudaFuncSetAttribute(stream_rows_ring_kernel<T, SB, LPR, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
           configured = true;
         }
+        p.batch_rows = br;
+        const int64_t batches = (rows + br - 1) / br;
         const int64_t ring_max = (int64_t)g->num_sms * IT_RING_MIN_BLOCKS * 2;
-        const int64_t want_r = (batches + (THREADS / 32) - 1) / (THREADS / 32);
-        unsigned rblocks = (unsigned)(want_r < ring_max ? want_r : ring_max);
-        IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_ring_kernel<T, SB, Policy><<<rblocks, THREADS, smem, st>>>(p, pol));
-      } else {
+        const int64_t want = (batches + (THREADS / 32) - 1) / (THREADS / 32);
+        unsigned blocks = (unsigned)(want < ring_max ? want : ring_max);
+        IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_ring_kernel<T, SB, LPR, Policy><<<blocks, THREADS, smem, st>>>(p, pol));
+      } else {                                // a group of LPR lanes per batch
+        if (br > LPR) br = LPR;
+        p.batch_rows = br;
+        const int64_t batches = (rows + br - 1) / br;
+        int64_t want = (batches + (THREADS / LPR) - 1) / (THREADS / LPR);
+        unsigned blocks = (unsigned)(want < max_blocks ? want : max_blocks);
         IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
       }
     }
@@ -779,16 +463,28 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
   return IT_OK;
 }
 
-// Pick the slice width and group size for a row of `row_bytes` bytes and call f.template operator()<SB, LPR>().
+// Pick the slice width and group size for a row of `row_bytes` bytes and call
+// f.template operator()<SB, LPR>(bound_lo, bound_hi) for the buckets that take them.  Rows of 128 and 256
+// bytes use 16-byte slices for their long rows (unless `wide` is false) and one slice per lane for the short ones.
+#ifndef IT_WIDE_ABOVE
+#define IT_WIDE_ABOVE 32   // buckets of rows longer than this use 16-byte slices
+#endif
 template <class F>
-it_status dispatch_row_bytes(int row_bytes, F f) {
+it_status dispatch_row_bytes(int row_bytes, bool wide, F f) {
+  constexpr int64_t ALL = INT64_MAX;
   switch (row_bytes) {
-    case 512: return f.template operator()<16, 32>();
-    case 256: return f.template operator()<8, 32>();
-    case 128: return f.template operator()<4, 32>();
-    case 64: return f.template operator()<4, 16>();
-    case 32: return f.template operator()<4, 8>();
-    case 16: return f.template operator()<4, 4>();
+    case 512: return f.template operator()<16, 32>(-1, ALL);
+    case 256:
+      if (!wide) return f.template operator()<8, 32>(-1, ALL);
+      IT_TRY((f.template operator()<16, 16>(IT_WIDE_ABOVE, ALL)));
+      return f.template operator()<8, 32>(-1, IT_WIDE_ABOVE);
+    case 128:
+      if (!wide) return f.template operator()<4, 32>(-1, ALL);
+      IT_TRY((f.template operator()<16, 8>(IT_WIDE_ABOVE, ALL)));
+      return f.template operator()<4, 32>(-1, IT_WIDE_ABOVE);
+    case 64: return f.template operator()<4, 16>(-1, ALL);
+    case 32: return f.template operator()<4, 8>(-1, ALL);
+    case 16: return f.template operator()<4, 4>(-1, ALL);
   }
   it_set_error("feature row of %d bytes is not 16, 32, 64, 128, 256 or 512 bytes", row_bytes);
   return IT_ERR_UNSUPPORTED;
