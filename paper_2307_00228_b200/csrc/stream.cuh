@@ -43,6 +43,12 @@
 #ifndef IT_RING_STAGES
 #define IT_RING_STAGES 2
 #endif
+#ifndef IT_SHORT_MIN_BLOCKS
+#define IT_SHORT_MIN_BLOCKS 4   // resident CTAs per SM of the short-row kernel (eight 16-byte slices in flight per lane)
+#endif
+#ifndef IT_SHORT_BELOW
+#define IT_SHORT_BELOW 32       // 128-byte rows: buckets of rows up to this long take the short-row kernel
+#endif
 #ifndef IT_GATHER_CTA_ABOVE
 #define IT_GATHER_CTA_ABOVE 1024   // rows longer than this get a whole CTA; shorter ones a lane group or a warp
 #endif
@@ -287,6 +293,66 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
   }
 }
 
+// ----------------------------------------------------------------------------- short rows: one lane group each, no edge stream
+// For rows of at most a few dozen edges the bookkeeping of a flat edge stream costs more than the edges.
+// Here a group of LPR lanes (16-byte slices, LPR >= 8) owns one row: lanes 0..7 of the group fetch eight
+// source indices with one load, the group issues the eight row loads back to back and then reduces them;
+// rows longer than eight edges take more rounds.  The groups of a warp run in lockstep (warp-wide loop
+// bounds, predicated edges), so a warp never splits.
+template <typename T, int LPR, class Policy>
+__global__ void __launch_bounds__(THREADS, IT_SHORT_MIN_BLOCKS) stream_short_rows_kernel(StreamParams p, Policy pol) {
+  constexpr int NS = Policy::NS;
+  constexpr int E = 8;   // edges per round
+  static_assert(LPR >= E, "lanes 0..7 of a group fetch the indices of a round");
+  using Slice = RowSlice<T, 16>;
+  const int lane = threadIdx.x & 31;
+  const int t = lane % LPR, gbase = lane - t;
+  pol.setup(t);
+  const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * 16;
+  constexpr uint32_t ROWB = LPR * 16;
+  const int64_t rows_per_sweep = (int64_t)gridDim.x * (THREADS / LPR);
+  // warp-uniform loop: every group of the warp takes one row per iteration
+  for (int64_t i0 = p.row_lo + (int64_t)blockIdx.x * (THREADS / LPR) + (threadIdx.x >> 5) * (32 / LPR); i0 < p.row_hi; i0 += rows_per_sweep) {
+    const int64_t i = i0 + lane / LPR;
+    const bool valid = i < p.row_hi;
+    int64_t j0 = 0;
+    int len = 0, dest = 0, owner = 0;
+    if (valid) {
+      const it_row_meta m = load_meta(p.meta + i);
+      j0 = m.j0; len = m.len; dest = m.dest;
+      if (Policy::NEEDS_OWNER) owner = __ldcs(p.owner + i);
+    }
+    const int maxlen = __reduce_max_sync(0xffffffffu, len);
+    float st[NS];
+    pol.init(st);
+    if (valid) pol.begin_row(dest, owner);
+    for (int k0 = 0; k0 < maxlen; k0 += E) {
+      int32_t idx = 0;
+      float w = 1.f;
+      if (t < E && k0 + t < len) {
+        idx = __ldcs(p.indices + j0 + k0 + t);
+        if (Policy::WEIGHTED) w = __ldcs(p.weights + j0 + k0 + t);
+      }
+      typename Slice::Raw v[E];
+      float ww[E], xx[E];
+#pragma unroll
+      for (int k = 0; k < E; ++k) {
+        const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idx, gbase + k);
+        ww[k] = Policy::WEIGHTED ? __shfl_sync(0xffffffffu, w, gbase + k) : 1.f;
+        xx[k] = 0.f;
+        if (k0 + k < len) {
+          v[k] = Slice::load(my_src + (uint64_t)s * ROWB);
+          if (Policy::HAS_EXTRA) xx[k] = pol.extra(s);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < E; ++k)
+        if (k0 + k < len) pol.edge(st, v[k], ww[k], xx[k]);
+    }
+    if (valid) pol.end_row(st, dest, owner, len);
+  }
+}
+
 // ----------------------------------------------------------------------------- very long rows: one CTA each
 template <typename T, int SB, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kernel(StreamParams p, Policy pol) {
@@ -436,6 +502,15 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
     } else {
       // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
       int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
+      if constexpr (SB == 16 && LPR == 8) {   // 128-byte rows
+        if (bound <= IT_SHORT_BELOW) {   // one lane group per row
+          const int64_t short_max = (int64_t)g->num_sms * IT_SHORT_MIN_BLOCKS * 4;
+          const int64_t want = (rows + (THREADS / LPR) - 1) / (THREADS / LPR);
+          unsigned blocks = (unsigned)(want < short_max ? want : short_max);
+          IT_LAUNCH(kid_rows, bytes, 0, st, stream_short_rows_kernel<T, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
+          continue;
+        }
+      }
       if constexpr (RING) {   // a whole warp per batch
         constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
         static bool configured = false;   // per template instance
@@ -464,8 +539,9 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
 }
 
 // Pick the slice width and group size for a row of `row_bytes` bytes and call
-// f.template operator()<SB, LPR>(bound_lo, bound_hi) for the buckets that take them.  Rows of 128 and 256
-// bytes use 16-byte slices for their long rows (unless `wide` is false) and one slice per lane for the short ones.
+// f.template operator()<SB, LPR>(bound_lo, bound_hi) for the buckets that take them.  Unless `wide` is false,
+// rows of 128 bytes use 16-byte slices throughout and rows of 256 bytes use them for their long rows, with
+// one slice per lane for the short ones (measured: the cheaper end of row wins there).
 #ifndef IT_WIDE_ABOVE
 #define IT_WIDE_ABOVE 32   // buckets of rows longer than this use 16-byte slices
 #endif
@@ -480,8 +556,7 @@ it_status dispatch_row_bytes(int row_bytes, bool wide, F f) {
       return f.template operator()<8, 32>(-1, IT_WIDE_ABOVE);
     case 128:
       if (!wide) return f.template operator()<4, 32>(-1, ALL);
-      IT_TRY((f.template operator()<16, 8>(IT_WIDE_ABOVE, ALL)));
-      return f.template operator()<4, 32>(-1, IT_WIDE_ABOVE);
+      return f.template operator()<16, 8>(-1, ALL);
     case 64: return f.template operator()<4, 16>(-1, ALL);
     case 32: return f.template operator()<4, 8>(-1, ALL);
     case 16: return f.template operator()<4, 4>(-1, ALL);
