@@ -5,21 +5,25 @@
 // HBM-bound: one 4- to 16-byte load per lane per edge, several edges in flight per lane, a fixed
 // order of operations (results are bit-reproducible; no floating-point atomics anywhere).
 //
-// Work decomposition.  A feature row is LPR lanes wide (32 for rows of 128 bytes and more).
-//   * stream_rows_kernel: a *group* of LPR lanes takes a batch of rows of its bucket (one coalesced
-//     16-byte metadata load per row) and walks the batch's edges as one flat stream: the lanes
-//     load LPR source ids at a time (the next chunk is prefetched while the current one is
-//     consumed), every id is broadcast by shuffle, all lanes load their slice of that source
-//     row, UNROLL rows in flight, and a row is finished when the stream crosses its end.
-//     Short rows therefore cost no dependent-load round trip of their own.
-//   * stream_cta_kernel: one CTA per very long row, each warp a contiguous chunk, SLOTS = 32 / LPR
-//     edges at once per warp; slot and warp states are merged in a fixed order.
+// Work decomposition.  A feature row is cut into lane slices of SB bytes and is LPR = row bytes / SB
+// lanes wide; rows are bucketed by length and each bucket gets the kernel that suits it.
+//   * stream_rows_ring_kernel, stream_cta_ring_kernel (stream_ring.cuh; rows of 128 bytes and more):
+//     a warp walks the edges of a batch of rows (or of its part of one very long row) as one flat
+//     stream and stages the source rows through a per-warp ring in shared memory with cp.async.
+//   * stream_short_rows_kernel (128-byte rows of at most a few dozen edges): one group of 8 lanes
+//     per row, eight row loads back to back, no edge stream.
+//   * stream_rows_kernel (rows narrower than 128 bytes): a *group* of LPR lanes takes a batch of rows
+//     and walks the batch's edges as one flat stream with UNROLL rows in flight per lane in registers.
+//   * stream_cta_kernel (the same rows, very long): one CTA per row, each warp a contiguous chunk,
+//     SLOTS = 32 / LPR edges at once per warp; slot and warp states are merged in a fixed order.
+//   * stream_empty_kernel: rows without edges.
 //
 // Policy interface (all __device__):
 //   static constexpr int NS;                 // floats of per-lane state
 //   static constexpr bool WEIGHTED, HAS_EXTRA, NEEDS_OWNER;
 //   void init(float (&st)[NS]);
 //   float extra(uint32_t src_row);           // per-edge scalar that is loaded with the row (HAS_EXTRA)
+//   const float *extra_ptr(uint32_t src_row);   // its address, for the asynchronous copies of the ring kernels
 //   void edge(float (&st)[NS], const Raw &raw, float w, float x);   // Raw = the packed slice
 //   void merge(float (&st)[NS], const float (&other)[NS]);     // other comes later in edge order
 //   void begin_row(int32_t dest, int32_t owner);               // prefetch what end_row needs
@@ -58,11 +62,9 @@ namespace it_stream {
 constexpr int THREADS = 256;
 constexpr int UNROLL = IT_GATHER_UNROLL;
 
-// One lane's slice of a feature row: SB = 4, 8 or 16 bytes.  Rows of 128 bytes and more are spread
-// over all 32 lanes of a warp (SB = row bytes / 32), so that every load instruction fetches one whole
-// row and a warp never has to split into independently running lane groups; narrower rows use 4-byte
-// slices and a group of LPR = row bytes / 4 lanes.  A slice stays packed in registers while it is in
-// flight and is widened to fp32 only when it is consumed.
+// One lane's slice of a feature row: SB = 4, 8 or 16 bytes, LPR = row bytes / SB lanes per row (see
+// dispatch_row_bytes for the choice).  A slice stays packed while it is in flight and is widened to fp32
+// only when it is consumed.
 template <int SB> struct SliceRaw;
 template <> struct SliceRaw<4> { using type = uint32_t; };
 template <> struct SliceRaw<8> { using type = uint2; };
