@@ -18,6 +18,14 @@
 
 #include "common.cuh"
 
+// fp32 mode: the tensor core ignores the low 13 mantissa bits of a tf32 operand, so the raw fp32 tile serves
+// as A_hi as it is and only A_lo = x - trunc(x) has to be written.  (Were the operand rounded instead, half
+// of the products would be off by 2^-11 relative, ten times the fp32 parity tolerance: the parity tests pin
+// this.)  Set to 1 to store the truncated hi part back over the raw tile.
+#ifndef IT_TC_REWRITE_HI
+#define IT_TC_REWRITE_HI 0
+#endif
+
 namespace {
 
 constexpr int TC_BM = 128;          // rows per tile (UMMA M)
@@ -156,7 +164,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // [nbc]
   float *att_s = bias_s + p.nbc;   // [2][nbc]: source vector, destination vector (only with scores)
 
-  const uint32_t acc_cols = (uint32_t)p.nbc;
+  // fp32 mode: columns [nbc, 2 nbc) of an accumulator hold A_hi * B_lo, added to the first half by the epilogue
+  const uint32_t acc_cols = (uint32_t)p.nbc * (TF32 ? 2u : 1u);
   uint32_t tmem_cols = 32;
   while (tmem_cols < 2 * acc_cols) tmem_cols <<= 1;
 
@@ -202,9 +211,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       // the weights of this CTA's columns, once
       mbar_arrive_expect_tx(b_full, (uint32_t)b_bytes);
       const int bk_elems = TF32 ? 32 : 64;
-      for (int part = 0; part < (TF32 ? 2 : 1); ++part)
+      // fp32 mode: the hi and the lo tile of a k-block sit next to each other, so that one descriptor covers
+      // both as a single operand of 2 nbc columns
+      constexpr int parts = TF32 ? 2 : 1;
+      for (int part = 0; part < parts; ++part)
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_2d(smem_b + (size_t)(part * KB + kb) * b_tile_bytes, &map_b, kb * bk_elems, part * p.NB + col_base, b_full);
+          tma_load_2d(smem_b + (size_t)(kb * parts + part) * b_tile_bytes, &map_b, kb * bk_elems, part * p.NB + col_base, b_full);
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -231,6 +243,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       // instruction descriptor: D = fp32, A/B = bf16 or tf32, both K-major, N = nbc, M = 128
       const uint32_t fmt = TF32 ? 2u : 1u;
       const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.nbc >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      const uint32_t idesc_wide = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)((2 * p.nbc) >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
       bool ok = mbar_wait(b_full, 0, abort_flag);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
@@ -246,16 +259,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
           if (!ok) break;
           tc_fence_after();
           const uint32_t a_hi = smem_u32(smem_a + (size_t)stage * a_tile_bytes);
-          const uint32_t b_hi = smem_u32(smem_b + (size_t)kb * b_tile_bytes);
+          const uint32_t b_hi = smem_u32(smem_b + (size_t)kb * (TF32 ? 2 : 1) * b_tile_bytes);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {   // four 32-byte K steps inside the 128-byte swizzle row
             const uint32_t first = (kb | k) != 0;
-            tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc, first);
             if (TF32) {
+              // A_hi * [B_hi | B_lo] in one instruction (A_hi is read once), then A_lo * B_hi onto the first half
               const uint32_t a_lo = smem_u32(smem_lo + (size_t)lo * a_tile_bytes);
-              const uint32_t b_lo = b_hi + (uint32_t)(KB * b_tile_bytes);
+              tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc_wide, first);
               tc_mma<TF32>(d_tmem, make_desc(a_lo + k * 32), make_desc(b_hi + k * 32), idesc, 1u);
-              tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_lo + k * 32), idesc, 1u);
+            } else {
+              tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc, first);
             }
           }
           tc_commit(&empty[stage]);   // stage reusable once these MMAs have read it
@@ -304,15 +318,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       for (int u = 0; u < n_units; ++u) {
         if (((unit0 + u) & 3) != sub) continue;
         float sc_a = 0.f, sc_b = 0.f;   // attention scores of this head
-        for (int j0 = 0; j0 < gph; j0 += 2) {
-          // up to two 16-column groups in flight from TMEM, one wait
+        constexpr int GSTEP = TF32 ? 1 : 2;
+        for (int j0 = 0; j0 < gph; j0 += GSTEP) {
+          // two loads of 16 columns in flight from TMEM, one wait: two groups, or (fp32 mode) one group and its
+          // A_hi * B_lo correction
           uint32_t r[2][16];
           const int c_first = (u * gph + j0) * 16;          // local column of the first group
-          const int n_g = (gph - j0) >= 2 ? 2 : 1;
+          const int n_g = TF32 ? 1 : ((gph - j0) >= 2 ? 2 : 1);
           tmem_ld16(taddr + (uint32_t)c_first, r[0]);
-          if (n_g == 2) tmem_ld16(taddr + (uint32_t)c_first + 16, r[1]);
+          if (TF32) tmem_ld16(taddr + (uint32_t)(p.nbc + c_first), r[1]);
+          else if (n_g == 2) tmem_ld16(taddr + (uint32_t)c_first + 16, r[1]);
           tmem_ld_wait();
-          if (u == last_u && j0 + 2 >= gph) release();
+          if (u == last_u && j0 + GSTEP >= gph) release();
+          if (TF32) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r[0][i] = __float_as_uint(__uint_as_float(r[0][i]) + __uint_as_float(r[1][i]));
+          }
 #pragma unroll
           for (int k = 0; k < 2; ++k) {
             if (k >= n_g) break;
@@ -433,7 +454,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
             h.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u); l.y = x.y - h.y;
             h.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); l.z = x.z - h.z;
             h.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u); l.w = x.w - h.w;
-            hi_t[i] = h;
+            if (IT_TC_REWRITE_HI) hi_t[i] = h;
             lo_t[i] = l;
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
@@ -531,7 +552,7 @@ static bool tc_split(bool tf32, int NB, int KB, int *n_splits, int *nbc) {
   for (int s = 1; s <= 16; ++s) {
     if (NB % s != 0) continue;
     const int c = NB / s;
-    if (c % 16 != 0 || c > 256) continue;
+    if (c % 16 != 0 || c > (tf32 ? 128 : 256)) continue;   // fp32 mode issues MMAs of 2 c columns and keeps 4 c TMEM columns
     if ((size_t)(tf32 ? 2 : 1) * KB * c * TC_KBLOCK_BYTES > 128 * 1024) continue;
     *n_splits = s; *nbc = c;
     return true;
