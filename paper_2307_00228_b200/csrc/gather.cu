@@ -96,14 +96,23 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
     const float inv = (p.is_mean && deg > 0) ? 1.f / (float)deg : 1.f;
     for (int c = lane * 4; c < p.dim; c += 128) {
       float4 acc = __ldg(reinterpret_cast<const float4 *>(p.partials + p0 * p.dim + c));
-      for (int64_t g = 1; g < r1 - r0; ++g) {
-        float4 y = __ldg(reinterpret_cast<const float4 *>(p.partials + (p0 + g) * p.dim + c));
+      auto fold = [&](const float4 &y) {
         if (p.is_max) {
           acc.x = fmaxf(acc.x, y.x); acc.y = fmaxf(acc.y, y.y); acc.z = fmaxf(acc.z, y.z); acc.w = fmaxf(acc.w, y.w);
         } else {
           acc.x += y.x; acc.y += y.y; acc.z += y.z; acc.w += y.w;
         }
+      };
+      const int64_t n = r1 - r0;
+      int64_t g = 1;
+      for (; g + 8 <= n; g += 8) {   // eight partial rows in flight, folded in group order
+        float4 y[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) y[k] = __ldg(reinterpret_cast<const float4 *>(p.partials + (p0 + g + k) * p.dim + c));
+#pragma unroll
+        for (int k = 0; k < 8; ++k) fold(y[k]);
       }
+      for (; g < n; ++g) fold(__ldg(reinterpret_cast<const float4 *>(p.partials + (p0 + g) * p.dim + c)));
       float o[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
       const int64_t off = v * p.dim + c;
       if (p.epi == IT_EPI_ADD_ACT) {
