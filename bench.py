@@ -166,6 +166,24 @@ class ClockSampler:
         return out
 
 
+# ----------------------------------------------------------------------------- ranks
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: the replicas run side by side, so the whole job takes as long as that rank."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Units all ranks processed per second (every rank runs the same workload: weak scaling)."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- the GPU arm
 
 def run_ours(args):
@@ -238,12 +256,9 @@ def run_ours(args):
     launches = B.it_kernel_launch_count() - launches0
     ms_total = ev0.elapsed_time(ev1)
     clocks = sampler.stop()
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
-    value = world * w.n / (ms_per_step * 1e-3)
+    value = whole_job_value(w.n, world, ms_per_step)
 
     # ---- per-layer edges/s (each layer alone, same buffers as a real pass)
     layer_stats = []
@@ -293,11 +308,9 @@ def run_ours(args):
             e2e_step()
         b.record()
         torch.cuda.synchronize()
-        t = torch.tensor([a.elapsed_time(b) / k], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * w.n / (float(t.item()) * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "ms_per_step": float(t.item()), "steps": k}
+        e2e_ms = max_over_ranks(a.elapsed_time(b) / k, world, dev)
+        e2e = {"value": whole_job_value(w.n, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": k}
 
     if rank != 0:
         if world > 1:
