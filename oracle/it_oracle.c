@@ -33,7 +33,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ITO_SUM = 0, ITO_MEAN = 1, ITO_MAX = 2 };
+enum { ITO_SUM = 0, ITO_MEAN = 1, ITO_MAX = 2, ITO_MIN = 3 };
 enum { ITO_ACT_NONE = 0, ITO_ACT_RELU = 1, ITO_ACT_ELU = 2 };
 
 /* ------------------------------------------------------------------ index side */
@@ -108,6 +108,8 @@ int ito_buckets(int64_t n_rows, const int64_t *shadow_indptr, int32_t nb, const 
  *   sum : a_v    = sum_j w_j h_{u_j}
  *   mean: a_v    = (sum_j w_j h_{u_j}) / d_v        (d_v = number of in-edges)
  *   max : a_v[f] = max_j (w_j h_{u_j}[f])
+ *   min : a_v[f] = min_j (w_j h_{u_j}[f])      (Section "Background", message passing: the reduce
+ *                                               may be sum, mean, max or min pooling)
  * An empty in-neighbourhood gives a_v = 0.  H is [n_src, F] row-major, A is [n, F]. */
 void ito_aggregate(int64_t n, const int64_t *indptr, const int32_t *indices, const double *w,
                    const double *H, int32_t F, int32_t op, double *A) {
@@ -122,6 +124,7 @@ void ito_aggregate(int64_t n, const int64_t *indptr, const int32_t *indices, con
             for (int32_t f = 0; f < F; ++f) {
                 double m = wj * h[f];
                 if (op == ITO_MAX) a[f] = (j == j0 || m > a[f]) ? m : a[f];
+                else if (op == ITO_MIN) a[f] = (j == j0 || m < a[f]) ? m : a[f];
                 else a[f] += m;
             }
         }
@@ -135,12 +138,12 @@ void ito_aggregate(int64_t n, const int64_t *indptr, const int32_t *indices, con
  * P is [R, F]. */
 void ito_partial_gather(int64_t n_rows, const int64_t *shadow_indptr, const int32_t *indices,
                         const double *w, const double *H, int32_t F, int32_t op, double *P) {
-    ito_aggregate(n_rows, shadow_indptr, indices, w, H, F, op == ITO_MAX ? ITO_MAX : ITO_SUM, P);
+    ito_aggregate(n_rows, shadow_indptr, indices, w, H, F, (op == ITO_MAX || op == ITO_MIN) ? op : ITO_SUM, P);
 }
 
 /* Combine: the receiver aggregates the partial results of one vertex "as usual", in
  * group order.  Empty groups can only occur for d = 0 (a single empty row), so a max
- * never sees a spurious 0.  deg[v] = indptr[v+1]-indptr[v] of the unsplit graph. */
+ * or a min never sees a spurious 0.  deg[v] = indptr[v+1]-indptr[v] of the unsplit graph. */
 void ito_combine(int64_t n, const int64_t *owner_indptr, const int64_t *indptr, const double *P,
                  int32_t F, int32_t op, double *A) {
 #pragma omp parallel for schedule(static)
@@ -152,6 +155,7 @@ void ito_combine(int64_t n, const int64_t *owner_indptr, const int64_t *indptr, 
             for (int32_t f = 0; f < F; ++f) {
                 double p = P[r * F + f];
                 if (op == ITO_MAX) a[f] = p > a[f] ? p : a[f];
+                else if (op == ITO_MIN) a[f] = p < a[f] ? p : a[f];
                 else a[f] += p;
             }
         int64_t d = indptr[v + 1] - indptr[v];

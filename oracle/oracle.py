@@ -26,7 +26,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_HERE, "libit_oracle.so")
 _SRC = os.path.join(_HERE, "it_oracle.c")
 
-OPS = {"sum": 0, "mean": 1, "max": 2}
+OPS = {"sum": 0, "mean": 1, "max": 2, "min": 3}
 ACTS = {"none": 0, "relu": 1, "elu": 2}
 
 
@@ -247,8 +247,8 @@ def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=
         indptr, indices, w = _sub_csr(indptr, indices, w, rows)
         Hself = H[_i64(rows)]
     if reorder:
-        if layer.op == "max":
-            raise ValueError("transform-before-aggregate is not valid for max")
+        if layer.op in ("max", "min"):
+            raise ValueError("transform-before-aggregate is not valid for max or min")
         if rows is None:
             Z = round_to(linear(H, W[Fi:]), storage)
         else:   # transform only the rows that are read

@@ -133,7 +133,7 @@ def tree_eval(v, depth, ip, ix, w, x, layers, memo=None):
     if hn:
         for f in range(Fi):
             msgs = [wj * h[f] for (_, wj), h in zip(nb, hn)]
-            agg[f] = max(msgs) if lay.op == "max" else sum(msgs)
+            agg[f] = max(msgs) if lay.op == "max" else (min(msgs) if lay.op == "min" else sum(msgs))
             if lay.op == "mean":
                 agg[f] /= len(msgs)
     out = []
@@ -144,7 +144,7 @@ def tree_eval(v, depth, ip, ix, w, x, layers, memo=None):
     return out
 
 
-@pytest.mark.parametrize("op", ["sum", "mean", "max", "gat"])
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "min", "gat"])
 @pytest.mark.parametrize("depth", [1, 2, 3])
 def test_layerwise_equals_computation_tree(op, depth):
     rng = np.random.default_rng(100 + depth)
@@ -253,7 +253,7 @@ def test_split_rule_closed_forms(T):
         assert np.all(np.diff(g) <= 0)        # the larger groups come first
 
 
-@pytest.mark.parametrize("op", ["sum", "mean", "max"])
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "min"])
 def test_split_invariance(op):
     """Partial gather + combine does not change the result (associativity): bit-exact for
     max and for integer-valued inputs, to rounding for general floats."""
@@ -268,7 +268,7 @@ def test_split_invariance(op):
         sp, so, owner = O.split_hubs(ip, T)
         got = O.combine(owner, ip, O.partial_gather(sp, ix, w, H, op), op)
         got_i = O.combine(owner, ip, O.partial_gather(sp, ix, wi, Hi, op), op)
-        if op == "max":
+        if op in ("max", "min"):
             assert np.array_equal(got, base)
         else:
             assert np.allclose(got, base, rtol=1e-12, atol=1e-12)
@@ -363,6 +363,29 @@ def test_mean_of_constant_is_constant_and_max_dominates_mean():
     # max of all-negative messages stays negative (no spurious 0 from the initial value)
     mxn = O.aggregate(ip, ix, None, -np.abs(H) - 1, "max")
     assert np.all(mxn[deg > 0] < 0)
+
+
+def test_min_pooling_against_numpy_and_against_max():
+    """min pooling (the reduce of Eq. (1) may be sum, mean, max or min): per destination the plain numpy
+    minimum over its gathered messages; equal to -max of the negated messages; an empty neighbourhood gives
+    0; all-positive messages stay positive (no spurious 0 from the initial value)."""
+    rng = np.random.default_rng(21)
+    n = 150
+    ip, ix = random_graph(rng, n, 10)
+    deg = np.diff(ip)
+    H = rng.standard_normal((n, 4))
+    w = rng.random(ix.shape[0]) + 0.1
+    for ww in (None, w):
+        got = O.aggregate(ip, ix, ww, H, "min")
+        for v in range(n):
+            msgs = H[ix[ip[v]:ip[v + 1]]] * (1.0 if ww is None else ww[ip[v]:ip[v + 1], None])
+            want = msgs.min(axis=0) if deg[v] else np.zeros(4)
+            assert np.array_equal(got[v], want)
+        assert np.array_equal(got, -O.aggregate(ip, ix, ww, -H, "max"))
+    pos = O.aggregate(ip, ix, None, np.abs(H) + 1, "min")
+    assert np.all(pos[deg > 0] > 0) and np.all(pos[deg == 0] == 0)
+    mn, me = O.aggregate(ip, ix, None, H, "min"), O.aggregate(ip, ix, None, H, "mean")
+    assert np.all(mn[deg > 0] <= me[deg > 0] + 1e-15)
 
 
 def test_permutation_invariance_inside_segments():
