@@ -41,7 +41,7 @@ typedef enum {
 
 typedef enum { IT_F32 = 0, IT_BF16 = 1 } it_dtype;
 typedef enum { IT_I32 = 0, IT_I64 = 1 } it_itype;
-typedef enum { IT_GATHER_SUM = 0, IT_GATHER_MEAN = 1, IT_GATHER_MAX = 2, IT_GATHER_GAT = 3 } it_gather_op;
+typedef enum { IT_GATHER_SUM = 0, IT_GATHER_MEAN = 1, IT_GATHER_MAX = 2, IT_GATHER_GAT = 3, IT_GATHER_MIN = 4 } it_gather_op;
 typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
 
 #define IT_MAX_BUCKETS 8
@@ -51,7 +51,7 @@ typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
  * `op` is the aggregate of the Gather stage, W / bias / act are apply_node, and
  * use_edge_weights selects the minimal apply_edge (message = w_e * h_src).
  *
- * GraphSAGE (op = SUM | MEAN | MAX):
+ * GraphSAGE (op = SUM | MEAN | MAX | MIN; the paper's message-passing paradigm lists all four poolings):
  *     a_v  = op_{e = (u -> v)} ( w_e * h_u )            (0 for a vertex with no in-edge;
  *                                                        MEAN divides by the edge count)
  *     h'_v = act( h_v * W[0:in_dim, :] + a_v * W[in_dim:2*in_dim, :] + bias )

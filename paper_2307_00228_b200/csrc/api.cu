@@ -16,7 +16,7 @@ struct LayerWs {
 
 it_status check_layer(const it_graph *g, const it_layer_desc *L) {
   IT_REQUIRE(L != nullptr, IT_ERR_INVALID_ARG, "layer is NULL");
-  IT_REQUIRE(L->op >= IT_GATHER_SUM && L->op <= IT_GATHER_GAT, IT_ERR_INVALID_ARG, "bad gather op %d", (int)L->op);
+  IT_REQUIRE(L->op >= IT_GATHER_SUM && L->op <= IT_GATHER_MIN, IT_ERR_INVALID_ARG, "bad gather op %d", (int)L->op);
   IT_REQUIRE(L->act >= IT_ACT_NONE && L->act <= IT_ACT_ELU, IT_ERR_INVALID_ARG, "bad activation %d", (int)L->act);
   IT_REQUIRE(L->feat_dtype == IT_F32 || L->feat_dtype == IT_BF16, IT_ERR_INVALID_ARG, "bad feat_dtype");
   IT_REQUIRE(L->weight_dtype == L->feat_dtype, IT_ERR_UNSUPPORTED, "weight_dtype must equal feat_dtype");

@@ -9,7 +9,9 @@ using namespace it_stream;
 constexpr int GATHER_THREADS = THREADS;
 
 // Per lane: VEC fp32 accumulators for its slice of the row.
-template <typename T, int SB, bool IS_MAX, bool WEIGHTED_>
+enum { RED_SUM = 0, RED_MAX = 1, RED_MIN = 2 };   // sum also serves mean (the division happens once, at the end)
+
+template <typename T, int SB, int RED, bool WEIGHTED_>
 struct SagePolicy {
   using Slice = RowSlice<T, SB>;
   static constexpr int VEC = Slice::VEC;
@@ -26,7 +28,7 @@ struct SagePolicy {
   __device__ __forceinline__ void setup(int t) { col = t * VEC; }
   __device__ __forceinline__ void init(float (&st)[NS]) const {
 #pragma unroll
-    for (int k = 0; k < NS; ++k) st[k] = IS_MAX ? -INFINITY : 0.f;
+    for (int k = 0; k < NS; ++k) st[k] = RED == RED_MAX ? -INFINITY : (RED == RED_MIN ? INFINITY : 0.f);
   }
   __device__ __forceinline__ float extra(uint32_t) const { return 0.f; }
   __device__ __forceinline__ const float *extra_ptr(uint32_t) const { return nullptr; }
@@ -35,20 +37,21 @@ struct SagePolicy {
     Slice::unpack(raw, f);
 #pragma unroll
     for (int k = 0; k < VEC; ++k) {
-      if (IS_MAX) st[k] = fmaxf(st[k], WEIGHTED ? w * f[k] : f[k]);
+      if (RED == RED_MAX) st[k] = fmaxf(st[k], WEIGHTED ? w * f[k] : f[k]);
+      else if (RED == RED_MIN) st[k] = fminf(st[k], WEIGHTED ? w * f[k] : f[k]);
       else st[k] = WEIGHTED ? fmaf(w, f[k], st[k]) : st[k] + f[k];
     }
   }
   __device__ __forceinline__ void merge(float (&st)[NS], const float (&o)[NS]) const {
 #pragma unroll
-    for (int k = 0; k < NS; ++k) st[k] = IS_MAX ? fmaxf(st[k], o[k]) : st[k] + o[k];
+    for (int k = 0; k < NS; ++k) st[k] = RED == RED_MAX ? fmaxf(st[k], o[k]) : (RED == RED_MIN ? fminf(st[k], o[k]) : st[k] + o[k]);
   }
   // the matching slice of the self term is fetched when the row starts, so that end_row does not wait for it
   __device__ __forceinline__ void begin_row(int32_t dest, int32_t) {
     if (epi == IT_EPI_ADD_ACT && dest >= 0) load_floats_stream<VEC>(self_term + (int64_t)dest * dim + col, self);
   }
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t len) const {
-    if (IS_MAX && len == 0) {
+    if (RED != RED_SUM && len == 0) {
 #pragma unroll
       for (int i = 0; i < VEC; ++i) st[i] = 0.f;
     }
@@ -81,7 +84,7 @@ struct CombineParams {
   const float *__restrict__ self_term;
   int64_t n_split_owners;
   int dim;
-  int is_max, is_mean, epi, act;
+  int red, is_mean, epi, act;   // red: RED_SUM / RED_MAX / RED_MIN
 };
 
 template <typename T>
@@ -97,8 +100,10 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
     for (int c = lane * 4; c < p.dim; c += 128) {
       float4 acc = __ldg(reinterpret_cast<const float4 *>(p.partials + p0 * p.dim + c));
       auto fold = [&](const float4 &y) {
-        if (p.is_max) {
+        if (p.red == RED_MAX) {
           acc.x = fmaxf(acc.x, y.x); acc.y = fmaxf(acc.y, y.y); acc.z = fmaxf(acc.z, y.z); acc.w = fmaxf(acc.w, y.w);
+        } else if (p.red == RED_MIN) {
+          acc.x = fminf(acc.x, y.x); acc.y = fminf(acc.y, y.y); acc.z = fminf(acc.z, y.z); acc.w = fminf(acc.w, y.w);
         } else {
           acc.x += y.x; acc.y += y.y; acc.z += y.z; acc.w += y.w;
         }
@@ -132,9 +137,9 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 }
 
 // ----------------------------------------------------------------------------- dispatch
-template <typename T, int SB, int LPR, bool IS_MAX, bool WEIGHTED>
+template <typename T, int SB, int LPR, int RED, bool WEIGHTED>
 it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
-  SagePolicy<T, SB, IS_MAX, WEIGHTED> pol;
+  SagePolicy<T, SB, RED, WEIGHTED> pol;
   pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.dim = a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
   const it_graph *g = a.g;
@@ -150,10 +155,11 @@ it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_
 
 template <typename T>
 it_status launch_lpr(const it_gather_args &a, StreamParams sp, cudaStream_t st) {
-  const bool mx = a.op == IT_GATHER_MAX, w = a.use_edge_weights != 0;
+  const bool w = a.use_edge_weights != 0;
   return dispatch_row_bytes(a.dim * (int)sizeof(T), true, [&]<int SB, int LPR>(int64_t lo, int64_t hi) {
-    if (mx) return w ? launch_policy<T, SB, LPR, true, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, true, false>(a, sp, lo, hi, st);
-    return w ? launch_policy<T, SB, LPR, false, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, false, false>(a, sp, lo, hi, st);
+    if (a.op == IT_GATHER_MAX) return w ? launch_policy<T, SB, LPR, RED_MAX, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, RED_MAX, false>(a, sp, lo, hi, st);
+    if (a.op == IT_GATHER_MIN) return w ? launch_policy<T, SB, LPR, RED_MIN, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, RED_MIN, false>(a, sp, lo, hi, st);
+    return w ? launch_policy<T, SB, LPR, RED_SUM, true>(a, sp, lo, hi, st) : launch_policy<T, SB, LPR, RED_SUM, false>(a, sp, lo, hi, st);
   });
 }
 
@@ -161,7 +167,8 @@ it_status launch_lpr(const it_gather_args &a, StreamParams sp, cudaStream_t st) 
 
 it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
   const it_graph *g = a.g;
-  IT_REQUIRE(a.op == IT_GATHER_SUM || a.op == IT_GATHER_MEAN || a.op == IT_GATHER_MAX, IT_ERR_INVALID_ARG, "gather: bad op");
+  IT_REQUIRE(a.op == IT_GATHER_SUM || a.op == IT_GATHER_MEAN || a.op == IT_GATHER_MAX || a.op == IT_GATHER_MIN, IT_ERR_INVALID_ARG,
+             "gather: bad op");
   IT_REQUIRE(!a.use_edge_weights || g->edge_weights, IT_ERR_INVALID_ARG, "layer uses edge weights but the graph has none");
   IT_REQUIRE(g->n_partial_rows == 0 || a.partials, IT_ERR_WORKSPACE, "gather: no partial buffer");
   if (g->n == 0) return IT_OK;
@@ -174,7 +181,7 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
     CombineParams c;
     c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.shadow_indptr = g->shadow_indptr;
     c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.n_split_owners = g->n_split_owners;
-    c.dim = a.dim; c.is_max = a.op == IT_GATHER_MAX; c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
+    c.dim = a.dim; c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
     int64_t want = (g->n_split_owners + 7) / 8;
     int64_t cap = (int64_t)g->num_sms * 8;
     unsigned blocks = (unsigned)(want < cap ? want : cap);

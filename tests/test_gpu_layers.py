@@ -15,13 +15,13 @@ HUBS = (257, 300, 1000, 2500, 33, 32, 9, 8, 1)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("op", ["sum", "mean", "max"])
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "min"])
 @pytest.mark.parametrize("weights", [False, True])
 @pytest.mark.parametrize("threshold", [0, 64, 1000])
 def test_sage_layer_parity(dtype, op, weights, threshold):
     # 1500 vertices: several 128-row GEMM tiles and a ragged tail; every degree bucket is populated
     fi, fo = 64, 32
-    for reorder in ([False, True] if op != "max" else [False]):
+    for reorder in ([False, True] if op in ("sum", "mean") else [False]):
         layer = make_sage_layer(1, op, "relu", fi, fo, dtype, weights=weights, allow_reorder=reorder)
         w = small_workload(2, 1500, 40, dtype, [layer], hubs=HUBS, weights=weights, threshold=threshold)
         got, d = run_device(w)
@@ -35,7 +35,7 @@ def test_sage_layer_parity(dtype, op, weights, threshold):
                                         ("bf16", (128, 64)), ("bf16", (256, 32))])
 def test_every_supported_row_width(dtype, dims):
     fi, fo = dims
-    for op in ("mean", "max"):
+    for op in ("mean", "max", "min"):
         layer = make_sage_layer(3, op, "none", fi, fo, dtype)
         w = small_workload(4, 700, 20, dtype, [layer], hubs=(400, 90), threshold=128)
         got, _ = run_device(w)
@@ -116,11 +116,12 @@ def test_run_to_run_results_are_bit_identical():
     assert all(torch.equal(outs[0], o) for o in outs[1:])
 
 
-def test_split_does_not_change_max_and_integer_sums():
-    """Partial gather + combine: exact for max, and for sums of small integers."""
+def test_split_does_not_change_max_min_and_integer_sums():
+    """Partial gather + combine: exact for max and min, and for sums of small integers."""
     lay_max = make_sage_layer(18, "max", "none", 32, 32, "f32")
+    lay_min = make_sage_layer(18, "min", "none", 32, 32, "f32")
     lay_sum = make_sage_layer(19, "sum", "none", 32, 32, "f32")
-    for lay in (lay_max, lay_sum):
+    for lay in (lay_max, lay_min, lay_sum):
         lay.W[:] = 0
         lay.W[32:] = np.eye(32, dtype=np.float32)   # output = the aggregate itself
         lay.bias = None
