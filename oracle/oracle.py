@@ -290,16 +290,54 @@ def gat_layer(indptr, indices, H, layer, storage=None, rows=None):
     return round_to(bias_act(O, layer.bias, layer.act), storage)
 
 
+def dense_layer(H, layer, storage=None, rows=None):
+    """A layer without a Gather stage: h' = act(h W + b), W [in, out].  This is the initialisation step of
+    the first superstep (raw vertex states -> initial embeddings) and the prediction part attached after
+    the last apply_node (Section "Implementation on Pregel")."""
+    H = _f64(H)
+    if rows is not None:
+        H = H[_i64(rows)]
+    return round_to(bias_act(linear(H, _f64(layer.W)), layer.bias, layer.act), storage)
+
+
+def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
+    """GCN in the message-passing form of Eq. (1): the message is the source state (times the edge weight,
+    which carries the degree normalisation; self loops are edges of the graph), the reduce is a sum, and
+    the update is dense on the aggregate alone: h'_v = act((sum_e w_e h_u) W + b), W [in, out].
+    reorder=True evaluates the algebraically equal form that gathers Z = H W."""
+    H = _f64(H)
+    W = _f64(layer.W)
+    w = edge_weights if layer.use_edge_weights else None
+    if rows is not None:
+        indptr, indices, w = _sub_csr(indptr, indices, w, rows)
+    if reorder:
+        if rows is None:
+            Z = round_to(linear(H, W), storage)
+        else:   # transform only the rows that are read
+            need = np.unique(indices.astype(np.int64))
+            Z = np.full((H.shape[0], layer.out_dim), np.nan)
+            Z[need] = round_to(linear(H[need], W), storage)
+        out = bias_act(_gathered(indptr, indices, w, Z, "sum", threshold), layer.bias, layer.act)
+    else:
+        A = round_to(_gathered(indptr, indices, w, H, "sum", threshold), storage)
+        out = bias_act(linear(A, W), layer.bias, layer.act)
+    return round_to(out, storage)
+
+
 def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
     if layer.op == "gat":
         return gat_layer(indptr, indices, H, layer, storage, rows)
+    if layer.op == "dense":
+        return dense_layer(H, layer, storage, rows)
+    if layer.op == "gcn":
+        return gcn_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows)
     return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows)
 
 
 def will_reorder(layer) -> bool:
     """The layer contract: transform first when it shrinks the rows that are gathered and
     the aggregate is linear."""
-    return bool(layer.allow_reorder) and layer.op in ("sum", "mean") and layer.out_dim < layer.in_dim
+    return bool(layer.allow_reorder) and layer.op in ("sum", "mean", "gcn") and layer.out_dim < layer.in_dim
 
 
 def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, follow_reorder=False):

@@ -17,7 +17,7 @@ GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "w5.json
 def L(op="sum", act="none", W=None, bias=None, heads=1, att_src=None, att_dst=None, slope=0.2,
       use_edge_weights=False, allow_reorder=True):
     W = np.asarray(W, dtype=np.float64)
-    in_dim = W.shape[0] if op == "gat" else W.shape[0] // 2
+    in_dim = W.shape[0] if op in ("gat", "dense", "gcn") else W.shape[0] // 2
     return NS(op=op, act=act, in_dim=in_dim, out_dim=W.shape[1], W=W,
               bias=None if bias is None else np.asarray(bias, dtype=np.float64), heads=heads,
               att_src=None if att_src is None else np.asarray(att_src, dtype=np.float64),
@@ -334,6 +334,59 @@ def test_self_and_neighbour_blocks_are_not_swapped():
     assert np.allclose(out, H @ Ws + (dense_adjacency(ip, ix, None, n) @ H) @ Wn + b, rtol=1e-13, atol=1e-13)
 
 
+def test_dense_layer_is_plain_matmul_bias_activation():
+    """The layer without a Gather stage (initial transform, prediction part): numpy's act(H W + b)."""
+    rng = np.random.default_rng(31)
+    H, W, b = rng.standard_normal((60, 5)), rng.standard_normal((5, 3)), rng.standard_normal(3)
+    for act, f in (("none", lambda y: y), ("relu", lambda y: np.maximum(y, 0)), ("elu", lambda y: np.where(y > 0, y, np.expm1(y)))):
+        lay = L("dense", act, W, b)
+        assert np.allclose(O.dense_layer(H, lay), f(H @ W + b), rtol=1e-13, atol=1e-13)
+        rows = np.array([7, 3, 3, 59])
+        assert np.array_equal(O.dense_layer(H, lay, rows=rows), O.dense_layer(H, lay)[rows])
+        # through the layer dispatcher the graph is ignored
+        ip, ix = random_graph(rng, 60, 4)
+        assert np.array_equal(O.layer_forward(ip, ix, None, H, lay), O.dense_layer(H, lay))
+    # a transposed weight matrix would not even have the right shape; a dropped bias is caught here
+    assert not np.allclose(O.dense_layer(H, L("dense", "none", W, None)), H @ W + b)
+
+
+def test_gcn_layer_is_normalised_adjacency_times_h_times_w():
+    """GCN: act(A_hat H W + b) with the normalisation carried by the edge weights and self loops as edges;
+    against the dense matrix product, and the textbook facts that a row-stochastic A_hat keeps constant
+    features constant and that the symmetric normalisation of an undirected graph gives a symmetric A_hat."""
+    rng = np.random.default_rng(32)
+    n, Fi, Fo = 40, 5, 3
+    ip, ix = random_graph(rng, n, 6)
+    w = rng.random(ix.shape[0])
+    H, W, b = rng.standard_normal((n, Fi)), rng.standard_normal((Fi, Fo)), rng.standard_normal(Fo)
+    lay = L("gcn", "relu", W, b, use_edge_weights=True)
+    A = dense_adjacency(ip, ix, w, n)
+    want = np.maximum(A @ H @ W + b, 0)
+    assert np.allclose(O.gcn_layer(ip, ix, w, H, lay), want, rtol=1e-12, atol=1e-12)
+    assert np.allclose(O.gcn_layer(ip, ix, w, H, lay, reorder=True), want, rtol=1e-12, atol=1e-12)
+    assert np.allclose(O.gcn_layer(ip, ix, w, H, lay, threshold=2), want, rtol=1e-12, atol=1e-12)
+    rows = np.array([5, 0, 39, 17])
+    assert np.allclose(O.gcn_layer(ip, ix, w, H, lay, rows=rows), want[rows], rtol=1e-12, atol=1e-12)
+    assert np.allclose(O.gcn_layer(ip, ix, w, H, lay, rows=rows, reorder=True), want[rows], rtol=1e-12, atol=1e-12)
+    # the vertex's own state enters only through a self-loop edge: no hidden self term
+    lone = L("gcn", "none", np.eye(Fi), None, use_edge_weights=False)
+    deg = np.diff(ip)
+    assert np.all(O.gcn_layer(ip, ix, None, H, lone)[deg == 0] == 0)
+    # row-stochastic weights (1 / in-degree): constant features stay constant where there is an in-edge
+    wrow = np.repeat(1.0 / np.maximum(deg, 1), deg)
+    const = np.full((n, Fi), 1.5)
+    out = O.gcn_layer(ip, ix, wrow, const, L("gcn", "none", np.eye(Fi), None, use_edge_weights=True))
+    assert np.allclose(out[deg > 0], 1.5, rtol=1e-14) and np.all(out[deg == 0] == 0)
+    # symmetric normalisation of an undirected ring with self loops: A_hat = (A + I) / 3, symmetric
+    m = 12
+    src = np.array([[(v - 1) % m, v, (v + 1) % m] for v in range(m)]).ravel().astype(np.int32)
+    rip = np.arange(0, 3 * m + 1, 3, dtype=np.int64)
+    wsym = np.full(3 * m, 1.0 / 3.0)     # 1 / sqrt(d_u d_v) with d = 3 everywhere
+    X = rng.standard_normal((m, 2))
+    out = O.gcn_layer(rip, src, wsym, X, L("gcn", "none", np.eye(2), None, use_edge_weights=True))
+    assert np.allclose(out, (np.roll(X, 1, 0) + X + np.roll(X, -1, 0)) / 3.0, rtol=1e-14, atol=1e-14)
+
+
 def test_linear_and_activations_against_numpy():
     rng = np.random.default_rng(13)
     X, W, b = rng.standard_normal((40, 7)), rng.standard_normal((7, 5)), rng.standard_normal(5)
@@ -466,6 +519,7 @@ def test_reorder_is_algebraically_equal():
     with pytest.raises(ValueError):
         O.sage_layer(ip, ix, w, H, L("max", "relu", rng.standard_normal((16, 3))), reorder=True)
     assert O.will_reorder(L("sum", W=np.zeros((16, 3)))) and not O.will_reorder(L("max", W=np.zeros((16, 3))))
+    assert O.will_reorder(L("gcn", W=np.zeros((8, 3)))) and not O.will_reorder(L("dense", W=np.zeros((8, 3))))
     assert not O.will_reorder(L("sum", W=np.zeros((16, 8)))) and not O.will_reorder(L("sum", W=np.zeros((16, 3)), allow_reorder=False))
 
 
