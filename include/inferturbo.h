@@ -41,7 +41,11 @@ typedef enum {
 
 typedef enum { IT_F32 = 0, IT_BF16 = 1 } it_dtype;
 typedef enum { IT_I32 = 0, IT_I64 = 1 } it_itype;
-typedef enum { IT_GATHER_SUM = 0, IT_GATHER_MEAN = 1, IT_GATHER_MAX = 2, IT_GATHER_GAT = 3, IT_GATHER_MIN = 4 } it_gather_op;
+typedef enum {
+  IT_GATHER_SUM = 0, IT_GATHER_MEAN = 1, IT_GATHER_MAX = 2, IT_GATHER_GAT = 3, IT_GATHER_MIN = 4,
+  IT_GATHER_NONE = 5,   /* no Gather stage: a dense layer */
+  IT_GATHER_GCN = 6     /* sum aggregate, update on the aggregate alone */
+} it_gather_op;
 typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
 
 #define IT_MAX_BUCKETS 8
@@ -62,6 +66,13 @@ typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
  *     h'_v = act( concat_k sum_e softmax_e(e) z_u^k + bias )
  *   The message-passing form is Eq. (1); the paper places GAT's reduce in apply_node
  *   because attention is not associative.
+ *
+ * Dense (op = NONE): h'_v = act( h_v * W + bias ), W is [in_dim, out_dim].  The paper's first superstep
+ *   (raw vertex states -> initial embeddings) and the prediction part attached after the last
+ *   apply_node (Section "Implementation on Pregel") are layers of this kind.
+ * GCN (op = GCN): a_v = sum_e w_e * h_u (w_e = 1 without edge weights), h'_v = act( a_v * W + bias ),
+ *   W is [in_dim, out_dim].  The degree normalisation is carried by the edge weights and a self loop is
+ *   an edge of the graph like any other; the vertex's own state enters in no other way.
  *
  * Storage contract: h_in, h_out (and the internal Z / aggregate tensors) are feat_dtype,
  * rounded to nearest even when written; all accumulation is fp32.  W is weight_dtype and
@@ -140,7 +151,7 @@ it_status it_workspace_bytes(const it_graph *g, const it_layer_desc *layers, int
  * the next layer reads ("scatter": on one device sending along out-edges is a store).
  *   h_in  [n, in_dim], h_out [n, out_dim], feat_dtype, device, must not overlap.
  *   workspace: device, 256-byte aligned, >= it_workspace_bytes(g, layer, 1).
- * If allow_reorder and op is SUM or MEAN and out_dim < in_dim, the neighbour transform is
+ * If allow_reorder and op is SUM, MEAN or GCN and out_dim < in_dim, the neighbour transform is
  * done before the gather (the paper's "computation flow would be reorganized", Section
  * "Inference"): Z = h_in * W[in_dim:, :] is stored in feat_dtype and gathered instead of
  * h_in; the self term h_in * W[0:in_dim, :] + bias stays fp32.

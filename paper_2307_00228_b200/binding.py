@@ -19,7 +19,7 @@ STATUS_NAMES = ["IT_OK", "IT_ERR_INVALID_ARG", "IT_ERR_BAD_GRAPH", "IT_ERR_UNSUP
                 "IT_ERR_OOM", "IT_ERR_CUDA", "IT_ERR_TIMEOUT"]
 IT_F32, IT_BF16 = 0, 1
 IT_I32, IT_I64 = 0, 1
-GATHER_OPS = {"sum": 0, "mean": 1, "max": 2, "gat": 3, "min": 4}
+GATHER_OPS = {"sum": 0, "mean": 1, "max": 2, "gat": 3, "min": 4, "dense": 5, "gcn": 6}
 ACTS = {"none": 0, "relu": 1, "elu": 2}
 IT_MAX_BUCKETS = 8
 EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspace_bytes", "it_layer_forward",

@@ -6,7 +6,7 @@
 
 namespace {
 
-enum LayerPlan { PLAN_SAGE = 0, PLAN_SAGE_REORDER = 1, PLAN_GAT = 2 };
+enum LayerPlan { PLAN_SAGE = 0, PLAN_SAGE_REORDER = 1, PLAN_GAT = 2, PLAN_DENSE = 3, PLAN_GCN = 4, PLAN_GCN_REORDER = 5 };
 
 struct LayerWs {
   LayerPlan plan;
@@ -16,7 +16,7 @@ struct LayerWs {
 
 it_status check_layer(const it_graph *g, const it_layer_desc *L) {
   IT_REQUIRE(L != nullptr, IT_ERR_INVALID_ARG, "layer is NULL");
-  IT_REQUIRE(L->op >= IT_GATHER_SUM && L->op <= IT_GATHER_MIN, IT_ERR_INVALID_ARG, "bad gather op %d", (int)L->op);
+  IT_REQUIRE(L->op >= IT_GATHER_SUM && L->op <= IT_GATHER_GCN, IT_ERR_INVALID_ARG, "bad gather op %d", (int)L->op);
   IT_REQUIRE(L->act >= IT_ACT_NONE && L->act <= IT_ACT_ELU, IT_ERR_INVALID_ARG, "bad activation %d", (int)L->act);
   IT_REQUIRE(L->feat_dtype == IT_F32 || L->feat_dtype == IT_BF16, IT_ERR_INVALID_ARG, "bad feat_dtype");
   IT_REQUIRE(L->weight_dtype == L->feat_dtype, IT_ERR_UNSUPPORTED, "weight_dtype must equal feat_dtype");
@@ -30,12 +30,13 @@ it_status check_layer(const it_graph *g, const it_layer_desc *L) {
   } else {
     IT_REQUIRE(L->heads <= 1, IT_ERR_INVALID_ARG, "heads > 1 needs op = IT_GATHER_GAT");
     IT_REQUIRE(!L->use_edge_weights || g->edge_weights, IT_ERR_INVALID_ARG, "layer uses edge weights but the graph has none");
+    IT_REQUIRE(L->op != IT_GATHER_NONE || !L->use_edge_weights, IT_ERR_INVALID_ARG, "a dense layer has no edges to weight");
   }
   return IT_OK;
 }
 
 bool reorders(const it_layer_desc *L) {
-  return L->allow_reorder && (L->op == IT_GATHER_SUM || L->op == IT_GATHER_MEAN) && L->out_dim < L->in_dim;
+  return L->allow_reorder && (L->op == IT_GATHER_SUM || L->op == IT_GATHER_MEAN || L->op == IT_GATHER_GCN) && L->out_dim < L->in_dim;
 }
 
 LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
@@ -50,6 +51,23 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
     w.off_partials = take(it_gat_partial_bytes(g, L->out_dim, L->heads));
     w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
     w.off_b = take(n * fo * s);                    // Z
+  } else if (L->op == IT_GATHER_NONE) {
+    w.plan = PLAN_DENSE;
+    w.off_B = take(fi * fo * 8);
+    w.off_partials = w.off_a = w.off_b = off;
+  } else if (L->op == IT_GATHER_GCN) {
+    w.off_B = take(fi * fo * 8);
+    if (reorders(L)) {
+      w.plan = PLAN_GCN_REORDER;
+      w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
+      w.off_a = off;
+      w.off_b = take(n * fo * s);  // Z
+    } else {
+      w.plan = PLAN_GCN;
+      w.off_partials = take((size_t)g->n_partial_rows * fi * 4);
+      w.off_a = take(n * fi * s);  // A
+      w.off_b = off;
+    }
   } else if (reorders(L)) {
     w.plan = PLAN_SAGE_REORDER;
     w.off_B = take(fi * 2 * fo * 8);
@@ -110,8 +128,40 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
     return it_launch_gat(aa, st);
   }
 
+  if (w.plan == PLAN_DENSE) {   // no Gather stage: h' = act(h W + b)
+    it_gemm_args ga{};
+    ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
+    ga.B = B; ga.NB = L->out_dim;
+    ga.n0 = L->out_dim; ga.out0 = h_out; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = L->act;
+    ga.n1 = 0; ga.out1 = nullptr; ga.dt1 = dt; ga.out2 = nullptr;
+    return run_apply(g, L, IT_PREP_DENSE, ga, B, nullptr, st);
+  }
+
   it_gather_args gg{};
-  gg.g = g; gg.op = L->op; gg.use_edge_weights = L->use_edge_weights; gg.dtype = dt; gg.partials = partials;
+  gg.g = g; gg.op = L->op == IT_GATHER_GCN ? IT_GATHER_SUM : L->op; gg.use_edge_weights = L->use_edge_weights; gg.dtype = dt;
+  gg.partials = partials;
+  if (w.plan == PLAN_GCN_REORDER) {   // Z = H W, then h' = act(sum_e w_e z_u + b) in the gather's epilogue
+    void *Z = ws + w.off_b;
+    it_gemm_args ga{};
+    ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
+    ga.B = B; ga.NB = L->out_dim;
+    ga.n0 = 0; ga.out0 = nullptr; ga.dt0 = dt; ga.bias0 = nullptr; ga.act0 = IT_ACT_NONE;
+    ga.n1 = L->out_dim; ga.out1 = Z; ga.dt1 = dt; ga.out2 = nullptr;
+    IT_TRY(run_apply(g, L, IT_PREP_DENSE, ga, B, nullptr, st));
+    gg.dim = L->out_dim; gg.src = Z; gg.dst = h_out; gg.epi = IT_EPI_BIAS_ACT; gg.self_term = nullptr; gg.bias = L->bias; gg.act = L->act;
+    return it_launch_gather(gg, st);
+  }
+  if (w.plan == PLAN_GCN) {   // A = sum_e w_e h_u, then h' = act(A W + b)
+    void *A = ws + w.off_a;
+    gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.bias = nullptr; gg.act = IT_ACT_NONE;
+    IT_TRY(it_launch_gather(gg, st));
+    it_gemm_args ga{};
+    ga.M = g->n; ga.x_dtype = dt; ga.X1 = A; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
+    ga.B = B; ga.NB = L->out_dim;
+    ga.n0 = L->out_dim; ga.out0 = h_out; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = L->act;
+    ga.n1 = 0; ga.out1 = nullptr; ga.dt1 = dt; ga.out2 = nullptr;
+    return run_apply(g, L, IT_PREP_DENSE, ga, B, nullptr, st);
+  }
   if (w.plan == PLAN_SAGE_REORDER) {
     float *S = reinterpret_cast<float *>(ws + w.off_a);
     void *Z = ws + w.off_b;

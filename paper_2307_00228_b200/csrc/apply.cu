@@ -25,8 +25,8 @@ struct PrepParams {
 
 __global__ void prep_weights_kernel(PrepParams p) {
   const int fi = p.in_dim, fo = p.out_dim;
-  if (p.kind == IT_PREP_SAGE) {
-    int64_t total = (int64_t)2 * fi * fo;
+  if (p.kind == IT_PREP_SAGE || p.kind == IT_PREP_DENSE) {
+    int64_t total = (int64_t)(p.kind == IT_PREP_SAGE ? 2 : 1) * fi * fo;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x)
       p.B[i] = load_as_float(p.W, i, p.w_is_bf16);
   } else if (p.kind == IT_PREP_SAGE_REORDER) {

@@ -104,7 +104,8 @@ static inline int it_dtype_size(it_dtype t) { return t == IT_F32 ? 4 : 2; }
 // What a gather / combine kernel does with the finished aggregate of vertex v.
 enum it_epilogue_kind {
   IT_EPI_STORE = 0,      // dst[v, :] = agg                      (feat dtype)
-  IT_EPI_ADD_ACT = 1     // dst[v, :] = act(self[v, :] + agg)    (self fp32, dst feat dtype)
+  IT_EPI_ADD_ACT = 1,    // dst[v, :] = act(self[v, :] + agg)    (self fp32, dst feat dtype)
+  IT_EPI_BIAS_ACT = 2    // dst[v, :] = act(bias + agg)          (bias fp32 [dim] or NULL)
 };
 
 struct it_gather_args {
@@ -118,7 +119,8 @@ struct it_gather_args {
   void *dst;               // [n, dim]
   it_epilogue_kind epi;
   const float *self_term;  // [n, dim] fp32, IT_EPI_ADD_ACT only
-  it_act act;              // IT_EPI_ADD_ACT only
+  const float *bias;       // [dim] fp32 or NULL, IT_EPI_BIAS_ACT only
+  it_act act;              // IT_EPI_ADD_ACT and IT_EPI_BIAS_ACT
 };
 it_status it_launch_gather(const it_gather_args &a, cudaStream_t stream);
 
@@ -157,7 +159,7 @@ struct it_gemm_args {
 };
 it_status it_launch_gemm(const it_gemm_args &a, cudaStream_t stream);
 
-enum it_prep_kind { IT_PREP_SAGE = 0, IT_PREP_SAGE_REORDER = 1, IT_PREP_GAT = 2 };
+enum it_prep_kind { IT_PREP_SAGE = 0, IT_PREP_SAGE_REORDER = 1, IT_PREP_GAT = 2, IT_PREP_DENSE = 3 };   // DENSE: B = W [in, out] as it is
 // Assemble the fp32 B matrix for a layer: SAGE [2*in, out] copy; REORDER [in, 2*out] =
 // [W_self | W_neigh]; GAT [in, out + 2*heads] = [W | W a_src | W a_dst].
 it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *layer, float *B,

@@ -20,6 +20,7 @@ struct SagePolicy {
   float *__restrict__ partials;
   void *__restrict__ dst;
   const float *__restrict__ self_term;
+  const float *__restrict__ bias;
   int dim, is_mean, epi, act;
   // per-thread
   int col;
@@ -67,6 +68,9 @@ struct SagePolicy {
     if (epi == IT_EPI_ADD_ACT) {
 #pragma unroll
       for (int i = 0; i < VEC; ++i) st[i] = act_apply(st[i] + self[i], act);
+    } else if (epi == IT_EPI_BIAS_ACT) {
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) st[i] = act_apply(st[i] + (bias ? __ldg(bias + col + i) : 0.f), act);
     }
     Slice::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, st);
   }
@@ -82,6 +86,7 @@ struct CombineParams {
   const float *__restrict__ partials;
   void *__restrict__ dst;
   const float *__restrict__ self_term;
+  const float *__restrict__ bias;
   int64_t n_split_owners;
   int dim;
   int red, is_mean, epi, act;   // red: RED_SUM / RED_MAX / RED_MIN
@@ -124,6 +129,9 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
         float4 s = __ldg(reinterpret_cast<const float4 *>(p.self_term + off));
         o[0] = act_apply(o[0] + s.x, p.act); o[1] = act_apply(o[1] + s.y, p.act);
         o[2] = act_apply(o[2] + s.z, p.act); o[3] = act_apply(o[3] + s.w, p.act);
+      } else if (p.epi == IT_EPI_BIAS_ACT) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[i] = act_apply(o[i] + (p.bias ? __ldg(p.bias + c + i) : 0.f), p.act);
       }
       T *d = reinterpret_cast<T *>(p.dst) + off;
       if (sizeof(T) == 4) {
@@ -140,7 +148,7 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 template <typename T, int SB, int LPR, int RED, bool WEIGHTED>
 it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   SagePolicy<T, SB, RED, WEIGHTED> pol;
-  pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.dim = a.dim;
+  pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
   const it_graph *g = a.g;
   // algorithmic bytes: per edge the index, the optional weight and one source row; per row its
@@ -180,7 +188,7 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
   if (g->n_split_owners > 0) {
     CombineParams c;
     c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.shadow_indptr = g->shadow_indptr;
-    c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.n_split_owners = g->n_split_owners;
+    c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.bias = a.bias; c.n_split_owners = g->n_split_owners;
     c.dim = a.dim; c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
     int64_t want = (g->n_split_owners + 7) / 8;
     int64_t cap = (int64_t)g->num_sms * 8;

@@ -49,6 +49,15 @@ def make_sage_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=T
                  use_edge_weights=weights, allow_reorder=allow_reorder)
 
 
+def make_plain_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=True, bias=True) -> Layer:
+    """op = "dense" (no Gather stage) or "gcn" (update on the aggregate alone): W is [fi, fo]."""
+    rng = np.random.default_rng(seed)
+    lim = np.sqrt(6.0 / (fi + fo))
+    return Layer(op=op, act=act, in_dim=fi, out_dim=fo, W=storage_exact(rng.uniform(-lim, lim, (fi, fo)), dtype),
+                 bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None,
+                 use_edge_weights=weights, allow_reorder=allow_reorder)
+
+
 def make_gat_layer(seed, act, fi, heads, hd, dtype, bias=True) -> Layer:
     rng = np.random.default_rng(seed)
     fo = heads * hd

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import (TOL, check_against_oracle, make_gat_layer, make_sage_layer, run_device, run_oracle,
+from gpu_util import (TOL, check_against_oracle, make_gat_layer, make_plain_layer, make_sage_layer, run_device, run_oracle,
                       small_workload, to_numpy)
 from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
@@ -81,6 +81,43 @@ def test_gat_on_a_split_graph(dtype, threshold):
     check_against_oracle(w, got, label=(dtype, threshold))
     base, _ = run_device(w, threshold=0)
     assert compare.rel_error(got, base)["max_rel"] <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dims", [(64, 32), (32, 64), (128, 128), (8, 16)])
+@pytest.mark.parametrize("act", ["none", "elu"])
+def test_dense_layer_parity(dtype, dims, act):
+    """No Gather stage (initial transform / prediction part): the graph must not matter."""
+    fi, fo = dims
+    layer = make_plain_layer(40, "dense", act, fi, fo, dtype)
+    w = small_workload(41, 1300, 10, dtype, [layer], hubs=(300,), threshold=64)
+    got, _ = run_device(w)
+    check_against_oracle(w, got, label=(dtype, dims, act))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("weights", [False, True])
+@pytest.mark.parametrize("threshold", [0, 64])
+def test_gcn_layer_parity(dtype, weights, threshold):
+    for fi, fo in ((64, 32), (32, 64), (64, 64)):      # the first shape reorders (transform before aggregate)
+        for reorder in (True, False):
+            layer = make_plain_layer(42, "gcn", "relu", fi, fo, dtype, weights=weights, allow_reorder=reorder)
+            w = small_workload(43, 1500, 30, dtype, [layer], hubs=HUBS, weights=weights, threshold=threshold)
+            got, d = run_device(w)
+            check_against_oracle(w, got, label=(dtype, weights, threshold, fi, fo, reorder))
+
+
+def test_embed_gnn_predict_pipeline():
+    """Initial transform of raw features, two message-passing layers, prediction head: the k-layer GNN
+    from raw vertex states to scores in one it_infer call."""
+    for dtype in ("f32", "bf16"):
+        layers = [make_plain_layer(44, "dense", "relu", 24 if dtype == "f32" else 40, 64, dtype),
+                  make_sage_layer(45, "mean", "relu", 64, 64, dtype),
+                  make_plain_layer(46, "gcn", "relu", 64, 32, dtype, weights=True),
+                  make_plain_layer(47, "dense", "none", 32, 8, dtype)]
+        w = small_workload(48, 2500, 18, dtype, layers, hubs=HUBS, weights=True, threshold=200)
+        got, _ = run_device(w)
+        check_against_oracle(w, got, label=dtype)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
