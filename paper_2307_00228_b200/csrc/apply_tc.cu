@@ -9,8 +9,10 @@
 //   bf16 : kind::f16 with bf16 inputs, fp32 accumulation.
 //   fp32 : three kind::tf32 products per step, A = A_hi + A_lo and B = B_hi + B_lo with
 //          A_hi*B_hi + A_lo*B_hi + A_hi*B_lo (the dropped A_lo*B_lo term is ~2^-22 relative);
-//          a single TF32 pass (10-bit mantissa) would miss the 1e-4 error bound.  A is split
-//          in shared memory by four dedicated warps, B is split once by the prep kernel.
+//          a single TF32 pass (10-bit mantissa) would miss the 1e-4 error bound.  Four dedicated
+//          warps read each raw A tile from shared memory once, split it and write both parts to
+//          TMEM (tcgen05.st), so that the MMAs take A from TMEM and read only the weights from
+//          shared memory; B is split once by the prep kernel.
 //
 // Every wait on an mbarrier is bounded: when one gives up, the CTA raises a flag that all
 // roles poll, drains, frees its TMEM and returns, and a status word in global memory is set.
@@ -18,13 +20,9 @@
 
 #include "common.cuh"
 
-// fp32 mode: the tensor core ignores the low 13 mantissa bits of a tf32 operand, so the raw fp32 tile serves
-// as A_hi as it is and only A_lo = x - trunc(x) has to be written.  (Were the operand rounded instead, half
-// of the products would be off by 2^-11 relative, ten times the fp32 parity tolerance: the parity tests pin
-// this.)  Set to 1 to store the truncated hi part back over the raw tile.
-#ifndef IT_TC_REWRITE_HI
-#define IT_TC_REWRITE_HI 0
-#endif
+// fp32 mode: A_hi = x with the low 13 mantissa bits cleared (what the tensor core keeps of a tf32 operand),
+// A_lo = x - A_hi, exact in fp32.  (Were the hi part rounded instead while the lo part assumed truncation,
+// half of the products would be off by 2^-11 relative, ten times the fp32 parity tolerance.)
 
 namespace {
 
@@ -32,7 +30,13 @@ constexpr int TC_BM = 128;          // rows per tile (UMMA M)
 constexpr int TC_KBLOCK_BYTES = 128;  // one swizzle row of K per k-block
 constexpr int TC_EPI_WARPS = 16;      // four warps per TMEM lane quarter, each takes every fourth 16-column group
 constexpr int TC_THREADS_BF16 = 64 + 32 * TC_EPI_WARPS;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2-17 epilogue
-constexpr int TC_THREADS_TF32 = TC_THREADS_BF16 + 128;    // ... plus four warps splitting A into hi / lo
+#ifndef IT_TC_SPLIT_GROUPS
+#define IT_TC_SPLIT_GROUPS 1   // groups of four split warps; group g takes every k-block c with c % groups == g (measured: a second group gains nothing)
+#endif
+constexpr int TC_SPLIT_GROUPS = IT_TC_SPLIT_GROUPS;
+constexpr int TC_THREADS_TF32 = TC_THREADS_BF16 + 128 * TC_SPLIT_GROUPS;   // ... plus the warps splitting A into hi / lo
+constexpr int TC_TSTAGES_MAX = 4;     // fp32 mode: split A tiles in flight in TMEM
+constexpr int TC_TSTAGE_COLS = 64;    // TMEM columns of one split A k-block: 32 of hi, 32 of lo
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -59,9 +63,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false if the CTA is aborting (or this wait ran out and started the abort).
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+// `backoff_ns` > 0: sleep between polls, for roles whose waits are long and off the critical path (their polling
+// would otherwise take issue slots from the warps that feed the tensor core).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t backoff_ns = 0) {
   for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (backoff_ns) __nanosleep(backoff_ns);
     if ((it & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -103,6 +110,23 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         : "memory");
   }
 }
+// The same product with the A operand in tensor memory (lane = row of the tile, one 32-bit column per tf32 element).
+__device__ __forceinline__ void tc_mma_tf32_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// Lane i of the warp writes 16 consecutive 32-bit columns of TMEM lane (lane base of taddr) + i.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -127,6 +151,7 @@ struct TcParams {
   int kb1, kb2;                   // k-blocks that come from X1 / X2
   int NB;                         // total columns
   int stages;
+  int tstages;                    // fp32 mode: split A k-blocks in flight in TMEM
   // epilogue routing (columns are global column ids)
   int n0; void *out0; int out0_bf16; const float *bias0; int act0;
   int n1; void *out1; int out1_bf16;
@@ -145,20 +170,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   const int b_bytes = (TF32 ? 2 : 1) * KB * b_tile_bytes;
   constexpr int a_tile_bytes = TC_BM * TC_KBLOCK_BYTES;          // 16 KB
 
-  // shared memory: resident weights | operand stages (raw / hi tiles) | fp32 mode: two lo tiles | barriers
+  // shared memory: resident weights | operand stages (bf16 tiles the MMAs read, or raw fp32 tiles the split warps read) | barriers
   unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char *smem_b = base;
   unsigned char *smem_a = base + b_bytes;   // b_bytes is a multiple of 1024 (nbc is a multiple of 16)
-  unsigned char *smem_lo = smem_a + (size_t)p.stages * a_tile_bytes;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_lo + (TF32 ? 2 * a_tile_bytes : 0));
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_a + (size_t)p.stages * a_tile_bytes);
   uint64_t *full = bars;                    // [stages]  TMA landed
-  uint64_t *empty = bars + p.stages;        // [stages]  MMAs that read the stage are done
-  uint64_t *ready = bars + 2 * p.stages;    // [stages]  (fp32 mode) hi / lo split written
-  uint64_t *b_full = bars + 3 * p.stages;   // [1]
+  uint64_t *empty = bars + p.stages;        // [stages]  the stage's readers are done (bf16: its MMAs; fp32: the split warps)
+  uint64_t *ready = bars + 2 * p.stages;    // [TC_TSTAGES_MAX]  (fp32 mode) hi / lo parts written to TMEM
+  uint64_t *a_free = ready + TC_TSTAGES_MAX;   // [TC_TSTAGES_MAX]  (fp32 mode) MMAs that read a TMEM stage are done
+  uint64_t *b_full = a_free + TC_TSTAGES_MAX;  // [1]
   uint64_t *acc_full = b_full + 1;          // [2]
   uint64_t *acc_empty = acc_full + 2;       // [2]
-  uint64_t *lo_free = acc_empty + 2;        // [2]  (fp32 mode) MMAs that read a lo tile are done
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(lo_free + 2);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   // per-column constants of this CTA's columns, 16-byte aligned: bias (0 where none applies), GAT attention vectors
   float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // [nbc]
@@ -166,20 +190,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
 
   // fp32 mode: columns [nbc, 2 nbc) of an accumulator hold A_hi * B_lo, added to the first half by the epilogue
   const uint32_t acc_cols = (uint32_t)p.nbc * (TF32 ? 2u : 1u);
+  const uint32_t a_col0 = 2 * acc_cols;   // fp32 mode: the split A stages follow the two accumulators
   uint32_t tmem_cols = 32;
-  while (tmem_cols < 2 * acc_cols) tmem_cols <<= 1;
+  while (tmem_cols < 2 * acc_cols + (TF32 ? (uint32_t)p.tstages * TC_TSTAGE_COLS : 0u)) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], 1);
+      mbar_init(&empty[s], TF32 ? 4 : 1);
+    }
+    for (int s = 0; s < TC_TSTAGES_MAX; ++s) {
       mbar_init(&ready[s], 4);
+      mbar_init(&a_free[s], 1);
     }
     mbar_init(b_full, 1);
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], TC_EPI_WARPS);
-      mbar_init(&lo_free[a], 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -222,7 +249,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile / p.n_splits) * TC_BM;
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag);
+          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, 64);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[stage], (uint32_t)a_tile_bytes);
           if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x1, kb * bk_elems, m0, &full[stage]);
@@ -247,34 +274,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       bool ok = mbar_wait(b_full, 0, abort_flag);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
-      uint32_t lo = 0;
-      uint64_t *const wait_bar = TF32 ? ready : full;
+      uint32_t ts = 0, tphase = 0;   // fp32 mode: TMEM stage of the split A k-block
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * acc_cols;
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(&wait_bar[stage], phase, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t a_hi = smem_u32(smem_a + (size_t)stage * a_tile_bytes);
           const uint32_t b_hi = smem_u32(smem_b + (size_t)kb * (TF32 ? 2 : 1) * b_tile_bytes);
+          if (TF32) {
+            ok = mbar_wait(&ready[ts], tphase, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_hi = tmem_base + a_col0 + ts * TC_TSTAGE_COLS, a_lo = a_hi + 32;
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {   // four 32-byte K steps inside the 128-byte swizzle row
-            const uint32_t first = (kb | k) != 0;
-            if (TF32) {
-              // A_hi * [B_hi | B_lo] in one instruction (A_hi is read once), then A_lo * B_hi onto the first half
-              const uint32_t a_lo = smem_u32(smem_lo + (size_t)lo * a_tile_bytes);
-              tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc_wide, first);
-              tc_mma<TF32>(d_tmem, make_desc(a_lo + k * 32), make_desc(b_hi + k * 32), idesc, 1u);
-            } else {
-              tc_mma<TF32>(d_tmem, make_desc(a_hi + k * 32), make_desc(b_hi + k * 32), idesc, first);
+            for (int k = 0; k < 4; ++k) {   // four K steps of 8 tf32 elements: 8 TMEM columns of A, 32 bytes of a B row
+              // A_hi * [B_hi | B_lo] in one instruction, then A_lo * B_hi onto the first half
+              tc_mma_tf32_tmem_a(d_tmem, a_hi + k * 8, make_desc(b_hi + k * 32), idesc_wide, (kb | k) != 0);
+              tc_mma_tf32_tmem_a(d_tmem, a_lo + k * 8, make_desc(b_hi + k * 32), idesc, 1u);
             }
+            tc_commit(&a_free[ts]);   // TMEM stage reusable once these MMAs have read it
+            if (++ts == (uint32_t)p.tstages) { ts = 0; tphase ^= 1u; }
+          } else {
+            ok = mbar_wait(&full[stage], phase, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_s = smem_u32(smem_a + (size_t)stage * a_tile_bytes);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)   // four 32-byte K steps inside the 128-byte swizzle row
+              tc_mma<TF32>(d_tmem, make_desc(a_s + k * 32), make_desc(b_hi + k * 32), idesc, (kb | k) != 0);
+            tc_commit(&empty[stage]);   // stage reusable once these MMAs have read it
+            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
           }
-          tc_commit(&empty[stage]);   // stage reusable once these MMAs have read it
-          if (TF32) { tc_commit(&lo_free[lo]); lo ^= 1u; }
-          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         tc_commit(&acc_full[acc]);    // accumulator complete
@@ -299,7 +330,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const int64_t m = (int64_t)(tile / p.n_splits) * TC_BM + row_in_tile;
       const int64_t m_even = m - (odd ? 1 : 0), m_odd = m_even + 1;   // the two rows a lane pair writes together
-      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
+      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, 128);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -432,36 +463,64 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   } else {
-    // ------------------------------------------------------------------ fp32 mode: split A into hi + lo
+    // ------------------------------------------------------------------ fp32 mode: split A into hi + lo, into TMEM
+    // Thread = one row of the tile (TMEM lane quarter = warp index % 4).  The row's 128 bytes of the k-block are
+    // eight 16-byte chunks, chunk c stored at position c ^ (row % 8) by the 128-byte swizzle of the TMA copy.
     if (TF32) {
-      const int tid = threadIdx.x - TC_THREADS_BF16;   // 0..127
+      const int row = (warp & 3) * 32 + lane;
+      const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + a_col0;
+      const uint32_t group = (uint32_t)(warp - (TC_THREADS_BF16 >> 5)) >> 2;
       uint32_t stage = 0, phase = 0;
-      uint32_t lo = 0, lo_phase = 0;
+      uint32_t ts = 0, tphase = 0;
+      uint32_t c = 0;   // k-blocks since the start of the CTA
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(&full[stage], phase, abort_flag) && mbar_wait(&lo_free[lo], lo_phase ^ 1u, abort_flag);
+        for (int kb = 0; kb < KB; ++kb, ++c) {
+          if (c % TC_SPLIT_GROUPS != group) {   // another group's k-block: only keep the ring positions in step
+            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+            if (++ts == (uint32_t)p.tstages) { ts = 0; tphase ^= 1u; }
+            continue;
+          }
+          ok = mbar_wait(&full[stage], phase, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          float4 *hi_t = reinterpret_cast<float4 *>(smem_a + (size_t)stage * a_tile_bytes);
-          float4 *lo_t = reinterpret_cast<float4 *>(smem_lo + (size_t)lo * a_tile_bytes);
+          const unsigned char *row_base = smem_a + (size_t)stage * a_tile_bytes + (size_t)row * TC_KBLOCK_BYTES;
+          float4 x[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {   // 1024 float4 per tile, 128 threads
-            const int i = tid + j * 128;
-            const float4 x = hi_t[i];
-            float4 h, l;
-            h.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); l.x = x.x - h.x;
-            h.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u); l.y = x.y - h.y;
-            h.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); l.z = x.z - h.z;
-            h.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u); l.w = x.w - h.w;
-            if (IT_TC_REWRITE_HI) hi_t[i] = h;
-            lo_t[i] = l;
+          for (int c = 0; c < 8; ++c) x[c] = *reinterpret_cast<const float4 *>(row_base + ((c ^ (row & 7)) << 4));
+          ok = mbar_wait(&a_free[ts], tphase ^ 1u, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t t_hi = t_lane + ts * TC_TSTAGE_COLS, t_lo = t_hi + 32;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t h[16], l[16];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float4 v = x[half * 4 + c];
+              const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t hb = __float_as_uint(e[i]) & 0xffffe000u;
+                h[c * 4 + i] = hb;
+                l[c * 4 + i] = __float_as_uint(e[i] - __uint_as_float(hb));
+              }
+            }
+            tmem_st16(t_hi + half * 16, h);
+            tmem_st16(t_lo + half * 16, l);
           }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
+          // Every value read from the stage has been used, so the reads are complete; the proxy fence orders these
+          // generic-proxy reads before the asynchronous-proxy write of the TMA copy that refills the stage.
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
-          if (lane == 0) mbar_arrive(&ready[stage]);
+          if (lane == 0) mbar_arrive(&empty[stage]);
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
-          if (++lo == 2) { lo = 0; lo_phase ^= 1u; }
+          tmem_st_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&ready[ts]);
+          if (++ts == (uint32_t)p.tstages) { ts = 0; tphase ^= 1u; }
         }
       }
     }
@@ -552,7 +611,8 @@ static bool tc_split(bool tf32, int NB, int KB, int *n_splits, int *nbc) {
   for (int s = 1; s <= 16; ++s) {
     if (NB % s != 0) continue;
     const int c = NB / s;
-    if (c % 16 != 0 || c > (tf32 ? 128 : 256)) continue;   // fp32 mode issues MMAs of 2 c columns and keeps 4 c TMEM columns
+    // fp32 mode issues MMAs of 2 c columns and keeps 4 c TMEM columns of accumulators next to the split A stages
+    if (c % 16 != 0 || c > (tf32 ? 64 : 256)) continue;
     if ((size_t)(tf32 ? 2 : 1) * KB * c * TC_KBLOCK_BYTES > 128 * 1024) continue;
     *n_splits = s; *nbc = c;
     return true;
@@ -599,13 +659,16 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   int n_splits = 1, nbc = NB;
   IT_REQUIRE(tc_split(tf32, NB, KB, &n_splits, &nbc), IT_ERR_UNSUPPORTED, "tensor-core apply: cannot tile %d columns with K = %d", NB, K);
   const int b_bytes = (tf32 ? 2 : 1) * KB * nbc * TC_KBLOCK_BYTES;
-  const int stage_bytes = TC_BM * TC_KBLOCK_BYTES;             // one raw / hi operand tile
-  const int lo_bytes = tf32 ? 2 * stage_bytes : 0;             // fp32 mode: two lo tiles shared by all stages
+  const int stage_bytes = TC_BM * TC_KBLOCK_BYTES;             // one operand tile (fp32 mode: the raw tile)
   const int const_bytes = nbc * 4 * (scores ? 3 : 1);          // bias (+ attention vectors) of this CTA's columns
-  int stages = (kSmemBudget - kSmemAux - const_bytes - b_bytes - lo_bytes) / stage_bytes;
+  int stages = (kSmemBudget - kSmemAux - const_bytes - b_bytes) / stage_bytes;
   if (stages > 8) stages = 8;
   IT_REQUIRE(stages >= 2, IT_ERR_UNSUPPORTED, "tensor-core apply: no room for two operand stages");
-  const int smem = b_bytes + stages * stage_bytes + lo_bytes + kSmemAux + const_bytes;
+  const int smem = b_bytes + stages * stage_bytes + kSmemAux + const_bytes;
+  // fp32 mode: TMEM holds two accumulators of 2 nbc columns; what is left of its 512 columns stages the split A
+  int tstages = tf32 ? (512 - 4 * nbc) / TC_TSTAGE_COLS : 0;
+  if (tstages > TC_TSTAGES_MAX) tstages = TC_TSTAGES_MAX;
+  IT_REQUIRE(!tf32 || tstages >= 2, IT_ERR_UNSUPPORTED, "tensor-core apply: no room in TMEM for two split A stages");
 
   CUtensorMap m1, m2, mb;
   IT_TRY(make_map(&m1, a.X1, elem, a.M, a.K1, TC_BM));
@@ -615,7 +678,7 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
 
   TcParams p;
   p.M = a.M; p.n_tiles_m = (int)((a.M + TC_BM - 1) / TC_BM); p.n_splits = n_splits; p.nbc = nbc;
-  p.kb1 = a.K1 / bk; p.kb2 = K2 / bk; p.NB = NB; p.stages = stages;
+  p.kb1 = a.K1 / bk; p.kb2 = K2 / bk; p.NB = NB; p.stages = stages; p.tstages = tstages;
   p.n0 = a.n0; p.out0 = a.out0; p.out0_bf16 = a.dt0 == IT_BF16; p.bias0 = a.bias0; p.act0 = a.act0;
   p.n1 = a.n1; p.out1 = a.out1; p.out1_bf16 = a.dt1 == IT_BF16;
   p.scores = scores; p.att_src = att_src; p.att_dst = att_dst; p.heads = heads; p.head_dim = head_dim > 0 ? head_dim : 1;
