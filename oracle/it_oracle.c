@@ -133,6 +133,32 @@ void ito_aggregate(int64_t n, const int64_t *indptr, const int32_t *indices, con
     }
 }
 
+/* aggregate of the edge features themselves (Eq. (1): the message function M may read the feature vector
+ * e_{v,u} of the edge; here that part of the message is e_{v,u} as it is).  EF is [n_edges, De] row-major,
+ * row j belonging to CSR entry j, so the in-edges of v own the consecutive rows indptr[v] .. indptr[v+1]-1:
+ *   sum : ae_v    = sum_j e_j          mean: divided by the number of in-edges
+ *   max : ae_v[f] = max_j e_j[f]       min : ae_v[f] = min_j e_j[f]
+ * An empty in-neighbourhood gives 0.  `segptr` may also be the shadow-row pointer (partial results per group;
+ * pass SUM for a mean then).  AE is [n_seg, De]. */
+void ito_aggregate_edges(int64_t n_seg, const int64_t *segptr, const double *EF, int32_t De, int32_t op, double *AE) {
+#pragma omp parallel for schedule(dynamic, 256)
+    for (int64_t v = 0; v < n_seg; ++v) {
+        double *a = AE + v * De;
+        int64_t j0 = segptr[v], j1 = segptr[v + 1];
+        for (int32_t f = 0; f < De; ++f) a[f] = 0.0;
+        for (int64_t j = j0; j < j1; ++j) {
+            const double *e = EF + j * De;
+            for (int32_t f = 0; f < De; ++f) {
+                if (op == ITO_MAX) a[f] = (j == j0 || e[f] > a[f]) ? e[f] : a[f];
+                else if (op == ITO_MIN) a[f] = (j == j0 || e[f] < a[f]) ? e[f] : a[f];
+                else a[f] += e[f];
+            }
+        }
+        if (op == ITO_MEAN && j1 > j0)
+            for (int32_t f = 0; f < De; ++f) a[f] /= (double)(j1 - j0);
+    }
+}
+
 /* Partial gather: the same aggregate, but per shadow row (one group of a vertex's
  * in-edges).  Mean rows hold plain sums; the division happens once, in combine.
  * P is [R, F]. */

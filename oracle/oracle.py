@@ -161,6 +161,15 @@ def combine(owner_indptr, indptr, P, op: str):
     return A
 
 
+def aggregate_edges(segptr, EF, op: str):
+    """Reduce of the edge-feature rows of every segment (in-edges of a vertex, or one shadow row)."""
+    segptr, EF = _i64(segptr), _f64(EF)
+    n, De = segptr.shape[0] - 1, EF.shape[1]
+    AE = np.empty((n, De), np.float64)
+    lib().ito_aggregate_edges(C.c_int64(n), _p(segptr), _p(EF), C.c_int32(De), C.c_int32(OPS[op]), _p(AE))
+    return AE
+
+
 def linear(X, W):
     X, W = _f64(X), _f64(W)
     out = np.empty((X.shape[0], W.shape[1]), np.float64)
@@ -204,15 +213,17 @@ def gat_aggregate(indptr, indices, Z, s_src, s_dst, heads: int, slope: float):
 
 # ----------------------------------------------------------------- layers
 
-def _sub_csr(indptr, indices, w, rows):
-    """CSR restricted to the destination vertices `rows` (source ids stay global)."""
+def _sub_csr(indptr, indices, w, rows, ef=None):
+    """CSR restricted to the destination vertices `rows` (source ids stay global).  With `ef` (edge features,
+    one row per CSR entry) the matching rows are returned as a fourth value."""
     indptr = _i64(indptr)
     rows = _i64(rows)
     deg = indptr[rows + 1] - indptr[rows]
     sub = np.zeros(rows.shape[0] + 1, np.int64)
     np.cumsum(deg, out=sub[1:])
     pos = np.repeat(indptr[rows] - sub[:-1], deg) + np.arange(sub[-1], dtype=np.int64)
-    return sub, _i32(indices)[pos], (None if w is None else np.asarray(w)[pos])
+    out = (sub, _i32(indices)[pos], (None if w is None else np.asarray(w)[pos]))
+    return out if ef is None else out + (np.asarray(ef)[pos],)
 
 
 def _gathered(indptr, indices, w, H, op, threshold):
@@ -224,28 +235,57 @@ def _gathered(indptr, indices, w, H, op, threshold):
     return aggregate(indptr, indices, w, H, op)
 
 
+def _gathered_edges(indptr, EF, op, threshold):
+    """The edge-feature part of the aggregate, optionally through shadow rows + combine."""
+    if threshold and threshold > 0:
+        sp, _, owner = split_hubs(indptr, threshold)
+        return combine(owner, indptr, aggregate_edges(sp, EF, "sum" if op == "mean" else op), op)
+    return aggregate_edges(indptr, EF, op)
+
+
+def _edge_dim(layer) -> int:
+    return int(getattr(layer, "edge_dim", 0) or 0)
+
+
 def _sources_of(indptr, indices, rows):
     """Sorted unique vertex ids that `rows` read: themselves and their in-neighbours."""
     sub, idx, _ = _sub_csr(indptr, indices, None, rows)
     return np.union1d(_i64(rows), idx.astype(np.int64))
 
 
-def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
+def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None,
+               edge_feat=None):
     """One GraphSAGE layer.  `layer` has op, act, in_dim, out_dim, W [2*in, out], bias,
     use_edge_weights.  reorder=True evaluates the algebraically equal transform-before-
     aggregate form (sum and mean only): gather Z = H W_neigh instead of H.
     rows=None: every vertex.  rows=array: only those destination vertices (H is still indexed
     by global vertex id; rows of H that they do not read are never touched); returns
-    [len(rows), out]."""
+    [len(rows), out].
+    layer.edge_dim > 0: the message is [w_e h_u | e_vu] (Eq. (1): M reads the edge features too), reduced
+    entry by entry, and W has in_dim + edge_dim neighbour rows: [2*in + edge_dim, out].  Not reordered."""
     H = _f64(H)
     W = _f64(layer.W)
     Fi = layer.in_dim
+    De = _edge_dim(layer)
     w = edge_weights if layer.use_edge_weights else None
+    ef = _f64(edge_feat) if De else None
     if rows is None:
         Hself = H
+    elif De:
+        indptr, indices, w, ef = _sub_csr(indptr, indices, w, rows, ef)
+        Hself = H[_i64(rows)]
     else:
         indptr, indices, w = _sub_csr(indptr, indices, w, rows)
         Hself = H[_i64(rows)]
+    if De:
+        if reorder:
+            raise ValueError("layers with edge features keep the plain order")
+        assert ef.shape[1] == De and W.shape[0] == 2 * Fi + De
+        A = np.concatenate([_gathered(indptr, indices, w, H, layer.op, threshold),
+                            _gathered_edges(indptr, ef, layer.op, threshold)], axis=1)
+        A = round_to(A, storage)
+        out = bias_act(linear(Hself, W[:Fi]) + linear(A, W[Fi:]), layer.bias, layer.act)
+        return round_to(out, storage)
     if reorder:
         if layer.op in ("max", "min"):
             raise ValueError("transform-before-aggregate is not valid for max or min")
@@ -300,7 +340,8 @@ def dense_layer(H, layer, storage=None, rows=None):
     return round_to(bias_act(linear(H, _f64(layer.W)), layer.bias, layer.act), storage)
 
 
-def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
+def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None,
+              edge_feat=None):
     """GCN in the message-passing form of Eq. (1): the message is the source state (times the edge weight,
     which carries the degree normalisation; self loops are edges of the graph), the reduce is a sum, and
     the update is dense on the aggregate alone: h'_v = act((sum_e w_e h_u) W + b), W [in, out].
@@ -308,6 +349,16 @@ def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0
     H = _f64(H)
     W = _f64(layer.W)
     w = edge_weights if layer.use_edge_weights else None
+    De = _edge_dim(layer)
+    if De:   # message [w_e h_u | e_vu], summed; W is [in + edge_dim, out]
+        if reorder:
+            raise ValueError("layers with edge features keep the plain order")
+        ef = _f64(edge_feat)
+        if rows is not None:
+            indptr, indices, w, ef = _sub_csr(indptr, indices, w, rows, ef)
+        A = np.concatenate([_gathered(indptr, indices, w, H, "sum", threshold),
+                            _gathered_edges(indptr, ef, "sum", threshold)], axis=1)
+        return round_to(bias_act(linear(round_to(A, storage), W), layer.bias, layer.act), storage)
     if rows is not None:
         indptr, indices, w = _sub_csr(indptr, indices, w, rows)
     if reorder:
@@ -324,34 +375,37 @@ def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0
     return round_to(out, storage)
 
 
-def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None):
+def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None,
+                  edge_feat=None):
     if layer.op == "gat":
         return gat_layer(indptr, indices, H, layer, storage, rows)
     if layer.op == "dense":
         return dense_layer(H, layer, storage, rows)
     if layer.op == "gcn":
-        return gcn_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows)
-    return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows)
+        return gcn_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows, edge_feat)
+    return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows, edge_feat)
 
 
 def will_reorder(layer) -> bool:
     """The layer contract: transform first when it shrinks the rows that are gathered and
     the aggregate is linear."""
-    return bool(layer.allow_reorder) and layer.op in ("sum", "mean", "gcn") and layer.out_dim < layer.in_dim
+    return (bool(layer.allow_reorder) and layer.op in ("sum", "mean", "gcn") and layer.out_dim < layer.in_dim
+            and _edge_dim(layer) == 0)
 
 
-def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, follow_reorder=False):
+def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, follow_reorder=False, edge_feat=None):
     """L layers in order over the whole graph; returns the list of every layer's output."""
     H = _f64(X)
     outs = []
     for layer in layers:
         H = layer_forward(indptr, indices, edge_weights, H, layer, storage, threshold,
-                          reorder=follow_reorder and will_reorder(layer))
+                          reorder=follow_reorder and will_reorder(layer), edge_feat=edge_feat)
         outs.append(H)
     return outs
 
 
-def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, threshold=0, follow_reorder=False):
+def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, threshold=0, follow_reorder=False,
+             edge_feat=None):
     """The L-layer result at the vertices `targets` only, computed from their L-hop
     in-neighbourhood (which is sufficient and necessary for an L-layer model, Section
     "K-hop Neighborhood and Sampling"): layer l is evaluated only where layer l+1 reads it.
@@ -366,24 +420,29 @@ def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, th
     n = H.shape[0]
     for l, layer in enumerate(layers, start=1):
         out_rows = layer_forward(indptr, indices, edge_weights, H, layer, storage, threshold,
-                                 reorder=follow_reorder and will_reorder(layer), rows=need[l])
+                                 reorder=follow_reorder and will_reorder(layer), rows=need[l], edge_feat=edge_feat)
         H = np.full((n, layer.out_dim), np.nan)
         H[need[l]] = out_rows
     return H[targets]
 
 
-def compact_neighbourhood(indptr, indices, edge_weights, targets, n_layers):
+def compact_neighbourhood(indptr, indices, edge_weights, targets, n_layers, edge_feat=None):
     """The part of the graph an n_layers-layer model reads to produce `targets`, relabelled to
     consecutive ids so that huge graphs can be checked without full-size fp64 arrays.
     Returns (vertex_ids, c_indptr, c_indices, c_weights, c_targets): vertex_ids are the global
     ids (sorted) of the compact vertices; a compact vertex keeps its in-edges only if some layer
-    output of it is needed (the others are read as layer-0 inputs only)."""
+    output of it is needed (the others are read as layer-0 inputs only).  With `edge_feat` the rows of
+    the kept edges are appended as a sixth value."""
     targets = _i64(targets)
     need = np.unique(targets)
     for _ in range(n_layers - 1):
         need = _sources_of(indptr, indices, need)          # where layer 1 .. L-1 outputs are needed
     ids = _sources_of(indptr, indices, need)               # plus the layer-0 inputs they read
-    sub, idx, w = _sub_csr(indptr, indices, edge_weights, need)
+    if edge_feat is None:
+        sub, idx, w = _sub_csr(indptr, indices, edge_weights, need)
+        ef = None
+    else:
+        sub, idx, w, ef = _sub_csr(indptr, indices, edge_weights, need, edge_feat)
     deg = np.zeros(ids.shape[0], np.int64)
     pos_need = np.searchsorted(ids, need)
     deg[pos_need] = np.diff(sub)
@@ -391,4 +450,5 @@ def compact_neighbourhood(indptr, indices, edge_weights, targets, n_layers):
     np.cumsum(deg, out=c_indptr[1:])
     # rows of `need` are ascending in both numberings, so the concatenated edge lists keep their order
     c_indices = np.searchsorted(ids, idx.astype(np.int64)).astype(np.int32)
-    return ids, c_indptr, c_indices, w, np.searchsorted(ids, targets)
+    out = (ids, c_indptr, c_indices, w, np.searchsorted(ids, targets))
+    return out if edge_feat is None else out + (ef,)

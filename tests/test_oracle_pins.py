@@ -15,10 +15,10 @@ GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "w5.json
 
 
 def L(op="sum", act="none", W=None, bias=None, heads=1, att_src=None, att_dst=None, slope=0.2,
-      use_edge_weights=False, allow_reorder=True):
+      use_edge_weights=False, allow_reorder=True, edge_dim=0):
     W = np.asarray(W, dtype=np.float64)
-    in_dim = W.shape[0] if op in ("gat", "dense", "gcn") else W.shape[0] // 2
-    return NS(op=op, act=act, in_dim=in_dim, out_dim=W.shape[1], W=W,
+    in_dim = (W.shape[0] - edge_dim) if op in ("gat", "dense", "gcn") else (W.shape[0] - edge_dim) // 2
+    return NS(op=op, act=act, in_dim=in_dim, out_dim=W.shape[1], W=W, edge_dim=edge_dim,
               bias=None if bias is None else np.asarray(bias, dtype=np.float64), heads=heads,
               att_src=None if att_src is None else np.asarray(att_src, dtype=np.float64),
               att_dst=None if att_dst is None else np.asarray(att_dst, dtype=np.float64),
@@ -99,15 +99,15 @@ def py_act(x, act):
     return x
 
 
-def tree_eval(v, depth, ip, ix, w, x, layers, memo=None):
+def tree_eval(v, depth, ip, ix, w, x, layers, memo=None, ef=None):
     """h_v^depth by direct recursion over the in-neighbourhood (Eq. (1)); pure Python floats.
     No memo: every path of the computation tree is evaluated, as a k-hop pipeline would."""
     if depth == 0:
         return [float(t) for t in x[v]]
     lay = layers[depth - 1]
-    hv = tree_eval(v, depth - 1, ip, ix, w, x, layers)
+    hv = tree_eval(v, depth - 1, ip, ix, w, x, layers, ef=ef)
     nb = [(int(ix[j]), (float(w[j]) if (w is not None and lay.use_edge_weights) else 1.0)) for j in range(ip[v], ip[v + 1])]
-    hn = [tree_eval(u, depth - 1, ip, ix, w, x, layers) for u, _ in nb]
+    hn = [tree_eval(u, depth - 1, ip, ix, w, x, layers, ef=ef) for u, _ in nb]
     Fi, Fo = lay.in_dim, lay.out_dim
     W = lay.W
     if lay.op == "gat":
@@ -129,17 +129,24 @@ def tree_eval(v, depth, ip, ix, w, x, layers, memo=None):
                     for c in range(D):
                         out[hd * D + c] += p / tot * z[hd * D + c]
         return [py_act(out[c] + (lay.bias[c] if lay.bias is not None else 0.0), lay.act) for c in range(Fo)]
-    agg = [0.0] * Fi
-    if hn:
-        for f in range(Fi):
-            msgs = [wj * h[f] for (_, wj), h in zip(nb, hn)]
+    De = getattr(lay, "edge_dim", 0)
+    Fm = Fi + De   # length of a message: [w_e h_u | e_vu]
+    full = [[wj * h[f] for f in range(Fi)] + [float(ef[j][f]) for f in range(De)]
+            for j, (_, wj), h in zip(range(ip[v], ip[v + 1]), nb, hn)]
+    agg = [0.0] * Fm
+    if full:
+        for f in range(Fm):
+            msgs = [m[f] for m in full]
             agg[f] = max(msgs) if lay.op == "max" else (min(msgs) if lay.op == "min" else sum(msgs))
             if lay.op == "mean":
                 agg[f] /= len(msgs)
     out = []
     for c in range(Fo):
         t = lay.bias[c] if lay.bias is not None else 0.0
-        t += sum(hv[k] * W[k][c] for k in range(Fi)) + sum(agg[k] * W[Fi + k][c] for k in range(Fi))
+        if lay.op != "gcn":
+            t += sum(hv[k] * W[k][c] for k in range(Fi))
+        r0 = 0 if lay.op == "gcn" else Fi
+        t += sum(agg[k] * W[r0 + k][c] for k in range(Fm))
         out.append(py_act(t, lay.act))
     return out
 
@@ -594,3 +601,130 @@ def test_compact_neighbourhood_gives_the_same_values():
     assert ids.shape[0] < n and np.all(np.diff(ids) > 0)
     part = O.infer_at(cip, cix, cw, X[ids], layers, ct, threshold=3)
     assert np.array_equal(part, full[targets])
+
+
+# ------------------------------------------------------------------ edge features in the message (Eq. (1): e_{v,u})
+
+class TestW5EdgeFeatures:
+    g = GOLD["edge_features"]
+    ip, ix, x = TestW5.ip, TestW5.ix, TestW5.x
+    ef = np.array(GOLD["edge_features"]["ef"], np.float64)
+
+    @pytest.mark.parametrize("op", ["sum", "mean", "max", "min"])
+    def test_edge_aggregates(self, op):
+        assert O.aggregate_edges(self.ip, self.ef, op).tolist() == self.g[op]
+
+    def test_partials_and_combine(self):
+        sp, _, owner = O.split_hubs(self.ip, GOLD["split_T"])
+        assert O.aggregate_edges(sp, self.ef, "sum")[:2].tolist() == self.g["partial_sum_v0"]
+        assert O.aggregate_edges(sp, self.ef, "max")[:2].tolist() == self.g["partial_max_v0"]
+        for op in ("sum", "mean", "max", "min"):
+            P = O.aggregate_edges(sp, self.ef, "sum" if op == "mean" else op)
+            assert O.combine(owner, self.ip, P, op).tolist() == self.g[op]
+
+    @pytest.mark.parametrize("op,key", [("sum", "sage_sum_out"), ("max", "sage_max_out")])
+    def test_sage_layer_with_edge_features(self, op, key):
+        layer = L(op, self.g["act"], self.g["W"], self.g["b"], edge_dim=1)
+        for thr in (0, 2):
+            out = O.sage_layer(self.ip, self.ix, None, self.x, layer, threshold=thr, edge_feat=self.ef)
+            assert out.tolist() == self.g[key]
+
+
+def test_edge_aggregate_is_a_segmented_reduce():
+    """Against numpy's own segmented reductions over the non-empty segments."""
+    rng = np.random.default_rng(31)
+    ip, ix = random_graph(rng, 60, 9)
+    ef = rng.standard_normal((ix.shape[0], 3))
+    deg = np.diff(ip)
+    nz = np.flatnonzero(deg > 0)
+    starts = ip[nz]
+    for op, ufunc in (("sum", np.add), ("max", np.maximum), ("min", np.minimum)):
+        got = O.aggregate_edges(ip, ef, op)
+        assert np.allclose(got[nz], ufunc.reduceat(ef, starts, axis=0), rtol=1e-13, atol=1e-13)
+        assert np.all(got[deg == 0] == 0)
+    mean = O.aggregate_edges(ip, ef, "mean")
+    assert np.allclose(mean[nz], np.add.reduceat(ef, starts, axis=0) / deg[nz][:, None], rtol=1e-13, atol=1e-13)
+
+
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "min", "gcn"])
+@pytest.mark.parametrize("depth", [1, 2])
+def test_edge_feature_layers_equal_computation_tree(op, depth):
+    rng = np.random.default_rng(300 + depth)
+    n, De = 12, 2
+    ip, ix = random_graph(rng, n, 3)
+    w = rng.random(ix.shape[0])
+    ef = rng.standard_normal((ix.shape[0], De))
+    dims = [3, 4, 2][:depth + 1]
+    x = rng.standard_normal((n, dims[0]))
+    layers = []
+    for i in range(depth):
+        fi, fo = dims[i], dims[i + 1]
+        rows = (fi if op == "gcn" else 2 * fi) + De
+        layers.append(L(op, ["relu", "none"][i % 2], rng.standard_normal((rows, fo)), rng.standard_normal(fo),
+                        use_edge_weights=(op != "mean"), edge_dim=De))
+    full = O.infer(ip, ix, w, x, layers, edge_feat=ef)[-1]
+    split = O.infer(ip, ix, w, x, layers, threshold=2, edge_feat=ef)[-1]
+    at = O.infer_at(ip, ix, w, x, layers, np.arange(n), threshold=2, edge_feat=ef)
+    for v in range(n):
+        ref = np.array(tree_eval(v, depth, ip, ix, w, x, layers, ef=ef))
+        assert np.allclose(full[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+        assert np.allclose(split[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+        assert np.allclose(at[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+
+
+def test_edge_feature_special_cases():
+    rng = np.random.default_rng(32)
+    n, Fi, De, Fo = 40, 3, 2, 2
+    ip, ix = random_graph(rng, n, 6)
+    x = rng.standard_normal((n, Fi))
+    ef = rng.standard_normal((ix.shape[0], De))
+    W = rng.standard_normal((2 * Fi + De, Fo))
+    b = rng.standard_normal(Fo)
+    # all-zero edge features: the layer without them whose W drops the edge rows (sum / mean; max of zeros is zero too)
+    for op in ("sum", "mean", "max"):
+        with_zero = O.sage_layer(ip, ix, None, x, L(op, "relu", W, b, edge_dim=De), edge_feat=np.zeros_like(ef))
+        without = O.sage_layer(ip, ix, None, x, L(op, "relu", W[:2 * Fi], b))
+        assert np.allclose(with_zero, without, rtol=1e-13, atol=1e-13)
+    # only the edge rows of W are non-zero and they are the identity: the output is the segment sum of the edge features
+    W2 = np.zeros((2 * Fi + De, De))
+    W2[2 * Fi:] = np.eye(De)
+    out = O.sage_layer(ip, ix, None, x, L("sum", "none", W2, None, edge_dim=De), edge_feat=ef)
+    dense = np.zeros((n, De))
+    for v in range(n):
+        for j in range(ip[v], ip[v + 1]):
+            dense[v] += ef[j]
+    assert np.allclose(out, dense, rtol=1e-13, atol=1e-13)
+    # the vertex part and the edge part of W are not swapped: perturbing an edge row changes the output only
+    # where there are in-edges
+    W3 = W.copy()
+    W3[2 * Fi] += 1.0
+    d = O.sage_layer(ip, ix, None, x, L("sum", "none", W3, b, edge_dim=De), edge_feat=ef) - \
+        O.sage_layer(ip, ix, None, x, L("sum", "none", W, b, edge_dim=De), edge_feat=ef)
+    assert np.allclose(d[:, 0], O.aggregate_edges(ip, ef, "sum")[:, 0], rtol=1e-12, atol=1e-12)
+
+
+def test_edge_feature_split_invariance_is_exact_for_max_and_integer_sums():
+    rng = np.random.default_rng(33)
+    ip, ix = random_graph(rng, 30, 40, p_zero=0.1)
+    ef_int = rng.integers(-5, 6, size=(ix.shape[0], 3)).astype(np.float64)
+    ef = rng.standard_normal((ix.shape[0], 3))
+    for T in (1, 3, 7):
+        sp, _, owner = O.split_hubs(ip, T)
+        for op, e in (("max", ef), ("min", ef), ("sum", ef_int), ("mean", ef_int)):
+            P = O.aggregate_edges(sp, e, "sum" if op == "mean" else op)
+            assert np.array_equal(O.combine(owner, ip, P, op), O.aggregate_edges(ip, e, op)), (op, T)
+
+
+def test_compact_neighbourhood_carries_edge_features():
+    rng = np.random.default_rng(34)
+    n, De = 50, 2
+    ip, ix = random_graph(rng, n, 4)
+    x = rng.standard_normal((n, 3))
+    ef = rng.standard_normal((ix.shape[0], De))
+    layers = [L("mean", "relu", rng.standard_normal((2 * 3 + De, 3)), rng.standard_normal(3), edge_dim=De),
+              L("max", "none", rng.standard_normal((2 * 3 + De, 2)), None, edge_dim=De)]
+    targets = np.array([3, 17, 41])
+    full = O.infer(ip, ix, None, x, layers, edge_feat=ef)[-1]
+    ids, cip, cix, cw, ct, cef = O.compact_neighbourhood(ip, ix, None, targets, 2, edge_feat=ef)
+    got = O.infer_at(cip, cix, cw, x[ids], layers, ct, edge_feat=cef)
+    assert np.allclose(got, full[targets], rtol=1e-12, atol=1e-12)
