@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--workload", default="medium")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--threshold", type=int, default=None, help="hub-split threshold instead of the workload's (0 = no split)")
+    ap.add_argument("--edge-dim", type=int, default=0, help="give every message an edge-feature vector of this length (GraphSAGE workloads)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -51,7 +52,7 @@ def workload_config(w, args):
     return {"workload": f"{w.name}" + ("" if args.scale == 1.0 else f" x{args.scale}"),
             "n_vertices": w.n, "n_edges": w.e, "feat_dim": int(w.layers[0].in_dim), "storage": w.dtype,
             "layers": [f"{l.op}:{l.in_dim}->{l.out_dim}:{l.act}" for l in w.layers],
-            "edge_weights": w.edge_weights is not None, "hub_threshold": w.threshold,
+            "edge_weights": w.edge_weights is not None, "edge_feature_dim": int(w.layers[0].edge_dim), "hub_threshold": w.threshold,
             "l2_policy": "inputs larger than L2 (features + CSR >> 126 MB); no explicit flush"}
 
 
@@ -72,6 +73,7 @@ def time_oracle_sample(w, target_seconds: float):
     O.lib()
     rng = np.random.default_rng(0)
     X = w.x_as_f32().astype(np.float64)
+    ef = w.edge_feat_as_f32()
     inputs = [X] + [rng.standard_normal((w.n, l.out_dim)) for l in w.layers[:-1]]
 
     def run(m):
@@ -79,7 +81,7 @@ def time_oracle_sample(w, target_seconds: float):
         t0 = time.perf_counter()
         for H, layer in zip(inputs, w.layers):
             O.layer_forward(w.indptr, w.indices, w.edge_weights, H, layer, storage=None, threshold=w.threshold,
-                            reorder=False, rows=rows)
+                            reorder=False, rows=rows, edge_feat=ef)
         return time.perf_counter() - t0
 
     m = min(w.n, 20_000)
@@ -95,8 +97,8 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from workloads import make
-    w = make(args.workload, args.scale)
+    from workloads import make, with_edge_features
+    w = with_edge_features(make(args.workload, args.scale), args.edge_dim)
     cores = affinity_cores()
     per_step = max(2.0, min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup)))
     vals, m, secs = [], 0, 0.0
@@ -192,7 +194,7 @@ def run_ours(args):
 
     from paper_2307_00228_b200 import binding as B
     from paper_2307_00228_b200 import host
-    from workloads import make
+    from workloads import make, with_edge_features
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -206,7 +208,7 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
 
-    w = make(args.workload, args.scale)
+    w = with_edge_features(make(args.workload, args.scale), args.edge_dim)
     if args.threshold is not None:
         w.threshold = args.threshold
     d = host.upload(w)
@@ -288,6 +290,9 @@ def run_ours(args):
         if w.edge_weights is not None:
             host_in.append(torch.from_numpy(w.edge_weights).pin_memory())
             dev_in.append(graph_t[2])
+        if w.edge_feat is not None:
+            host_in.append(torch.from_numpy(w.edge_feat if w.dtype == "f32" else w.edge_feat.view(np.int16)).pin_memory())
+            dev_in.append(d.graph._edge_feat.view(torch.int16) if w.dtype == "bf16" else d.graph._edge_feat)
         host_out = torch.empty(d.out.shape, dtype=d.out.dtype).pin_memory()
         h2d = sum(t_.numel() * t_.element_size() for t_ in host_in)
         d2h = host_out.numel() * host_out.element_size()

@@ -74,6 +74,15 @@ typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
  *   W is [in_dim, out_dim].  The degree normalisation is carried by the edge weights and a self loop is
  *   an edge of the graph like any other; the vertex's own state enters in no other way.
  *
+ * Edge features (edge_dim > 0; pooling layers and GCN): Eq. (1) lets the message function M read the feature
+ *   vector e_{v,u} of the edge next to the source state.  The message here is the concatenation
+ *       m_{v,u} = [ w_e * h_u | e_{v,u} ]                      (in_dim + edge_dim entries)
+ *   reduced entry by entry with the layer's op (MEAN divides both parts by the edge count), so that
+ *       GraphSAGE: h'_v = act( h_v * W[0:in_dim] + a_v * W[in_dim : 2*in_dim + edge_dim] + bias ),  W is [2*in_dim + edge_dim, out_dim]
+ *       GCN:       h'_v = act( a_v * W + bias ),                                                  W is [in_dim + edge_dim, out_dim]
+ *   Every message function that is linear in (h_u, e_{v,u}) and is followed by a sum or mean and a dense update
+ *   folds into this form.  The vectors come from it_graph_set_edge_features; such layers are never reordered.
+ *
  * Storage contract: h_in, h_out (and the internal Z / aggregate tensors) are feat_dtype,
  * rounded to nearest even when written; all accumulation is fp32.  W is weight_dtype and
  * must equal feat_dtype.  bias, att_src, att_dst are fp32.  All are device pointers.
@@ -89,6 +98,7 @@ typedef struct {
   float leaky_slope;                    /* GAT only */
   int32_t use_edge_weights;             /* 0/1; needs a graph created with edge weights */
   int32_t allow_reorder;                /* 0/1: allow transform-before-aggregate (see it_layer_forward) */
+  int32_t edge_dim;                     /* 0, or the length of the edge-feature vectors the messages carry (see below) */
 } it_layer_desc;
 
 /*
@@ -107,6 +117,14 @@ typedef struct {
 it_status it_graph_create(int64_t n_vertices, int64_t n_edges, const void *indptr,
                           it_itype indptr_type, const int32_t *indices,
                           const float *edge_weights, void *stream, it_graph **out);
+
+/*
+ * it_graph_set_edge_features — attach the edge features E of G = {V, E, X, E} (Section "K-hop Neighborhood and
+ * Sampling"; e_{v,u} of Eq. (1)): a device matrix [n_edges, edge_dim] of `dtype`, row j belonging to CSR entry j
+ * (the same order as `indices` and `edge_weights`).  Borrowed until it_graph_destroy or the next call; NULL with
+ * edge_dim = 0 detaches them.  A row must be 16, 32, 64, 128, 256 or 512 bytes.  Nothing is launched.
+ */
+it_status it_graph_set_edge_features(it_graph *g, const void *edge_feat, int32_t edge_dim, it_dtype dtype);
 
 /*
  * it_split_hubs — the shadow-node rule ("divide the edges into n groups evenly ... the id

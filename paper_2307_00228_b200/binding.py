@@ -24,7 +24,8 @@ ACTS = {"none": 0, "relu": 1, "elu": 2}
 IT_MAX_BUCKETS = 8
 EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspace_bytes", "it_layer_forward",
            "it_infer", "it_graph_destroy", "it_status_string", "it_last_error_message", "it_profile_begin",
-           "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static", "it_graph_check"]
+           "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static", "it_graph_check",
+           "it_graph_set_edge_features"]
 
 
 class ItError(RuntimeError):
@@ -39,7 +40,8 @@ class it_layer_desc(C.Structure):
                 ("in_dim", C.c_int32), ("out_dim", C.c_int32), ("heads", C.c_int32),
                 ("feat_dtype", C.c_int), ("weight_dtype", C.c_int),
                 ("W", C.c_void_p), ("bias", C.c_void_p), ("att_src", C.c_void_p), ("att_dst", C.c_void_p),
-                ("leaky_slope", C.c_float), ("use_edge_weights", C.c_int32), ("allow_reorder", C.c_int32)]
+                ("leaky_slope", C.c_float), ("use_edge_weights", C.c_int32), ("allow_reorder", C.c_int32),
+                ("edge_dim", C.c_int32)]
 
 
 _lib = None
@@ -107,6 +109,7 @@ class LayerDesc:
     leaky_slope: float = 0.2
     use_edge_weights: bool = False
     allow_reorder: bool = True
+    edge_dim: int = 0
 
     def to_c(self) -> it_layer_desc:
         for t in (self.W, self.bias, self.att_src, self.att_dst):
@@ -124,6 +127,7 @@ class LayerDesc:
         d.leaky_slope = self.leaky_slope
         d.use_edge_weights = int(self.use_edge_weights)
         d.allow_reorder = int(self.allow_reorder)
+        d.edge_dim = int(self.edge_dim)
         return d
 
 
@@ -158,6 +162,20 @@ def it_graph_create(indptr: torch.Tensor, indices: torch.Tensor, edge_weights: t
     _check(lib().it_graph_create(n, e, _ptr(indptr), IT_I64 if indptr.dtype == torch.int64 else IT_I32,
                                  _ptr(indices), _ptr(edge_weights), _stream(stream), C.byref(out)))
     return Graph(out, n, e, (indptr, indices, edge_weights))
+
+
+def it_graph_set_edge_features(g: Graph, edge_feat: torch.Tensor | None):
+    """Attach [n_edges, edge_dim] edge features (CSR order), or detach them with None."""
+    L = lib()
+    L.it_graph_set_edge_features.restype = C.c_int
+    L.it_graph_set_edge_features.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int]
+    if edge_feat is None:
+        _check(L.it_graph_set_edge_features(g.handle, None, 0, IT_F32))
+        g._edge_feat = None
+        return
+    assert edge_feat.is_cuda and edge_feat.is_contiguous() and edge_feat.dim() == 2 and edge_feat.shape[0] == g.e
+    _check(L.it_graph_set_edge_features(g.handle, _ptr(edge_feat), edge_feat.shape[1], _dt(edge_feat.dtype)))
+    g._edge_feat = edge_feat   # borrowed by the library: keep it alive
 
 
 def it_split_hubs(g: Graph, threshold: int, stream=None):

@@ -32,17 +32,25 @@ it_status check_layer(const it_graph *g, const it_layer_desc *L) {
     IT_REQUIRE(!L->use_edge_weights || g->edge_weights, IT_ERR_INVALID_ARG, "layer uses edge weights but the graph has none");
     IT_REQUIRE(L->op != IT_GATHER_NONE || !L->use_edge_weights, IT_ERR_INVALID_ARG, "a dense layer has no edges to weight");
   }
+  IT_REQUIRE(L->edge_dim >= 0, IT_ERR_INVALID_ARG, "edge_dim is negative");
+  if (L->edge_dim > 0) {
+    IT_REQUIRE(L->op != IT_GATHER_GAT && L->op != IT_GATHER_NONE, IT_ERR_UNSUPPORTED, "edge features are taken by the pooling layers and GCN only");
+    IT_REQUIRE(g->edge_feat != nullptr, IT_ERR_INVALID_ARG, "layer uses edge features but the graph has none (it_graph_set_edge_features)");
+    IT_REQUIRE(g->edge_dim == L->edge_dim && g->edge_dtype == L->feat_dtype, IT_ERR_INVALID_ARG,
+               "layer expects edge features [%d] of its feat_dtype, the graph holds [%d]", L->edge_dim, g->edge_dim);
+  }
   return IT_OK;
 }
 
 bool reorders(const it_layer_desc *L) {
-  return L->allow_reorder && (L->op == IT_GATHER_SUM || L->op == IT_GATHER_MEAN || L->op == IT_GATHER_GCN) && L->out_dim < L->in_dim;
+  // with edge features the aggregate of the edge part would need its own transform: such layers keep the plain order
+  return L->allow_reorder && L->edge_dim == 0 && (L->op == IT_GATHER_SUM || L->op == IT_GATHER_MEAN || L->op == IT_GATHER_GCN) && L->out_dim < L->in_dim;
 }
 
 LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
   LayerWs w;
   const size_t n = (size_t)g->n, s = (size_t)it_dtype_size(L->feat_dtype);
-  const size_t fi = (size_t)L->in_dim, fo = (size_t)L->out_dim;
+  const size_t fi = (size_t)L->in_dim, fo = (size_t)L->out_dim, fe = (size_t)L->edge_dim;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += it_align_up(bytes); return o; };
   if (L->op == IT_GATHER_GAT) {
@@ -56,7 +64,7 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
     w.off_B = take(fi * fo * 8);
     w.off_partials = w.off_a = w.off_b = off;
   } else if (L->op == IT_GATHER_GCN) {
-    w.off_B = take(fi * fo * 8);
+    w.off_B = take((fi + fe) * fo * 8);
     if (reorders(L)) {
       w.plan = PLAN_GCN_REORDER;
       w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
@@ -64,8 +72,8 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
       w.off_b = take(n * fo * s);  // Z
     } else {
       w.plan = PLAN_GCN;
-      w.off_partials = take((size_t)g->n_partial_rows * fi * 4);
-      w.off_a = take(n * fi * s);  // A
+      w.off_partials = take((size_t)g->n_partial_rows * (fi > fe ? fi : fe) * 4);
+      w.off_a = take(n * (fi + fe) * s);  // A = [sum_e w_e h_u | sum_e e_vu]
       w.off_b = off;
     }
   } else if (reorders(L)) {
@@ -76,9 +84,9 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
     w.off_b = take(n * fo * s);  // Z
   } else {
     w.plan = PLAN_SAGE;
-    w.off_B = take(2 * fi * fo * 8);
-    w.off_partials = take((size_t)g->n_partial_rows * fi * 4);
-    w.off_a = take(n * fi * s);  // A
+    w.off_B = take((2 * fi + fe) * fo * 8);
+    w.off_partials = take((size_t)g->n_partial_rows * (fi > fe ? fi : fe) * 4);
+    w.off_a = take(n * (fi + fe) * s);  // A = [aggregate of w_e h_u | aggregate of e_vu]
     w.off_b = off;
   }
   w.bytes = off;
@@ -99,8 +107,17 @@ it_status run_apply(const it_graph *g, const it_layer_desc *L, it_prep_kind kind
                              g->d_status, st);
   }
   ga.B = B;
-  IT_TRY(it_launch_prep_weights(kind, L, B, st));
+  IT_TRY(it_launch_prep_weights(kind, L, K, B, st));
   return it_launch_gemm(ga, st);
+}
+
+// The edge-feature half of the message [w_e h_u | e_vu]: the same reduce over the rows of the edge-feature
+// matrix, which lie in edge order, written to columns [in_dim, in_dim + edge_dim) of the aggregate.
+it_status gather_edge_part(it_gather_args gg, const it_layer_desc *L, void *A, int a_ld, cudaStream_t st) {
+  if (L->edge_dim == 0) return IT_OK;
+  gg.src = gg.g->edge_feat; gg.per_edge_rows = 1; gg.use_edge_weights = 0; gg.dim = L->edge_dim;
+  gg.dst = (char *)A + (size_t)L->in_dim * it_dtype_size(gg.dtype); gg.dst_ld = a_ld;
+  return it_launch_gather(gg, st);
 }
 
 it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const void *h_in, void *h_out, char *ws,
@@ -140,6 +157,7 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
   it_gather_args gg{};
   gg.g = g; gg.op = L->op == IT_GATHER_GCN ? IT_GATHER_SUM : L->op; gg.use_edge_weights = L->use_edge_weights; gg.dtype = dt;
   gg.partials = partials;
+  const int a_ld = L->in_dim + L->edge_dim;   // row length of the aggregate handed to apply
   if (w.plan == PLAN_GCN_REORDER) {   // Z = H W, then h' = act(sum_e w_e z_u + b) in the gather's epilogue
     void *Z = ws + w.off_b;
     it_gemm_args ga{};
@@ -151,12 +169,13 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
     gg.dim = L->out_dim; gg.src = Z; gg.dst = h_out; gg.epi = IT_EPI_BIAS_ACT; gg.self_term = nullptr; gg.bias = L->bias; gg.act = L->act;
     return it_launch_gather(gg, st);
   }
-  if (w.plan == PLAN_GCN) {   // A = sum_e w_e h_u, then h' = act(A W + b)
+  if (w.plan == PLAN_GCN) {   // A = sum_e [w_e h_u | e_vu], then h' = act(A W + b)
     void *A = ws + w.off_a;
-    gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.bias = nullptr; gg.act = IT_ACT_NONE;
+    gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.dst_ld = a_ld; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.bias = nullptr; gg.act = IT_ACT_NONE;
     IT_TRY(it_launch_gather(gg, st));
+    IT_TRY(gather_edge_part(gg, L, A, a_ld, st));
     it_gemm_args ga{};
-    ga.M = g->n; ga.x_dtype = dt; ga.X1 = A; ga.K1 = L->in_dim; ga.X2 = nullptr; ga.K2 = 0;
+    ga.M = g->n; ga.x_dtype = dt; ga.X1 = A; ga.K1 = a_ld; ga.X2 = nullptr; ga.K2 = 0;
     ga.B = B; ga.NB = L->out_dim;
     ga.n0 = L->out_dim; ga.out0 = h_out; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = L->act;
     ga.n1 = 0; ga.out1 = nullptr; ga.dt1 = dt; ga.out2 = nullptr;
@@ -175,10 +194,11 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
     return it_launch_gather(gg, st);
   }
   void *A = ws + w.off_a;
-  gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.act = IT_ACT_NONE;
+  gg.dim = L->in_dim; gg.src = h_in; gg.dst = A; gg.dst_ld = a_ld; gg.epi = IT_EPI_STORE; gg.self_term = nullptr; gg.act = IT_ACT_NONE;
   IT_TRY(it_launch_gather(gg, st));
+  IT_TRY(gather_edge_part(gg, L, A, a_ld, st));
   it_gemm_args ga{};
-  ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = A; ga.K2 = L->in_dim;
+  ga.M = g->n; ga.x_dtype = dt; ga.X1 = h_in; ga.K1 = L->in_dim; ga.X2 = A; ga.K2 = a_ld;
   ga.B = B; ga.NB = L->out_dim;
   ga.n0 = L->out_dim; ga.out0 = h_out; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = L->act;
   ga.n1 = 0; ga.out1 = nullptr; ga.dt1 = dt; ga.out2 = nullptr;

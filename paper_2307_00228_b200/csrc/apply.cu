@@ -18,6 +18,7 @@ __device__ __forceinline__ float load_as_float(const void *p, int64_t i, int is_
 // ----------------------------------------------------------------------------- weight prep
 struct PrepParams {
   int kind, in_dim, out_dim, heads, w_is_bf16;
+  int k_rows;   // rows of W that a plain copy takes (SAGE: 2 in_dim + edge_dim; dense / GCN: in_dim (+ edge_dim))
   const void *W;
   const float *att_src, *att_dst;
   float *B;
@@ -26,7 +27,7 @@ struct PrepParams {
 __global__ void prep_weights_kernel(PrepParams p) {
   const int fi = p.in_dim, fo = p.out_dim;
   if (p.kind == IT_PREP_SAGE || p.kind == IT_PREP_DENSE) {
-    int64_t total = (int64_t)(p.kind == IT_PREP_SAGE ? 2 : 1) * fi * fo;
+    int64_t total = (int64_t)p.k_rows * fo;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x)
       p.B[i] = load_as_float(p.W, i, p.w_is_bf16);
   } else if (p.kind == IT_PREP_SAGE_REORDER) {
@@ -149,8 +150,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_fp32_kernel(GemmParams p) {
 
 }  // namespace
 
-it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *L, float *B, cudaStream_t st) {
+it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *L, int K, float *B, cudaStream_t st) {
   PrepParams p;
+  p.k_rows = K;
   p.kind = kind; p.in_dim = L->in_dim; p.out_dim = L->out_dim; p.heads = L->heads;
   p.w_is_bf16 = L->weight_dtype == IT_BF16; p.W = L->W; p.att_src = L->att_src; p.att_dst = L->att_dst; p.B = B;
   IT_LAUNCH(IT_K_PREP, 0, 0, st, prep_weights_kernel<<<64, 256, 0, st>>>(p));

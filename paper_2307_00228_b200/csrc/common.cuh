@@ -73,6 +73,9 @@ struct it_graph {
   it_itype indptr_type = IT_I64;
   const int32_t *indices = nullptr;
   const float *edge_weights = nullptr;
+  const void *edge_feat = nullptr;   // [e, edge_dim] rows in CSR order (borrowed), set by it_graph_set_edge_features
+  int32_t edge_dim = 0;
+  it_dtype edge_dtype = IT_F32;
   int device = 0;
   int num_sms = IT_NUM_SMS_FALLBACK;
 
@@ -115,8 +118,10 @@ struct it_gather_args {
   it_dtype dtype;          // of src rows and of dst rows
   int dim;                 // row length in elements
   const void *src;         // [n, dim] rows that are gathered
+  int per_edge_rows;       // 1: src is [n_edges, dim] and row j belongs to edge j (edge features); 0: rows are looked up by source vertex
   float *partials;         // [n_partial_rows, dim] fp32 scratch (may be NULL when nothing is split)
-  void *dst;               // [n, dim]
+  void *dst;               // row v starts at dst + v * dst_ld elements and takes dim of them
+  int dst_ld;              // 0 means dim
   it_epilogue_kind epi;
   const float *self_term;  // [n, dim] fp32, IT_EPI_ADD_ACT only
   const float *bias;       // [dim] fp32 or NULL, IT_EPI_BIAS_ACT only
@@ -160,9 +165,9 @@ struct it_gemm_args {
 it_status it_launch_gemm(const it_gemm_args &a, cudaStream_t stream);
 
 enum it_prep_kind { IT_PREP_SAGE = 0, IT_PREP_SAGE_REORDER = 1, IT_PREP_GAT = 2, IT_PREP_DENSE = 3 };   // DENSE: B = W [in, out] as it is
-// Assemble the fp32 B matrix for a layer: SAGE [2*in, out] copy; REORDER [in, 2*out] =
+// Assemble the fp32 B matrix for a layer (K = its row count): SAGE and dense / GCN: a copy of W [K, out]; REORDER [in, 2*out] =
 // [W_self | W_neigh]; GAT [in, out + 2*heads] = [W | W a_src | W a_dst].
-it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *layer, float *B,
+it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *layer, int K, float *B,
                                  cudaStream_t stream);
 
 // ----------------------------------------------------------------------------- apply_tc.cu

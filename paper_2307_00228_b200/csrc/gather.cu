@@ -21,7 +21,7 @@ struct SagePolicy {
   void *__restrict__ dst;
   const float *__restrict__ self_term;
   const float *__restrict__ bias;
-  int dim, is_mean, epi, act;
+  int dim, dst_ld, is_mean, epi, act;
   // per-thread
   int col;
   float self[VEC];
@@ -72,7 +72,7 @@ struct SagePolicy {
 #pragma unroll
       for (int i = 0; i < VEC; ++i) st[i] = act_apply(st[i] + (bias ? __ldg(bias + col + i) : 0.f), act);
     }
-    Slice::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dim + col, st);
+    Slice::store(reinterpret_cast<T *>(dst) + (int64_t)dest * dst_ld + col, st);
   }
 };
 
@@ -88,7 +88,7 @@ struct CombineParams {
   const float *__restrict__ self_term;
   const float *__restrict__ bias;
   int64_t n_split_owners;
-  int dim;
+  int dim, dst_ld;
   int red, is_mean, epi, act;   // red: RED_SUM / RED_MAX / RED_MIN
 };
 
@@ -125,6 +125,7 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
       for (; g < n; ++g) fold(__ldg(reinterpret_cast<const float4 *>(p.partials + (p0 + g) * p.dim + c)));
       float o[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
       const int64_t off = v * p.dim + c;
+      const int64_t doff = v * p.dst_ld + c;
       if (p.epi == IT_EPI_ADD_ACT) {
         float4 s = __ldg(reinterpret_cast<const float4 *>(p.self_term + off));
         o[0] = act_apply(o[0] + s.x, p.act); o[1] = act_apply(o[1] + s.y, p.act);
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 #pragma unroll
         for (int i = 0; i < 4; ++i) o[i] = act_apply(o[i] + (p.bias ? __ldg(p.bias + c + i) : 0.f), p.act);
       }
-      T *d = reinterpret_cast<T *>(p.dst) + off;
+      T *d = reinterpret_cast<T *>(p.dst) + doff;
       if (sizeof(T) == 4) {
         *reinterpret_cast<float4 *>(d) = make_float4(o[0], o[1], o[2], o[3]);
       } else {
@@ -148,14 +149,14 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 template <typename T, int SB, int LPR, int RED, bool WEIGHTED>
 it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   SagePolicy<T, SB, RED, WEIGHTED> pol;
-  pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim;
+  pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim; pol.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
   const it_graph *g = a.g;
   // algorithmic bytes: per edge the index, the optional weight and one source row; per row its
   // metadata and one output row (plus the self row it is added to)
   const double row_bytes = (double)a.dim * sizeof(T);
   auto bytes_of = [=](int b, int64_t rows) {
-    return (double)g->h_bucket_edges[b] * (4.0 + (WEIGHTED ? 4.0 : 0.0) + row_bytes) +
+    return (double)g->h_bucket_edges[b] * ((a.per_edge_rows ? 0.0 : 4.0) + (WEIGHTED ? 4.0 : 0.0) + row_bytes) +
            (double)rows * (16.0 + row_bytes + (a.epi == IT_EPI_ADD_ACT ? 4.0 * a.dim : 0.0));
   };
   return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, bound_lo, bound_hi, st);
@@ -181,7 +182,7 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
   IT_REQUIRE(g->n_partial_rows == 0 || a.partials, IT_ERR_WORKSPACE, "gather: no partial buffer");
   if (g->n == 0) return IT_OK;
   StreamParams sp;
-  sp.meta = g->bucket_meta; sp.owner = nullptr; sp.indices = g->indices; sp.weights = g->edge_weights;
+  sp.meta = g->bucket_meta; sp.owner = nullptr; sp.indices = a.per_edge_rows ? nullptr : g->indices; sp.weights = g->edge_weights;
   sp.src = a.src; sp.row_lo = sp.row_hi = 0; sp.dim = a.dim; sp.batch_rows = 1;
   if (a.dtype == IT_F32) IT_TRY(launch_lpr<float>(a, sp, st));
   else IT_TRY(launch_lpr<__nv_bfloat16>(a, sp, st));
@@ -189,7 +190,7 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
     CombineParams c;
     c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.shadow_indptr = g->shadow_indptr;
     c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.bias = a.bias; c.n_split_owners = g->n_split_owners;
-    c.dim = a.dim; c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
+    c.dim = a.dim; c.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
     int64_t want = (g->n_split_owners + 7) / 8;
     int64_t cap = (int64_t)g->num_sms * 8;
     unsigned blocks = (unsigned)(want < cap ? want : cap);

@@ -380,6 +380,22 @@ static it_status split_impl(it_graph *g, int64_t T, cudaStream_t st) {
   return IT_OK;
 }
 
+extern "C" it_status it_graph_set_edge_features(it_graph *g, const void *edge_feat, int32_t edge_dim, it_dtype dtype) {
+  IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
+  if (edge_feat == nullptr || edge_dim == 0) {
+    IT_REQUIRE(edge_feat == nullptr && edge_dim == 0, IT_ERR_INVALID_ARG, "edge features need both a pointer and a dimension");
+    g->edge_feat = nullptr; g->edge_dim = 0;
+    return IT_OK;
+  }
+  IT_REQUIRE(dtype == IT_F32 || dtype == IT_BF16, IT_ERR_INVALID_ARG, "bad edge feature dtype");
+  const int64_t row = (int64_t)edge_dim * it_dtype_size(dtype);
+  IT_REQUIRE(edge_dim > 0 && row >= 16 && row <= 512 && (row & (row - 1)) == 0, IT_ERR_INVALID_ARG,
+             "an edge-feature row must be 16, 32, 64, 128, 256 or 512 bytes (got %lld)", (long long)row);
+  IT_REQUIRE(((uintptr_t)edge_feat % 16) == 0, IT_ERR_INVALID_ARG, "edge features must be 16-byte aligned");
+  g->edge_feat = edge_feat; g->edge_dim = edge_dim; g->edge_dtype = dtype;
+  return IT_OK;
+}
+
 extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, it_itype indptr_type,
                                      const int32_t *indices, const float *edge_weights, void *stream,
                                      it_graph **out) {

@@ -150,9 +150,9 @@ __device__ __forceinline__ float act_apply(float x, int act) {
 struct StreamParams {
   const it_row_meta *__restrict__ meta;   // bucket order
   const int32_t *__restrict__ owner;      // bucket order: vertex a row belongs to (policies with NEEDS_OWNER)
-  const int32_t *__restrict__ indices;
+  const int32_t *__restrict__ indices;    // source vertex of every edge; NULL: row j of src belongs to edge j itself (edge features)
   const float *__restrict__ weights;
-  const void *__restrict__ src;           // [n, dim] rows that are gathered
+  const void *__restrict__ src;           // [n, dim] rows that are gathered ([n_edges, dim] when indices is NULL)
   int64_t row_lo, row_hi;                 // range inside the bucket-ordered row list
   int dim;
   int batch_rows;                         // rows a lane group takes at a time (<= LPR)
@@ -224,7 +224,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
       idx = 0;
       w = 1.f;
       if (q < total) {
-        idx = __ldcs(p.indices + j);
+        idx = p.indices ? __ldcs(p.indices + j) : (int32_t)j;
         if (Policy::WEIGHTED) w = __ldcs(p.weights + j);
       }
       ends = (__ballot_sync(gmask, q < total && q + 1 == row_end) >> (lane - t)) & gbits;
@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(THREADS, IT_SHORT_MIN_BLOCKS) stream_short_row
       int32_t idx = 0;
       float w = 1.f;
       if (t < E && k0 + t < len) {
-        idx = __ldcs(p.indices + j0 + k0 + t);
+        idx = p.indices ? __ldcs(p.indices + j0 + k0 + t) : (int32_t)(j0 + k0 + t);
         if (Policy::WEIGHTED) w = __ldcs(p.weights + j0 + k0 + t);
       }
       typename Slice::Raw v[E];
@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
     auto load_chunk = [&](int64_t base, int32_t &idx, float &w) {
       idx = 0; w = 1.f;
       if (base + lane < b) {
-        idx = __ldcs(p.indices + base + lane);
+        idx = p.indices ? __ldcs(p.indices + base + lane) : (int32_t)(base + lane);
         if (Policy::WEIGHTED) w = __ldcs(p.weights + base + lane);
       }
     };

@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_
       idx = 0;
       w = 1.f;
       if (q < total) {
-        idx = __ldcs(p.indices + j);
+        idx = p.indices ? __ldcs(p.indices + j) : (int32_t)j;
         if (Policy::WEIGHTED) w = __ldcs(p.weights + j);
       }
       ends = __ballot_sync(0xffffffffu, q < total && q + 1 == row_end);
@@ -298,7 +298,7 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_cta_ring_k
     auto load_chunk = [&](int base, int32_t &idx, float &w, unsigned &ends) {
       idx = 0; w = 1.f; ends = 0u;
       if (base + lane < total) {
-        idx = __ldcs(p.indices + a + base + lane);
+        idx = p.indices ? __ldcs(p.indices + a + base + lane) : (int32_t)(a + base + lane);
         if (Policy::WEIGHTED) w = __ldcs(p.weights + a + base + lane);
       }
     };

@@ -28,7 +28,8 @@ def layer_to_device(layer, dtype: str, device="cuda") -> B.LayerDesc:
     return B.LayerDesc(op=layer.op, act=layer.act, in_dim=layer.in_dim, out_dim=layer.out_dim,
                        W=param_to_device(layer.W, dtype, device), bias=f32(layer.bias), heads=layer.heads,
                        att_src=f32(layer.att_src), att_dst=f32(layer.att_dst), leaky_slope=float(layer.leaky_slope),
-                       use_edge_weights=bool(layer.use_edge_weights), allow_reorder=bool(layer.allow_reorder))
+                       use_edge_weights=bool(layer.use_edge_weights), allow_reorder=bool(layer.allow_reorder),
+                       edge_dim=int(getattr(layer, "edge_dim", 0) or 0))
 
 
 @dataclass
@@ -51,6 +52,8 @@ def upload(w, device="cuda", int32_indptr=False, threshold=None) -> DeviceWorklo
     indices = torch.from_numpy(w.indices).to(device)
     ew = None if w.edge_weights is None else torch.from_numpy(w.edge_weights).to(device)
     g = B.it_graph_create(indptr, indices, ew)
+    if getattr(w, "edge_feat", None) is not None:
+        B.it_graph_set_edge_features(g, features_to_device(w.edge_feat, w.dtype, device))
     thr = w.threshold if threshold is None else threshold
     n_rows, n_split = B.it_split_hubs(g, thr)
     layers = [layer_to_device(l, w.dtype, device) for l in w.layers]

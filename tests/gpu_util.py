@@ -24,7 +24,7 @@ def storage_exact(a: np.ndarray, dtype: str) -> np.ndarray:
     return wrng.bf16_bits_to_f32(wrng.f32_to_bf16_bits(a)) if dtype == "bf16" else a
 
 
-def small_workload(seed, n, max_deg, dtype, layers, hubs=(), weights=False, threshold=0, p_zero=0.2) -> Workload:
+def small_workload(seed, n, max_deg, dtype, layers, hubs=(), weights=False, threshold=0, p_zero=0.2, edge_dim=0) -> Workload:
     rng = np.random.default_rng(seed)
     deg = rng.integers(0, max_deg + 1, size=n)
     deg[rng.random(n) < p_zero] = 0
@@ -37,25 +37,30 @@ def small_workload(seed, n, max_deg, dtype, layers, hubs=(), weights=False, thre
     w = rng.random(e, dtype=np.float32) if weights else None
     x = rng.standard_normal((n, layers[0].in_dim)).astype(np.float32)
     xs = x if dtype == "f32" else wrng.f32_to_bf16_bits(x)
-    return Workload("small", n, e, indptr, indices, w, dtype, xs, layers, threshold)
+    ef = None
+    if edge_dim:
+        ef = rng.standard_normal((e, edge_dim)).astype(np.float32)
+        ef = ef if dtype == "f32" else wrng.f32_to_bf16_bits(ef)
+    return Workload("small", n, e, indptr, indices, w, dtype, xs, layers, threshold, ef)
 
 
-def make_sage_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=True, bias=True) -> Layer:
+def make_sage_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=True, bias=True, edge_dim=0) -> Layer:
     rng = np.random.default_rng(seed)
-    lim = np.sqrt(6.0 / (2 * fi + fo))
+    lim = np.sqrt(6.0 / (2 * fi + edge_dim + fo))
     return Layer(op=op, act=act, in_dim=fi, out_dim=fo,
-                 W=storage_exact(rng.uniform(-lim, lim, (2 * fi, fo)), dtype),
+                 W=storage_exact(rng.uniform(-lim, lim, (2 * fi + edge_dim, fo)), dtype),
                  bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None,
-                 use_edge_weights=weights, allow_reorder=allow_reorder)
+                 use_edge_weights=weights, allow_reorder=allow_reorder, edge_dim=edge_dim)
 
 
-def make_plain_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=True, bias=True) -> Layer:
-    """op = "dense" (no Gather stage) or "gcn" (update on the aggregate alone): W is [fi, fo]."""
+def make_plain_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=True, bias=True, edge_dim=0) -> Layer:
+    """op = "dense" (no Gather stage) or "gcn" (update on the aggregate alone): W is [fi (+ edge_dim), fo]."""
     rng = np.random.default_rng(seed)
-    lim = np.sqrt(6.0 / (fi + fo))
-    return Layer(op=op, act=act, in_dim=fi, out_dim=fo, W=storage_exact(rng.uniform(-lim, lim, (fi, fo)), dtype),
+    lim = np.sqrt(6.0 / (fi + edge_dim + fo))
+    return Layer(op=op, act=act, in_dim=fi, out_dim=fo,
+                 W=storage_exact(rng.uniform(-lim, lim, (fi + edge_dim, fo)), dtype),
                  bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None,
-                 use_edge_weights=weights, allow_reorder=allow_reorder)
+                 use_edge_weights=weights, allow_reorder=allow_reorder, edge_dim=edge_dim)
 
 
 def make_gat_layer(seed, act, fi, heads, hd, dtype, bias=True) -> Layer:
@@ -82,7 +87,7 @@ def run_oracle(w: Workload, storage="same", threshold=None):
     st = w.dtype if storage == "same" else storage
     thr = w.threshold if threshold is None else threshold
     return O.infer(w.indptr, w.indices, w.edge_weights, w.x_as_f32(), w.layers, storage=st, threshold=thr,
-                   follow_reorder=True)
+                   follow_reorder=True, edge_feat=w.edge_feat_as_f32())
 
 
 def check_against_oracle(w: Workload, got: np.ndarray, tol=None, label=""):

@@ -85,6 +85,73 @@ def test_extreme_hub_rows_at_scale():
     check_sampled(w, d, sampled_targets(w, 3, 200), "extreme")
 
 
+FULL = pytest.mark.skipif(not (os.environ.get("IT_RUN_FULL") or os.environ.get("IT_RUN_LARGE")),
+                          reason="set IT_RUN_FULL=1: full-size GAT and Extreme take a few minutes of host time to generate and check")
+
+
+def check_compact(w, d, targets, label):
+    """Sampled vertices of a big workload against the oracle evaluated on their L-hop in-neighbourhood,
+    relabelled to a compact graph so that no full-size fp64 array is needed."""
+    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, w.edge_weights, targets, len(w.layers))
+    xc = w.x[ids] if w.dtype == "f32" else wrng.bf16_bits_to_f32(w.x[ids])
+    ref = O.infer_at(cip, cix, cw, xc, w.layers, ct, storage=w.dtype, threshold=w.threshold, follow_reorder=True)
+    got = to_numpy(d.out[torch.from_numpy(targets).cuda()])
+    err = compare.rel_error(got, ref)
+    print(f"{label} full size:", err, "rows", d.n_rows, "split owners", d.n_split_owners, "compact vertices", len(ids))
+    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], (label, err)
+    assert bool(torch.isfinite(d.out.float()).all())
+
+
+@FULL
+def test_gat_full_size_sampled():
+    """5M vertices, 100M edges, bf16, two GAT layers of 4 heads, hubs split at 4096 (partial softmax states
+    merged): the two largest hubs and a random sample."""
+    w = make("gat")
+    d = host.upload(w)
+    assert d.n_split_owners > 0
+    d.infer()
+    B.it_graph_check(d.graph)
+    check_compact(w, d, sampled_targets(w, 2, 200), "gat")
+
+
+@FULL
+def test_extreme_full_size_sampled():
+    """20M vertices, 200M edges, 100 hubs of 1M in-edges (245 shadow rows each), bf16, three max-pooling layers.
+    A hub's 3-hop in-neighbourhood is the whole graph, so the final output is checked on random vertices
+    with no hub within two hops, and the hubs themselves on the output of the first layer alone."""
+    w = make("extreme")
+    d = host.upload(w)
+    assert d.n_split_owners == 100
+    d.infer()
+    B.it_graph_check(d.graph)
+    deg = np.diff(w.indptr)
+    hubs = np.flatnonzero(deg >= 1_000_000)
+    assert hubs.size == 100
+    is_hub = np.zeros(w.n, bool)
+    is_hub[hubs] = True
+    cand = np.random.default_rng(11).choice(w.n, size=600, replace=False)
+    keep = []
+    for v in cand:
+        hop1 = w.indices[w.indptr[v]:w.indptr[v + 1]]
+        hop2 = np.concatenate([w.indices[w.indptr[u]:w.indptr[u + 1]] for u in hop1]) if hop1.size else hop1
+        if not (is_hub[v] or is_hub[hop1].any() or is_hub[hop2].any()):
+            keep.append(v)
+    targets = np.unique(np.array(keep[:300], dtype=np.int64))
+    assert targets.size >= 100
+    check_compact(w, d, targets, "extreme")
+    # the hubs after one layer: 245 partial max rows each, combined
+    h3 = hubs[:3].astype(np.int64)
+    o1 = torch.empty((w.n, w.layers[0].out_dim), dtype=d.x.dtype, device="cuda")
+    B.it_layer_forward(d.graph, d.layers[0], d.x, o1, d.workspace)
+    B.it_graph_check(d.graph)
+    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, None, h3, 1)
+    ref = O.infer_at(cip, cix, cw, wrng.bf16_bits_to_f32(w.x[ids]), w.layers[:1], ct, storage=w.dtype,
+                     threshold=w.threshold, follow_reorder=True)
+    err = compare.rel_error(to_numpy(o1[torch.from_numpy(h3).cuda()]), ref)
+    print("extreme hubs after layer 1:", err)
+    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], err
+
+
 @pytest.mark.skipif(not os.environ.get("IT_RUN_LARGE"), reason="set IT_RUN_LARGE=1: needs ~100 GB of HBM, ~60 GB of host RAM and ~10 minutes")
 def test_large_full_size_sampled():
     """100M vertices, 1.5B edges, int32 CSR, bf16: sampled vertices against the oracle evaluated on

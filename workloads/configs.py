@@ -31,6 +31,7 @@ class Layer:
     leaky_slope: float = 0.2
     use_edge_weights: bool = False
     allow_reorder: bool = True
+    edge_dim: int = 0        # > 0: the message carries the edge's feature vector; W has edge_dim more neighbour rows
 
 
 @dataclass
@@ -45,9 +46,15 @@ class Workload:
     x: np.ndarray             # float32 [n, f] (f32) or uint16 bf16 bit patterns [n, f] (bf16)
     layers: list = field(default_factory=list)
     threshold: int = 0        # shadow-row threshold; <= 0 means no split
+    edge_feat: np.ndarray | None = None   # [e, edge_dim], float32 or bf16 bit patterns like x; row j belongs to CSR entry j
 
     def x_as_f32(self) -> np.ndarray:
         return self.x if self.dtype == "f32" else wrng.bf16_bits_to_f32(self.x)
+
+    def edge_feat_as_f32(self) -> np.ndarray | None:
+        if self.edge_feat is None:
+            return None
+        return self.edge_feat if self.dtype == "f32" else wrng.bf16_bits_to_f32(self.edge_feat)
 
 
 def _glorot(rng, fan_in: int, fan_out: int, shape) -> np.ndarray:
@@ -62,16 +69,17 @@ def _storage_round(a: np.ndarray, dtype: str) -> np.ndarray:
     return a
 
 
-def sage_layers(dims, op, acts, dtype, use_edge_weights=False) -> list:
-    """GraphSAGE layers dims[0]->dims[1]->...; Glorot-uniform over the whole [2*in, out]
+def sage_layers(dims, op, acts, dtype, use_edge_weights=False, edge_dim=0) -> list:
+    """GraphSAGE layers dims[0]->dims[1]->...; Glorot-uniform over the whole [2*in (+ edge_dim), out]
     matrix; bias ~ U(-0.1, 0.1)."""
     out = []
     for i in range(len(dims) - 1):
         fi, fo = dims[i], dims[i + 1]
-        W = _glorot(wrng.stream(wrng.SEED_WEIGHTS, i), 2 * fi, fo, (2 * fi, fo))
+        k = 2 * fi + edge_dim
+        W = _glorot(wrng.stream(wrng.SEED_WEIGHTS, i), k, fo, (k, fo))
         b = wrng.stream(wrng.SEED_BIAS, i).uniform(-0.1, 0.1, size=fo).astype(np.float32)
         out.append(Layer(op=op, act=acts[i], in_dim=fi, out_dim=fo, W=_storage_round(W, dtype),
-                         bias=b, use_edge_weights=use_edge_weights))
+                         bias=b, use_edge_weights=use_edge_weights, edge_dim=edge_dim))
     return out
 
 
@@ -93,6 +101,21 @@ def gat_layers(dims, heads, acts, dtype, slope=0.2) -> list:
 def _features(n, f, dtype):
     r = wrng.stream(wrng.SEED_FEATURES)
     return wrng.normal_f32(r, (n, f)) if dtype == "f32" else wrng.normal_bf16_bits(r, (n, f))
+
+
+def with_edge_features(w: Workload, edge_dim: int) -> Workload:
+    """The same workload with seeded N(0,1) edge features of length edge_dim in every message (GraphSAGE
+    workloads only): the layers are redrawn with edge_dim more neighbour rows."""
+    if edge_dim <= 0:
+        return w
+    if any(l.op == "gat" for l in w.layers):
+        raise ValueError("edge features are defined for the pooling layers and GCN")
+    r = wrng.stream(wrng.SEED_EDGE_FEATURES)
+    w.edge_feat = wrng.normal_f32(r, (w.e, edge_dim)) if w.dtype == "f32" else wrng.normal_bf16_bits(r, (w.e, edge_dim))
+    dims = [w.layers[0].in_dim] + [l.out_dim for l in w.layers]
+    w.layers = sage_layers(dims, w.layers[0].op, [l.act for l in w.layers], w.dtype,
+                           use_edge_weights=w.layers[0].use_edge_weights, edge_dim=edge_dim)
+    return w
 
 
 def make(name: str, scale: float = 1.0) -> Workload:

@@ -17,6 +17,7 @@ SEED_GRAPH = 1
 SEED_FEATURES = 2
 SEED_EDGE_WEIGHTS = 3
 SEED_BIAS = 4
+SEED_EDGE_FEATURES = 5
 
 
 def stream(seed: int, substream: int = 0) -> np.random.Generator:
