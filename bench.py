@@ -58,6 +58,9 @@ def workload_config(w, args):
 
 # ----------------------------------------------------------------------------- CPU oracle timing
 
+COMPACT_ABOVE_BYTES = 16e9   # fp64 bytes of one whole layer input above which the oracle sample is compacted
+
+
 def affinity_cores() -> int:
     try:
         return len(os.sched_getaffinity(0))
@@ -68,16 +71,32 @@ def affinity_cores() -> int:
 def time_oracle_sample(w, target_seconds: float):
     """The oracle as it stands, on destinations [0, m) of the workload's graph: every layer's
     pass over those vertices (layer inputs beyond the first are a seeded stand-in of the right
-    shape: the time does not depend on the values).  Returns (vertices/s, m, seconds)."""
+    shape: the time does not depend on the values).  Returns (vertices/s, m, seconds).
+    Where fp64 copies of whole layer inputs would not fit comfortably in host memory (the 100M-vertex
+    workload), the sampled destinations and the vertices they read are first relabelled to a compact
+    graph, outside the timed region; the timed arithmetic is the same."""
     from oracle import oracle as O
+    from workloads import rng as wrng
     O.lib()
     rng = np.random.default_rng(0)
-    X = w.x_as_f32().astype(np.float64)
     ef = w.edge_feat_as_f32()
-    inputs = [X] + [rng.standard_normal((w.n, l.out_dim)) for l in w.layers[:-1]]
+    dims = [w.layers[0].in_dim] + [l.out_dim for l in w.layers[:-1]]
+    compact = w.n * max(dims) * 8 > COMPACT_ABOVE_BYTES
+
+    if not compact:
+        X = w.x_as_f32().astype(np.float64)
+        inputs = [X] + [rng.standard_normal((w.n, l.out_dim)) for l in w.layers[:-1]]
 
     def run(m):
         rows = np.arange(m, dtype=np.int64)
+        if compact:
+            ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, w.edge_weights, rows, 1)[:5]
+            x0 = w.x[ids] if w.dtype == "f32" else wrng.bf16_bits_to_f32(w.x[ids])
+            ins = [x0.astype(np.float64)] + [rng.standard_normal((len(ids), l.out_dim)) for l in w.layers[:-1]]
+            t0 = time.perf_counter()
+            for H, layer in zip(ins, w.layers):
+                O.layer_forward(cip, cix, cw, H, layer, storage=None, threshold=w.threshold, reorder=False, rows=ct)
+            return time.perf_counter() - t0
         t0 = time.perf_counter()
         for H, layer in zip(inputs, w.layers):
             O.layer_forward(w.indptr, w.indices, w.edge_weights, H, layer, storage=None, threshold=w.threshold,
@@ -88,6 +107,8 @@ def time_oracle_sample(w, target_seconds: float):
     t = run(m)
     if m < w.n and t < target_seconds / 2:
         m = int(min(w.n, max(m, m * target_seconds / max(t, 1e-3))))
+        if compact:
+            m = min(m, 500_000)   # keeps the fp64 inputs of the compact graph to a few GB
         t = run(m)
     return m / t, m, t
 
@@ -211,7 +232,8 @@ def run_ours(args):
     w = with_edge_features(make(args.workload, args.scale), args.edge_dim)
     if args.threshold is not None:
         w.threshold = args.threshold
-    d = host.upload(w)
+    int32_csr = w.name == "large"   # that workload is defined with an int32 CSR
+    d = host.upload(w, int32_indptr=int32_csr)
     dev = torch.device("cuda", local)
 
     for _ in range(max(3, args.warmup)):
@@ -285,7 +307,8 @@ def run_ours(args):
     if not args.no_e2e:
         graph_t = d.graph._keep
         host_in = [torch.from_numpy(w.x if w.dtype == "f32" else w.x.view(np.int16)).pin_memory(),
-                   torch.from_numpy(w.indptr).pin_memory(), torch.from_numpy(w.indices).pin_memory()]
+                   torch.from_numpy(w.indptr.astype(np.int32) if int32_csr else w.indptr).pin_memory(),
+                   torch.from_numpy(w.indices).pin_memory()]
         dev_in = [d.x.view(torch.int16) if w.dtype == "bf16" else d.x, graph_t[0], graph_t[1]]
         if w.edge_weights is not None:
             host_in.append(torch.from_numpy(w.edge_weights).pin_memory())

@@ -11,7 +11,10 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
  *     enqueued on it; a call synchronises that stream only where it must read a status
  *     or a count back (it_graph_create, it_split_hubs).
- *   - Matrices are row-major and dense.  Feature rows must be a multiple of 16 bytes.
+ *   - Matrices are row-major and dense.  Feature rows (layer inputs and outputs, edge features) must be a
+ *     multiple of 16 bytes; the pooling layers and GCN take any such width (rows other than 16, 32, ..., 512
+ *     bytes are gathered in column chunks of those widths), GAT rows must be one of those widths.  The dense
+ *     transform runs on the tensor cores when out_dim is a multiple of 16 and on the CUDA cores otherwise.
  *   - Errors are return codes only: nothing throws, aborts or traps the device.  On
  *     error no output is defined.  it_status_string() names a code;
  *     it_last_error_message() gives the detail of the calling thread's last failure.
@@ -122,7 +125,7 @@ it_status it_graph_create(int64_t n_vertices, int64_t n_edges, const void *indpt
  * it_graph_set_edge_features — attach the edge features E of G = {V, E, X, E} (Section "K-hop Neighborhood and
  * Sampling"; e_{v,u} of Eq. (1)): a device matrix [n_edges, edge_dim] of `dtype`, row j belonging to CSR entry j
  * (the same order as `indices` and `edge_weights`).  Borrowed until it_graph_destroy or the next call; NULL with
- * edge_dim = 0 detaches them.  A row must be 16, 32, 64, 128, 256 or 512 bytes.  Nothing is launched.
+ * edge_dim = 0 detaches them.  A row must be a multiple of 16 bytes.  Nothing is launched.
  */
 it_status it_graph_set_edge_features(it_graph *g, const void *edge_feat, int32_t edge_dim, it_dtype dtype);
 

@@ -51,20 +51,21 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
   LayerWs w;
   const size_t n = (size_t)g->n, s = (size_t)it_dtype_size(L->feat_dtype);
   const size_t fi = (size_t)L->in_dim, fo = (size_t)L->out_dim, fe = (size_t)L->edge_dim;
+  const size_t kpad = 128;   // the tensor-core path pads the K of each operand to whole k-blocks (at most 63 + 63 rows)
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += it_align_up(bytes); return o; };
   if (L->op == IT_GATHER_GAT) {
     w.plan = PLAN_GAT;
-    w.off_B = take(fi * (fo + 2 * (size_t)L->heads) * 8);
+    w.off_B = take((fi + kpad) * (fo + 2 * (size_t)L->heads) * 8);
     w.off_partials = take(it_gat_partial_bytes(g, L->out_dim, L->heads));
     w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
     w.off_b = take(n * fo * s);                    // Z
   } else if (L->op == IT_GATHER_NONE) {
     w.plan = PLAN_DENSE;
-    w.off_B = take(fi * fo * 8);
+    w.off_B = take((fi + kpad) * fo * 8);
     w.off_partials = w.off_a = w.off_b = off;
   } else if (L->op == IT_GATHER_GCN) {
-    w.off_B = take((fi + fe) * fo * 8);
+    w.off_B = take((fi + fe + kpad) * fo * 8);
     if (reorders(L)) {
       w.plan = PLAN_GCN_REORDER;
       w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
@@ -78,13 +79,13 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
     }
   } else if (reorders(L)) {
     w.plan = PLAN_SAGE_REORDER;
-    w.off_B = take(fi * 2 * fo * 8);
+    w.off_B = take((fi + kpad) * 2 * fo * 8);
     w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
     w.off_a = take(n * fo * 4);  // S (fp32)
     w.off_b = take(n * fo * s);  // Z
   } else {
     w.plan = PLAN_SAGE;
-    w.off_B = take((2 * fi + fe) * fo * 8);
+    w.off_B = take((2 * fi + fe + kpad) * fo * 8);
     w.off_partials = take((size_t)g->n_partial_rows * (fi > fe ? fi : fe) * 4);
     w.off_a = take(n * (fi + fe) * s);  // A = [aggregate of w_e h_u | aggregate of e_vu]
     w.off_b = off;
@@ -102,7 +103,7 @@ it_status run_apply(const it_graph *g, const it_layer_desc *L, it_prep_kind kind
   const bool want_scores = kind == IT_PREP_GAT;
   const int heads = L->heads > 0 ? L->heads : 1, hd = L->out_dim / heads;
   if (it_tc_supported(ga, heads, hd, want_scores)) {
-    IT_TRY(it_launch_prep_weights_tc(kind, L, ga.n0 + ga.n1, K, B, st));
+    IT_TRY(it_launch_prep_weights_tc(kind, L, ga.n0 + ga.n1, ga.K1, ga.X2 ? ga.K2 : 0, B, st));
     return it_launch_gemm_tc(ga, B, L->att_src, L->att_dst, heads, hd, want_scores ? scores : nullptr, g->num_sms,
                              g->d_status, st);
   }
@@ -115,7 +116,7 @@ it_status run_apply(const it_graph *g, const it_layer_desc *L, it_prep_kind kind
 // matrix, which lie in edge order, written to columns [in_dim, in_dim + edge_dim) of the aggregate.
 it_status gather_edge_part(it_gather_args gg, const it_layer_desc *L, void *A, int a_ld, cudaStream_t st) {
   if (L->edge_dim == 0) return IT_OK;
-  gg.src = gg.g->edge_feat; gg.per_edge_rows = 1; gg.use_edge_weights = 0; gg.dim = L->edge_dim;
+  gg.src = gg.g->edge_feat; gg.src_ld = 0; gg.per_edge_rows = 1; gg.use_edge_weights = 0; gg.dim = L->edge_dim;
   gg.dst = (char *)A + (size_t)L->in_dim * it_dtype_size(gg.dtype); gg.dst_ld = a_ld;
   return it_launch_gather(gg, st);
 }

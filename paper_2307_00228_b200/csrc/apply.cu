@@ -6,7 +6,7 @@ namespace {
 
 __device__ __forceinline__ float act_apply(float x, int act) {
   if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
-  if (act == IT_ACT_ELU) return x > 0.f ? x : expm1f(x);
+  if (act == IT_ACT_ELU) return it_elu(x);
   return x;
 }
 

@@ -30,6 +30,9 @@ constexpr int TC_BM = 128;          // rows per tile (UMMA M)
 constexpr int TC_KBLOCK_BYTES = 128;  // one swizzle row of K per k-block
 constexpr int TC_EPI_WARPS = 16;      // four warps per TMEM lane quarter, each takes every fourth 16-column group
 constexpr int TC_THREADS_BF16 = 64 + 32 * TC_EPI_WARPS;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2-17 epilogue
+#ifndef IT_TC_MAX_STAGES
+#define IT_TC_MAX_STAGES 8   // operand stages in shared memory (as many as fit, up to this)
+#endif
 #ifndef IT_TC_SPLIT_GROUPS
 #define IT_TC_SPLIT_GROUPS 1   // groups of four split warps; group g takes every k-block c with c % groups == g (measured: a second group gains nothing)
 #endif
@@ -399,7 +402,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
                 for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
               } else if (p.act0 == IT_ACT_ELU) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = v[i] > 0.f ? v[i] : expm1f(v[i]);
+                for (int i = 0; i < 16; ++i) v[i] = it_elu(v[i]);
               }
               dst = p.out0; bf16 = p.out0_bf16; ld = p.n0; lc = gc;
             } else {
@@ -538,22 +541,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
 
 // ----------------------------------------------------------------------------- weight prep (K-major, split)
 struct PrepTcParams {
-  int kind, in_dim, out_dim, w_is_bf16, NB, K;
+  int kind, in_dim, out_dim, w_is_bf16, NB;
+  int K1, K1p, K2, K2p;   // rows of W behind X1 / X2, and the same rounded up to whole k-blocks (the padding is zero)
   const void *W;
-  void *B;   // bf16 [NB, K]  or  fp32 [2, NB, K] (hi, lo)
+  void *B;   // bf16 [NB, K1p + K2p]  or  fp32 [2, NB, K1p + K2p] (hi, lo)
 };
 
 __global__ void prep_weights_tc_kernel(PrepTcParams p) {
-  const int64_t total = (int64_t)p.NB * p.K;
+  const int Kp = p.K1p + p.K2p;
+  const int64_t total = (int64_t)p.NB * Kp;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    const int n = (int)(i / p.K), k = (int)(i % p.K);
+    const int n = (int)(i / Kp), kp = (int)(i % Kp);
+    // padded position -> row of the unpadded product (or none)
+    const bool second = kp >= p.K1p;
+    const int kin = second ? kp - p.K1p : kp;
+    const bool real = kin < (second ? p.K2 : p.K1);
+    const int k = second ? p.K1 + kin : kin;
     int64_t src;   // element of W that is B[k, n]
     if (p.kind == IT_PREP_SAGE_REORDER) src = n < p.out_dim ? (int64_t)k * p.out_dim + n : (int64_t)(p.in_dim + k) * p.out_dim + (n - p.out_dim);
     else src = (int64_t)k * p.out_dim + n;
     if (p.w_is_bf16) {
-      reinterpret_cast<__nv_bfloat16 *>(p.B)[i] = reinterpret_cast<const __nv_bfloat16 *>(p.W)[src];
+      reinterpret_cast<__nv_bfloat16 *>(p.B)[i] = real ? reinterpret_cast<const __nv_bfloat16 *>(p.W)[src] : __float2bfloat16_rn(0.f);
     } else {
-      const float w = reinterpret_cast<const float *>(p.W)[src];
+      const float w = real ? reinterpret_cast<const float *>(p.W)[src] : 0.f;
       // hi = w rounded to tf32 (nearest even on the 13 dropped bits), lo = the exact remainder
       uint32_t u = __float_as_uint(w);
       u += 0xfffu + ((u >> 13) & 1u);
@@ -602,7 +612,7 @@ constexpr int kSmemAux = 1024 /*alignment slack*/ + 288 /*barriers, TMEM slot, a
 }  // namespace
 
 size_t it_tc_weights_bytes(const it_layer_desc *L, int NB, int K) {
-  return (size_t)NB * K * (L->feat_dtype == IT_BF16 ? 2 : 8);
+  return (size_t)NB * (K + 128) * (L->feat_dtype == IT_BF16 ? 2 : 8);   // room for the padding of both operands' K
 }
 
 // Column split of the tensor-core path: the largest columns-per-CTA count (a multiple of 16
@@ -626,19 +636,22 @@ bool it_tc_supported(const it_gemm_args &a, int heads, int head_dim, bool want_s
   const int bk = TC_KBLOCK_BYTES / elem;
   if (a.M <= 0 || a.M > (int64_t)INT32_MAX) return false;
   const int K2 = a.X2 ? a.K2 : 0;
-  if (a.K1 <= 0 || a.K1 % bk != 0 || K2 % bk != 0) return false;
+  // operand rows must be TMA-addressable (a multiple of 16 bytes); a K that is not a whole number of k-blocks is
+  // padded: the TMA copy fills what lies beyond a row with zeros and the prepared weights carry zero rows there
+  if (a.K1 <= 0 || (a.K1 * elem) % 16 != 0 || (K2 * elem) % 16 != 0) return false;
   const int NB = a.n0 + a.n1;   // score columns are not materialised on this path
   if (NB <= 0 || NB % 16 != 0 || a.n0 % 16 != 0) return false;
   int n_splits, nbc;
-  if (!tc_split(tf32, NB, (a.K1 + K2) / bk, &n_splits, &nbc)) return false;
+  if (!tc_split(tf32, NB, (a.K1 + bk - 1) / bk + (K2 + bk - 1) / bk, &n_splits, &nbc)) return false;
   if (want_scores && (heads > 8 || head_dim % 16 != 0 || nbc % head_dim != 0)) return false;
   return true;
 }
 
-it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *L, int NB, int K, void *B, cudaStream_t st) {
+it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *L, int NB, int K1, int K2, void *B, cudaStream_t st) {
   PrepTcParams p;
+  const int bk = TC_KBLOCK_BYTES / (L->weight_dtype == IT_BF16 ? 2 : 4);
   p.kind = kind; p.in_dim = L->in_dim; p.out_dim = L->out_dim; p.w_is_bf16 = L->weight_dtype == IT_BF16;
-  p.NB = NB; p.K = K; p.W = L->W; p.B = B;
+  p.NB = NB; p.K1 = K1; p.K2 = K2; p.K1p = (K1 + bk - 1) / bk * bk; p.K2p = (K2 + bk - 1) / bk * bk; p.W = L->W; p.B = B;
   IT_LAUNCH(IT_K_PREP, 0, 0, st, prep_weights_tc_kernel<<<64, 256, 0, st>>>(p));
   IT_CUDA_TRY(cudaGetLastError());
   return IT_OK;
@@ -655,14 +668,15 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   const int NB = a.n0 + a.n1;
   const int K2 = a.X2 ? a.K2 : 0;
   const int K = a.K1 + K2;
-  const int KB = K / bk;
+  const int kb1 = (a.K1 + bk - 1) / bk, kb2 = (K2 + bk - 1) / bk;
+  const int KB = kb1 + kb2;
   int n_splits = 1, nbc = NB;
   IT_REQUIRE(tc_split(tf32, NB, KB, &n_splits, &nbc), IT_ERR_UNSUPPORTED, "tensor-core apply: cannot tile %d columns with K = %d", NB, K);
   const int b_bytes = (tf32 ? 2 : 1) * KB * nbc * TC_KBLOCK_BYTES;
   const int stage_bytes = TC_BM * TC_KBLOCK_BYTES;             // one operand tile (fp32 mode: the raw tile)
   const int const_bytes = nbc * 4 * (scores ? 3 : 1);          // bias (+ attention vectors) of this CTA's columns
   int stages = (kSmemBudget - kSmemAux - const_bytes - b_bytes) / stage_bytes;
-  if (stages > 8) stages = 8;
+  if (stages > IT_TC_MAX_STAGES) stages = IT_TC_MAX_STAGES;
   IT_REQUIRE(stages >= 2, IT_ERR_UNSUPPORTED, "tensor-core apply: no room for two operand stages");
   const int smem = b_bytes + stages * stage_bytes + kSmemAux + const_bytes;
   // fp32 mode: TMEM holds two accumulators of 2 nbc columns; what is left of its 512 columns stages the split A
@@ -674,11 +688,11 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   IT_TRY(make_map(&m1, a.X1, elem, a.M, a.K1, TC_BM));
   if (a.X2) IT_TRY(make_map(&m2, a.X2, elem, a.M, K2, TC_BM));
   else m2 = m1;
-  IT_TRY(make_map(&mb, B, elem, (int64_t)(tf32 ? 2 : 1) * NB, K, nbc));
+  IT_TRY(make_map(&mb, B, elem, (int64_t)(tf32 ? 2 : 1) * NB, (int64_t)KB * bk, nbc));
 
   TcParams p;
   p.M = a.M; p.n_tiles_m = (int)((a.M + TC_BM - 1) / TC_BM); p.n_splits = n_splits; p.nbc = nbc;
-  p.kb1 = a.K1 / bk; p.kb2 = K2 / bk; p.NB = NB; p.stages = stages; p.tstages = tstages;
+  p.kb1 = kb1; p.kb2 = kb2; p.NB = NB; p.stages = stages; p.tstages = tstages;
   p.n0 = a.n0; p.out0 = a.out0; p.out0_bf16 = a.dt0 == IT_BF16; p.bias0 = a.bias0; p.act0 = a.act0;
   p.n1 = a.n1; p.out1 = a.out1; p.out1_bf16 = a.dt1 == IT_BF16;
   p.scores = scores; p.att_src = att_src; p.att_dst = att_dst; p.heads = heads; p.head_dim = head_dim > 0 ? head_dim : 1;

@@ -101,6 +101,22 @@ struct it_graph {
 };
 
 static inline size_t it_align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// ELU on the device.  The negative branch is exp(x) - 1 with the hardware exponential: its absolute error stays
+// below 1e-6 (the result lies in (-1, 0)), far inside the parity bounds of both storage types, and it costs a
+// handful of instructions where expm1f costs a few dozen in the end-of-row code of every short row.
+#ifndef IT_FAST_ELU
+#define IT_FAST_ELU 1
+#endif
+#ifdef __CUDACC__
+__device__ __forceinline__ float it_elu(float x) {
+#if IT_FAST_ELU
+  return x > 0.f ? x : __expf(x) - 1.f;
+#else
+  return x > 0.f ? x : expm1f(x);
+#endif
+}
+#endif
 static inline int it_dtype_size(it_dtype t) { return t == IT_F32 ? 4 : 2; }
 
 // ----------------------------------------------------------------------------- gather.cu
@@ -116,14 +132,16 @@ struct it_gather_args {
   it_gather_op op;         // SUM / MEAN / MAX
   int use_edge_weights;
   it_dtype dtype;          // of src rows and of dst rows
-  int dim;                 // row length in elements
-  const void *src;         // [n, dim] rows that are gathered
+  int dim;                 // elements of a row that are gathered (any multiple of 16 bytes)
+  const void *src;         // rows that are gathered: row u starts at src + u * src_ld elements
+  int src_ld;              // 0 means dim
   int per_edge_rows;       // 1: src is [n_edges, dim] and row j belongs to edge j (edge features); 0: rows are looked up by source vertex
   float *partials;         // [n_partial_rows, dim] fp32 scratch (may be NULL when nothing is split)
   void *dst;               // row v starts at dst + v * dst_ld elements and takes dim of them
   int dst_ld;              // 0 means dim
   it_epilogue_kind epi;
-  const float *self_term;  // [n, dim] fp32, IT_EPI_ADD_ACT only
+  const float *self_term;  // fp32, IT_EPI_ADD_ACT only: row v starts at self_term + v * self_ld
+  int self_ld;             // 0 means dim
   const float *bias;       // [dim] fp32 or NULL, IT_EPI_BIAS_ACT only
   it_act act;              // IT_EPI_ADD_ACT and IT_EPI_BIAS_ACT
 };
@@ -171,12 +189,12 @@ it_status it_launch_prep_weights(it_prep_kind kind, const it_layer_desc *layer, 
                                  cudaStream_t stream);
 
 // ----------------------------------------------------------------------------- apply_tc.cu
-// The same product on the tensor cores (tcgen05 + TMEM + TMA).  Needs K1, K2 multiples of 128
-// bytes and n0, n0 + n1 multiples of 16; computes the n0 + n1 columns and, for GAT, the
+// The same product on the tensor cores (tcgen05 + TMEM + TMA).  Needs operand rows that are multiples of 16
+// bytes (K1, K2 are padded to whole 128-byte k-blocks with zeros) and n0, n0 + n1 multiples of 16; computes the n0 + n1 columns and, for GAT, the
 // attention scores [M, 2*heads] in its epilogue (a.B, a.NB and a.out2 are not used).  B is the
-// matrix written by it_launch_prep_weights_tc: bf16 [NB, K] or fp32 [2, NB, K] (hi, lo), K-major.
+// matrix written by it_launch_prep_weights_tc: bf16 [NB, Kp] or fp32 [2, NB, Kp] (hi, lo), K-major, Kp = padded K1 + padded K2.
 bool it_tc_supported(const it_gemm_args &a, int heads, int head_dim, bool want_scores);
-it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *layer, int NB, int K, void *B,
+it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *layer, int NB, int K1, int K2, void *B,
                                     cudaStream_t stream);
 it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *att_src, const float *att_dst,
                             int heads, int head_dim, float *scores, int num_sms, int *status, cudaStream_t stream);

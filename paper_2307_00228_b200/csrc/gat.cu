@@ -177,6 +177,7 @@ it_status it_launch_gat(const it_gat_args &a, cudaStream_t st) {
   StreamParams sp;
   sp.meta = g->bucket_meta; sp.owner = g->bucket_owner; sp.indices = g->indices; sp.weights = nullptr;
   sp.src = a.z; sp.row_lo = sp.row_hi = 0; sp.dim = a.heads * a.head_dim; sp.batch_rows = 1;
+  sp.src_pitch = (uint32_t)(sp.dim * it_dtype_size(a.dtype));
   if (a.dtype == IT_F32) IT_TRY(launch_gat<float>(a, sp, st));
   else IT_TRY(launch_gat<__nv_bfloat16>(a, sp, st));
   if (g->n_split_owners > 0) {

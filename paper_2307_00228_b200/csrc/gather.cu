@@ -21,7 +21,7 @@ struct SagePolicy {
   void *__restrict__ dst;
   const float *__restrict__ self_term;
   const float *__restrict__ bias;
-  int dim, dst_ld, is_mean, epi, act;
+  int dim, dst_ld, self_ld, is_mean, epi, act;   // dim: width of this column chunk; *_ld: row lengths of dst / the self term
   // per-thread
   int col;
   float self[VEC];
@@ -49,7 +49,7 @@ struct SagePolicy {
   }
   // the matching slice of the self term is fetched when the row starts, so that end_row does not wait for it
   __device__ __forceinline__ void begin_row(int32_t dest, int32_t) {
-    if (epi == IT_EPI_ADD_ACT && dest >= 0) load_floats_stream<VEC>(self_term + (int64_t)dest * dim + col, self);
+    if (epi == IT_EPI_ADD_ACT && dest >= 0) load_floats_stream<VEC>(self_term + (int64_t)dest * self_ld + col, self);
   }
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t len) const {
     if (RED != RED_SUM && len == 0) {
@@ -88,7 +88,7 @@ struct CombineParams {
   const float *__restrict__ self_term;
   const float *__restrict__ bias;
   int64_t n_split_owners;
-  int dim, dst_ld;
+  int dim, dst_ld, self_ld;
   int red, is_mean, epi, act;   // red: RED_SUM / RED_MAX / RED_MIN
 };
 
@@ -124,10 +124,9 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
       }
       for (; g < n; ++g) fold(__ldg(reinterpret_cast<const float4 *>(p.partials + (p0 + g) * p.dim + c)));
       float o[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
-      const int64_t off = v * p.dim + c;
       const int64_t doff = v * p.dst_ld + c;
       if (p.epi == IT_EPI_ADD_ACT) {
-        float4 s = __ldg(reinterpret_cast<const float4 *>(p.self_term + off));
+        float4 s = __ldg(reinterpret_cast<const float4 *>(p.self_term + v * p.self_ld + c));
         o[0] = act_apply(o[0] + s.x, p.act); o[1] = act_apply(o[1] + s.y, p.act);
         o[2] = act_apply(o[2] + s.z, p.act); o[3] = act_apply(o[3] + s.w, p.act);
       } else if (p.epi == IT_EPI_BIAS_ACT) {
@@ -149,7 +148,7 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
 template <typename T, int SB, int LPR, int RED, bool WEIGHTED>
 it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   SagePolicy<T, SB, RED, WEIGHTED> pol;
-  pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim; pol.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim;
+  pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim; pol.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; pol.self_ld = a.self_ld > 0 ? a.self_ld : a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
   const it_graph *g = a.g;
   // algorithmic bytes: per edge the index, the optional weight and one source row; per row its
@@ -174,23 +173,22 @@ it_status launch_lpr(const it_gather_args &a, StreamParams sp, cudaStream_t st) 
 
 }  // namespace
 
-it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
+// One column chunk of the rows: `a.dim` is the chunk's width (a power of two between 16 and 512 bytes), the
+// pointers already point at its first column, and the *_ld fields / src_ld carry the full row lengths.
+static it_status launch_gather_chunk(const it_gather_args &a, cudaStream_t st) {
   const it_graph *g = a.g;
-  IT_REQUIRE(a.op == IT_GATHER_SUM || a.op == IT_GATHER_MEAN || a.op == IT_GATHER_MAX || a.op == IT_GATHER_MIN, IT_ERR_INVALID_ARG,
-             "gather: bad op");
-  IT_REQUIRE(!a.use_edge_weights || g->edge_weights, IT_ERR_INVALID_ARG, "layer uses edge weights but the graph has none");
-  IT_REQUIRE(g->n_partial_rows == 0 || a.partials, IT_ERR_WORKSPACE, "gather: no partial buffer");
-  if (g->n == 0) return IT_OK;
   StreamParams sp;
   sp.meta = g->bucket_meta; sp.owner = nullptr; sp.indices = a.per_edge_rows ? nullptr : g->indices; sp.weights = g->edge_weights;
   sp.src = a.src; sp.row_lo = sp.row_hi = 0; sp.dim = a.dim; sp.batch_rows = 1;
+  sp.src_pitch = (uint32_t)((a.src_ld > 0 ? a.src_ld : a.dim) * it_dtype_size(a.dtype));
   if (a.dtype == IT_F32) IT_TRY(launch_lpr<float>(a, sp, st));
   else IT_TRY(launch_lpr<__nv_bfloat16>(a, sp, st));
   if (g->n_split_owners > 0) {
     CombineParams c;
     c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.shadow_indptr = g->shadow_indptr;
     c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.bias = a.bias; c.n_split_owners = g->n_split_owners;
-    c.dim = a.dim; c.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
+    c.dim = a.dim; c.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; c.self_ld = a.self_ld > 0 ? a.self_ld : a.dim;
+    c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
     int64_t want = (g->n_split_owners + 7) / 8;
     int64_t cap = (int64_t)g->num_sms * 8;
     unsigned blocks = (unsigned)(want < cap ? want : cap);
@@ -198,6 +196,39 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
                           (double)g->n_split_owners * a.dim * (a.dtype == IT_F32 ? 4.0 : 2.0);
     if (a.dtype == IT_F32) IT_LAUNCH(IT_K_COMBINE, cbytes, 0, st, combine_kernel<float><<<blocks, GATHER_THREADS, 0, st>>>(c));
     else IT_LAUNCH(IT_K_COMBINE, cbytes, 0, st, combine_kernel<__nv_bfloat16><<<blocks, GATHER_THREADS, 0, st>>>(c));
+  }
+  return IT_OK;
+}
+
+// Rows of any multiple of 16 bytes: the kernels take rows of 16, 32, ..., 512 bytes, so a wider or odd row is cut
+// into column chunks of those widths (largest first) and each chunk is gathered on its own, reading and writing
+// its columns in place.  The aggregate is entry by entry, so the chunks are independent; each pass re-reads
+// the edge indices (4 bytes against a chunk of up to 512 per edge).
+it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
+  const it_graph *g = a.g;
+  IT_REQUIRE(a.op == IT_GATHER_SUM || a.op == IT_GATHER_MEAN || a.op == IT_GATHER_MAX || a.op == IT_GATHER_MIN, IT_ERR_INVALID_ARG,
+             "gather: bad op");
+  IT_REQUIRE(!a.use_edge_weights || g->edge_weights, IT_ERR_INVALID_ARG, "layer uses edge weights but the graph has none");
+  IT_REQUIRE(g->n_partial_rows == 0 || a.partials, IT_ERR_WORKSPACE, "gather: no partial buffer");
+  const int es = it_dtype_size(a.dtype);
+  IT_REQUIRE(a.dim > 0 && (a.dim * es) % 16 == 0, IT_ERR_INVALID_ARG, "gather: a row of %d bytes is not a multiple of 16", a.dim * es);
+  if (g->n == 0) return IT_OK;
+  const int full = a.dim;
+  int c0 = 0;   // first column of the chunk
+  while (c0 < full) {
+    int bytes = 512;
+    while (bytes > (full - c0) * es) bytes >>= 1;
+    it_gather_args c = a;
+    c.dim = bytes / es;
+    c.src = (const char *)a.src + (size_t)c0 * es;
+    c.src_ld = a.src_ld > 0 ? a.src_ld : full;
+    c.dst = (char *)a.dst + (size_t)c0 * es;
+    c.dst_ld = a.dst_ld > 0 ? a.dst_ld : full;
+    c.self_term = a.self_term ? a.self_term + c0 : nullptr;
+    c.self_ld = a.self_ld > 0 ? a.self_ld : full;
+    c.bias = a.bias ? a.bias + c0 : nullptr;
+    IT_TRY(launch_gather_chunk(c, st));
+    c0 += c.dim;
   }
   return IT_OK;
 }

@@ -389,8 +389,7 @@ extern "C" it_status it_graph_set_edge_features(it_graph *g, const void *edge_fe
   }
   IT_REQUIRE(dtype == IT_F32 || dtype == IT_BF16, IT_ERR_INVALID_ARG, "bad edge feature dtype");
   const int64_t row = (int64_t)edge_dim * it_dtype_size(dtype);
-  IT_REQUIRE(edge_dim > 0 && row >= 16 && row <= 512 && (row & (row - 1)) == 0, IT_ERR_INVALID_ARG,
-             "an edge-feature row must be 16, 32, 64, 128, 256 or 512 bytes (got %lld)", (long long)row);
+  IT_REQUIRE(edge_dim > 0 && row % 16 == 0, IT_ERR_INVALID_ARG, "an edge-feature row must be a multiple of 16 bytes (got %lld)", (long long)row);
   IT_REQUIRE(((uintptr_t)edge_feat % 16) == 0, IT_ERR_INVALID_ARG, "edge features must be 16-byte aligned");
   g->edge_feat = edge_feat; g->edge_dim = edge_dim; g->edge_dtype = dtype;
   return IT_OK;

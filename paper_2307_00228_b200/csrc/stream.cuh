@@ -142,7 +142,7 @@ __device__ __forceinline__ void load_floats_stream(const float *p, float (&v)[VE
 
 __device__ __forceinline__ float act_apply(float x, int act) {
   if (act == IT_ACT_RELU) return fmaxf(x, 0.f);
-  if (act == IT_ACT_ELU) return x > 0.f ? x : expm1f(x);
+  if (act == IT_ACT_ELU) return it_elu(x);
   return x;
 }
 
@@ -154,7 +154,8 @@ struct StreamParams {
   const float *__restrict__ weights;
   const void *__restrict__ src;           // [n, dim] rows that are gathered ([n_edges, dim] when indices is NULL)
   int64_t row_lo, row_hi;                 // range inside the bucket-ordered row list
-  int dim;
+  int dim;                                // elements of a row that are gathered (one column chunk of the source rows)
+  uint32_t src_pitch;                     // bytes from one source row to the next (>= dim elements)
   int batch_rows;                         // rows a lane group takes at a time (<= LPR)
 };
 
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
   const int64_t groups_total = (int64_t)gridDim.x * (THREADS / G);
   const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * SB;
   using Slice = RowSlice<T, SB>;
-  const uint32_t row_bytes = (uint32_t)p.dim * (uint32_t)sizeof(T);
+  const uint32_t row_bytes = p.src_pitch;
 
   for (int64_t b = (int64_t)blockIdx.x * (THREADS / G) + threadIdx.x / G; b < n_batches; b += groups_total) {
     // ---- batch metadata: lane t owns row t of the batch
@@ -311,7 +312,7 @@ __global__ void __launch_bounds__(THREADS, IT_SHORT_MIN_BLOCKS) stream_short_row
   const int t = lane % LPR, gbase = lane - t;
   pol.setup(t);
   const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * 16;
-  constexpr uint32_t ROWB = LPR * 16;
+  const uint32_t ROWB = p.src_pitch;
   const int64_t rows_per_sweep = (int64_t)gridDim.x * (THREADS / LPR);
   // warp-uniform loop: every group of the warp takes one row per iteration
   for (int64_t i0 = p.row_lo + (int64_t)blockIdx.x * (THREADS / LPR) + (threadIdx.x >> 5) * (32 / LPR); i0 < p.row_hi; i0 += rows_per_sweep) {
@@ -368,7 +369,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_cta_kern
   pol.setup(t);
   const char *my_src = reinterpret_cast<const char *>(p.src) + (size_t)t * SB;
   using Slice = RowSlice<T, SB>;
-  const uint32_t row_bytes = (uint32_t)p.dim * (uint32_t)sizeof(T);
+  const uint32_t row_bytes = p.src_pitch;
   for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {
     const it_row_meta m = load_meta(p.meta + i);
     const int32_t owner = Policy::NEEDS_OWNER ? __ldcs(p.owner + i) : 0;

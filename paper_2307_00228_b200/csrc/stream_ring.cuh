@@ -52,7 +52,7 @@ __device__ __forceinline__ float lds_f32(uint32_t a) {
 template <int SB, int LPR>
 struct RingGeom {
   static constexpr int SL = 32 / LPR;                        // edge slots: rows a warp moves per instruction
-  static constexpr int ROWB = LPR * SB;                      // bytes of a feature row
+  static constexpr int ROWB = LPR * SB;                      // bytes of a row that are gathered (the source rows may be wider)
   static constexpr int GB = 32 * SB;                         // bytes of a group: what one instruction moves
   static constexpr int R = IT_RING_STAGE_ROWS * (16 / SB);   // groups per stage
   static constexpr int GE = R * SL;                          // edges per stage
@@ -71,9 +71,11 @@ struct RingWarp {
   using Raw = typename SliceRaw<SB>::type;
   uint32_t my_ring, my_xring;   // shared-window addresses of my slice / my per-edge scalar in group 0 of stage 0
   const char *my_src;           // my slice of source row 0
+  uint32_t pitch;               // bytes from one source row to the next
   int slot;
 
-  __device__ __forceinline__ void setup(uint32_t ring_base, const void *src, int lane) {
+  __device__ __forceinline__ void setup(uint32_t ring_base, const void *src, uint32_t src_pitch, int lane) {
+    pitch = src_pitch;
     my_ring = ring_base + lane * SB;
     my_xring = ring_base + G::S * G::R * G::GB + lane * 4;
     my_src = reinterpret_cast<const char *>(src) + (size_t)(lane % LPR) * SB;
@@ -87,14 +89,14 @@ struct RingWarp {
 #pragma unroll
       for (int u = 0; u < G::R; ++u) {
         const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u * G::SL + slot);
-        cp_async_slice<SB>(d + u * G::GB, my_src + (uint64_t)s * G::ROWB);
+        cp_async_slice<SB>(d + u * G::GB, my_src + (uint64_t)s * pitch);
         if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
       }
     } else {
       for (int u = 0; u * G::SL < n; ++u) {
         const uint32_t s = (uint32_t)__shfl_sync(0xffffffffu, idxreg, k0 + u * G::SL + slot);
         if (u * G::SL + slot < n) {
-          cp_async_slice<SB>(d + u * G::GB, my_src + (uint64_t)s * G::ROWB);
+          cp_async_slice<SB>(d + u * G::GB, my_src + (uint64_t)s * pitch);
           if (Policy::HAS_EXTRA) cp_async_slice<4>(dx + u * 128, pol.extra_ptr(s));
         }
       }
@@ -199,7 +201,7 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_
   const int lane = threadIdx.x & 31;
   RingWarp<T, SB, LPR, Policy> rw;
   rw.setup((uint32_t)__cvta_generic_to_shared(ring_raw) + (uint32_t)(threadIdx.x >> 5) * (uint32_t)ring_bytes_per_warp<SB, Policy::HAS_EXTRA>(),
-           p.src, lane);
+           p.src, p.src_pitch, lane);
   const int slot = rw.slot;
   pol.setup(lane % LPR);
   const int64_t n_rows = p.row_hi - p.row_lo;
@@ -281,7 +283,7 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_cta_ring_k
   __shared__ float red[WARPS][LPR][NS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   RingWarp<T, SB, LPR, Policy> rw;
-  rw.setup((uint32_t)__cvta_generic_to_shared(ring_raw) + (uint32_t)warp * (uint32_t)ring_bytes_per_warp<SB, Policy::HAS_EXTRA>(), p.src, lane);
+  rw.setup((uint32_t)__cvta_generic_to_shared(ring_raw) + (uint32_t)warp * (uint32_t)ring_bytes_per_warp<SB, Policy::HAS_EXTRA>(), p.src, p.src_pitch, lane);
   pol.setup(lane % LPR);
 
   for (int64_t i = p.row_lo + blockIdx.x; i < p.row_hi; i += gridDim.x) {

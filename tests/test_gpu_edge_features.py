@@ -31,7 +31,8 @@ def test_sage_layer_with_edge_features(dtype, op, threshold):
 
 
 @pytest.mark.parametrize("dtype,fi,de", [("f32", 32, 4), ("f32", 64, 64), ("f32", 128, 128), ("f32", 16, 8),
-                                         ("bf16", 64, 8), ("bf16", 64, 64), ("bf16", 128, 128), ("bf16", 32, 256)])
+                                         ("bf16", 64, 8), ("bf16", 64, 64), ("bf16", 128, 128), ("bf16", 32, 256),
+                                         ("f32", 100, 12), ("bf16", 72, 40)])
 def test_every_edge_row_width(dtype, fi, de):
     for op in ("mean", "max"):
         layer = make_sage_layer(3, op, "none", fi, 32, dtype, edge_dim=de)
