@@ -50,6 +50,9 @@
 #ifndef IT_SHORT_MIN_BLOCKS
 #define IT_SHORT_MIN_BLOCKS 4   // resident CTAs per SM of the short-row kernel (eight 16-byte slices in flight per lane)
 #endif
+#ifndef IT_SHORT_EDGES
+#define IT_SHORT_EDGES 8         // source rows a lane of the short-row kernel has in flight per round
+#endif
 #ifndef IT_SHORT_BELOW
 #define IT_SHORT_BELOW 32       // 128-byte rows: buckets of rows up to this long take the short-row kernel
 #endif
@@ -305,7 +308,7 @@ __global__ void __launch_bounds__(THREADS, IT_GATHER_MIN_BLOCKS) stream_rows_ker
 template <typename T, int LPR, class Policy>
 __global__ void __launch_bounds__(THREADS, IT_SHORT_MIN_BLOCKS) stream_short_rows_kernel(StreamParams p, Policy pol) {
   constexpr int NS = Policy::NS;
-  constexpr int E = 8;   // edges per round
+  constexpr int E = IT_SHORT_EDGES;   // edges per round
   static_assert(LPR >= E, "lanes 0..7 of a group fetch the indices of a round");
   using Slice = RowSlice<T, 16>;
   const int lane = threadIdx.x & 31;
