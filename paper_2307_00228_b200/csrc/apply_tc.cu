@@ -30,6 +30,18 @@ constexpr int TC_BM = 128;          // rows per tile (UMMA M)
 constexpr int TC_KBLOCK_BYTES = 128;  // one swizzle row of K per k-block
 constexpr int TC_EPI_WARPS = 16;      // four warps per TMEM lane quarter, each takes every fourth 16-column group
 constexpr int TC_THREADS_BF16 = 64 + 32 * TC_EPI_WARPS;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2-17 epilogue
+#ifndef IT_TC_EPI_BACKOFF
+#define IT_TC_EPI_BACKOFF 128   // ns the epilogue warps sleep between polls of the accumulator barrier
+#endif
+#ifndef IT_TC_TMA_BACKOFF
+#define IT_TC_TMA_BACKOFF 64    // ns the TMA producer sleeps between polls of a stage's empty barrier
+#endif
+#ifndef IT_TC_EPI_GROUPS
+#define IT_TC_EPI_GROUPS 2   // staged epilogue: groups of epilogue warps that take alternate tiles (1 or 2)
+#endif
+#ifndef IT_TC_TMA_STORE
+#define IT_TC_TMA_STORE 1   // 0: always store the results straight from registers
+#endif
 #ifndef IT_TC_MAX_STAGES
 #define IT_TC_MAX_STAGES 8   // operand stages in shared memory (as many as fit, up to this)
 #endif
@@ -82,6 +94,40 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
       : "memory");
+}
+// TMA store of one 128-byte-swizzled panel [128 rows x 128 bytes] from shared memory; rows past the end of the
+// tensor are clipped by the copy engine.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void *src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Named barriers of the epilogue warps (immediate operands): barrier 1 over all sixteen warps, or barriers 1 and 2
+// over the eight warps of a group.  The reducing form also tells every thread whether any of them failed.
+__device__ __forceinline__ void epi_bar_sync(int groups, int group) {
+  if (groups == 1) asm volatile("bar.sync 1, %0;" ::"n"(32 * TC_EPI_WARPS) : "memory");
+  else if (group == 0) asm volatile("bar.sync 1, %0;" ::"n"(16 * TC_EPI_WARPS) : "memory");
+  else asm volatile("bar.sync 2, %0;" ::"n"(16 * TC_EPI_WARPS) : "memory");
+}
+#define IT_EPI_BAR_RED(ID, N)                                                        \
+  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"                 \
+               "bar.red.or.pred q, " #ID ", %2, p;\n\t"                              \
+               "selp.u32 %0, 1, 0, q;\n\t}"                                          \
+               : "=r"(r)                                                             \
+               : "r"((uint32_t)flag), "n"(N)                                         \
+               : "memory")
+__device__ __forceinline__ bool epi_bar_any(int groups, int group, bool flag) {
+  uint32_t r;
+  if (groups == 1) IT_EPI_BAR_RED(1, 32 * TC_EPI_WARPS);
+  else if (group == 0) IT_EPI_BAR_RED(1, 16 * TC_EPI_WARPS);
+  else IT_EPI_BAR_RED(2, 16 * TC_EPI_WARPS);
+  return r != 0;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols));
@@ -160,12 +206,16 @@ struct TcParams {
   int n1; void *out1; int out1_bf16;
   float *scores; const float *att_src; const float *att_dst; int heads, head_dim;  // GAT: scores [M, 2*heads]
   int *status;                    // set to 1 if a bounded wait gave up
+  int tma_store;                  // 1: the epilogue stages each output tile in shared memory and writes it with TMA stores
+  int out_panels;                 // 16 KB panels of one staging tile (128 rows x 128 bytes each)
+  int epi_groups;                 // staged epilogue: 1, or 2 groups of eight warps that take alternate tiles (one staging tile each)
 };
 
 template <bool TF32>
 __global__ void __launch_bounds__(TF32 ? TC_THREADS_TF32 : TC_THREADS_BF16, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant__ CUtensorMap map_x2,
-               const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+               const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_o0,
+               const __grid_constant__ CUtensorMap map_o1, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = p.kb1 + p.kb2;
@@ -173,11 +223,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   const int b_bytes = (TF32 ? 2 : 1) * KB * b_tile_bytes;
   constexpr int a_tile_bytes = TC_BM * TC_KBLOCK_BYTES;          // 16 KB
 
-  // shared memory: resident weights | operand stages (bf16 tiles the MMAs read, or raw fp32 tiles the split warps read) | barriers
+  // shared memory: resident weights | operand stages (bf16 tiles the MMAs read, or raw fp32 tiles the split warps read) |
+  // output staging panels | barriers
   unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char *smem_b = base;
   unsigned char *smem_a = base + b_bytes;   // b_bytes is a multiple of 1024 (nbc is a multiple of 16)
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_a + (size_t)p.stages * a_tile_bytes);
+  unsigned char *smem_out = smem_a + (size_t)p.stages * a_tile_bytes;   // output staging panels (TMA-store epilogue), 1024-byte aligned
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_out + (size_t)p.out_panels * p.epi_groups * a_tile_bytes);
   uint64_t *full = bars;                    // [stages]  TMA landed
   uint64_t *empty = bars + p.stages;        // [stages]  the stage's readers are done (bf16: its MMAs; fp32: the split warps)
   uint64_t *ready = bars + 2 * p.stages;    // [TC_TSTAGES_MAX]  (fp32 mode) hi / lo parts written to TMEM
@@ -209,7 +261,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
     mbar_init(b_full, 1);
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], TC_EPI_WARPS);
+      mbar_init(&acc_empty[a], p.tma_store ? TC_EPI_WARPS / p.epi_groups : TC_EPI_WARPS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -252,7 +304,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile / p.n_splits) * TC_BM;
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, 64);
+          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, IT_TC_TMA_BACKOFF);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[stage], (uint32_t)a_tile_bytes);
           if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x1, kb * bk_elems, m0, &full[stage]);
@@ -330,10 +382,149 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
     const int gph = p.scores ? p.head_dim / 16 : 1;          // 16-column groups per ownership unit
     const int n_units = (p.nbc / 16) / gph;                   // units in this CTA's columns
     const int unit0 = p.scores ? col_base / p.head_dim : 0;   // global index of the first unit (head)
+    if (p.tma_store) {
+      // ---- staged epilogue: every warp converts its 16-column groups and drops them, 128-byte-swizzled, into the
+      // panels of the staging tile; one thread then writes each panel with a TMA store (whole 128-byte lines, and
+      // per lane only: TMEM load, bias, activation, pack, shared-memory store).  The output columns of this CTA
+      // are a run of out0 columns [lo0, hi0) and a run of out1 columns; each run is a whole number of panels.
+      const int s0 = p.out0_bf16 ? 2 : 4, s1 = p.out1_bf16 ? 2 : 4;
+      const int lo0 = col_base < p.n0 ? col_base : p.n0;
+      const int hi0 = (col_base + p.nbc) < p.n0 ? (col_base + p.nbc) : p.n0;
+      const int lo1 = col_base > p.n0 ? col_base : p.n0;
+      const int hi1 = (col_base + p.nbc) < n01 ? (col_base + p.nbc) : n01;
+      const int pan0 = hi0 > lo0 ? ((hi0 - lo0) * s0) / 128 : 0;
+      const int pan1 = hi1 > lo1 ? ((hi1 - lo1) * s1) / 128 : 0;
+      // With two groups, group g takes the tiles that land in accumulator g, so that the epilogues of two tiles run
+      // side by side (one tile's epilogue is a chain of latencies: barrier, TMEM loads, shared-memory stores, fence).
+      const int G = p.epi_groups, wpg = TC_EPI_WARPS / G;   // groups, warps per group
+      const int group = (warp - 2) / wpg;
+      const int gsub = ((warp - 2) % wpg) >> 2, n_sub = wpg >> 2;   // this warp's column sub-set inside its group
+      unsigned char *my_out = smem_out + (size_t)group * p.out_panels * a_tile_bytes;
+      const uint32_t out_base = smem_u32(my_out) + (uint32_t)row_in_tile * 128u;
+      const uint32_t swz = (uint32_t)(row_in_tile & 7);
+      const bool issuer = (warp - 2) % wpg == 0 && lane == 0;
+      int last_u = -1;   // the last unit this warp owns (ownership: (unit0 + u) % n_sub == gsub)
+      for (int u = n_units - 1; u >= 0; --u)
+        if ((unit0 + u) % n_sub == gsub) { last_u = u; break; }
+      int it = 0;   // tiles of this CTA so far: tile `it` uses accumulator it % 2, for the (it / 2)-th time
+      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+        if (G == 2 && (it & 1) != group) continue;
+        acc = (uint32_t)it & 1u;
+        acc_phase = ((uint32_t)it >> 1) & 1u;
+        const int m0 = (tile / p.n_splits) * TC_BM;
+        const int64_t m = (int64_t)m0 + row_in_tile;
+        ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, IT_TC_EPI_BACKOFF);
+        if (issuer) tma_store_wait_read();   // the stores of this group's previous tile have read the staging tile
+        // one decision for all warps of the group (they meet at named barriers below, so none may leave alone)
+        __syncwarp();
+        if (epi_bar_any(G, group, !ok)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * acc_cols;
+        bool released = false;
+        for (int u = 0; u < n_units; ++u) {
+          if ((unit0 + u) % n_sub != gsub) continue;
+          float sc_a = 0.f, sc_b = 0.f;   // attention scores of this head
+          for (int j0 = 0; j0 < gph; ++j0) {
+            const int c = (u * gph + j0) * 16;   // local column of the group
+            const int gc = col_base + c;         // global column; a group never straddles an output segment
+            uint32_t r[16];
+            tmem_ld16(taddr + (uint32_t)c, r);
+            if (TF32) {
+              uint32_t r2[16];
+              tmem_ld16(taddr + (uint32_t)(p.nbc + c), r2);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+            } else {
+              tmem_ld_wait();
+            }
+            if (u == last_u && j0 + 1 == gph) {   // everything this warp needs is in registers: hand the accumulator back
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&acc_empty[acc]);
+              released = true;
+            }
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+            if (p.scores) {   // GAT: attention scores from the unrounded accumulators
+              const float4 *as4 = reinterpret_cast<const float4 *>(att_s + c);
+              const float4 *ad4 = reinterpret_cast<const float4 *>(att_s + p.nbc + c);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float4 a4 = as4[i], d4 = ad4[i];
+                sc_a = fmaf(v[4 * i], a4.x, sc_a); sc_a = fmaf(v[4 * i + 1], a4.y, sc_a);
+                sc_a = fmaf(v[4 * i + 2], a4.z, sc_a); sc_a = fmaf(v[4 * i + 3], a4.w, sc_a);
+                sc_b = fmaf(v[4 * i], d4.x, sc_b); sc_b = fmaf(v[4 * i + 1], d4.y, sc_b);
+                sc_b = fmaf(v[4 * i + 2], d4.z, sc_b); sc_b = fmaf(v[4 * i + 3], d4.w, sc_b);
+              }
+            }
+            if (gc >= n01) continue;
+            int bf16, boff;   // output type, byte offset of the group inside the staging row of this CTA
+            if (gc < p.n0) {
+              const float4 *bs = reinterpret_cast<const float4 *>(bias_s + c);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float4 b4 = bs[i];
+                v[4 * i] += b4.x; v[4 * i + 1] += b4.y; v[4 * i + 2] += b4.z; v[4 * i + 3] += b4.w;
+              }
+              if (p.act0 == IT_ACT_RELU) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+              } else if (p.act0 == IT_ACT_ELU) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = it_elu(v[i]);
+              }
+              bf16 = p.out0_bf16; boff = (gc - lo0) * s0;
+            } else {
+              bf16 = p.out1_bf16; boff = pan0 * 128 + (gc - lo1) * s1;
+            }
+            // panel = boff / 128 (16 KB each), 16-byte chunk inside the row = (boff % 128) / 16, swizzled by the row
+            const uint32_t pbase = out_base + (uint32_t)(boff >> 7) * (uint32_t)a_tile_bytes;
+            const uint32_t ch = (uint32_t)(boff & 127) >> 4;
+            if (bf16) {
+              uint32_t w[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                w[i] = *reinterpret_cast<uint32_t *>(&h2);
+              }
+              st_shared_v4(pbase + (((ch + 0) ^ swz) << 4), w[0], w[1], w[2], w[3]);
+              st_shared_v4(pbase + (((ch + 1) ^ swz) << 4), w[4], w[5], w[6], w[7]);
+            } else {
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                st_shared_v4(pbase + (((ch + q) ^ swz) << 4), __float_as_uint(v[4 * q]), __float_as_uint(v[4 * q + 1]),
+                             __float_as_uint(v[4 * q + 2]), __float_as_uint(v[4 * q + 3]));
+            }
+          }
+          if (p.scores && m < p.M) {
+            const int h = unit0 + u;
+            p.scores[m * 2 * p.heads + h] = sc_a;
+            p.scores[m * 2 * p.heads + p.heads + h] = sc_b;
+          }
+        }
+        if (!released) {   // a warp that owns no columns of this CTA still has to sign off
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA store's reads
+        epi_bar_sync(G, group);
+        if (issuer) {
+          for (int k = 0; k < pan0; ++k)
+            tma_store_2d(&map_o0, my_out + (size_t)k * a_tile_bytes, lo0 + k * (128 / s0), m0);
+          for (int k = 0; k < pan1; ++k)
+            tma_store_2d(&map_o1, my_out + (size_t)(pan0 + k) * a_tile_bytes, (lo1 - p.n0) + k * (128 / s1), m0);
+          tma_store_commit();
+        }
+      }
+      if (issuer) tma_store_wait_all();   // the staging tile must outlive the last stores
+    } else
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const int64_t m = (int64_t)(tile / p.n_splits) * TC_BM + row_in_tile;
       const int64_t m_even = m - (odd ? 1 : 0), m_odd = m_even + 1;   // the two rows a lane pair writes together
-      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, 128);
+      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, IT_TC_EPI_BACKOFF);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -675,10 +866,32 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   const int b_bytes = (tf32 ? 2 : 1) * KB * nbc * TC_KBLOCK_BYTES;
   const int stage_bytes = TC_BM * TC_KBLOCK_BYTES;             // one operand tile (fp32 mode: the raw tile)
   const int const_bytes = nbc * 4 * (scores ? 3 : 1);          // bias (+ attention vectors) of this CTA's columns
-  int stages = (kSmemBudget - kSmemAux - const_bytes - b_bytes) / stage_bytes;
+  // Staged epilogue (TMA stores): possible when, for every column split, the out0 columns and the out1 columns of
+  // the CTA are whole 128-byte panels that start on a panel boundary, and three operand stages still fit beside
+  // the staging tile (three stages already give the time of eight).
+  const int s0 = a.dt0 == IT_BF16 ? 2 : 4, s1 = a.dt1 == IT_BF16 ? 2 : 4;
+  int out_panels = 0;
+  bool staged = IT_TC_TMA_STORE != 0;
+  for (int sp = 0; sp < n_splits && staged; ++sp) {
+    const int cb = sp * nbc, ce = cb + nbc;
+    const int lo0 = cb < a.n0 ? cb : a.n0, hi0 = ce < a.n0 ? ce : a.n0;
+    const int lo1 = cb > a.n0 ? cb : a.n0, hi1 = ce < NB ? ce : NB;
+    const int b0 = hi0 > lo0 ? (hi0 - lo0) * s0 : 0, b1 = hi1 > lo1 ? (hi1 - lo1) * s1 : 0;
+    if (b0 % 128 != 0 || b1 % 128 != 0 || (b0 > 0 && (lo0 * s0) % 128 != 0) || (b1 > 0 && ((lo1 - a.n0) * s1) % 128 != 0)) staged = false;
+    if (b0 / 128 + b1 / 128 > out_panels) out_panels = b0 / 128 + b1 / 128;
+  }
+  // two groups of epilogue warps (alternate tiles, a staging tile each) when the second staging tile still fits
+  int epi_groups = IT_TC_EPI_GROUPS;
+  if (staged && epi_groups == 2 && (kSmemBudget - kSmemAux - const_bytes - b_bytes - 2 * out_panels * stage_bytes) / stage_bytes < 3) {
+    epi_groups = 1;
+    if (!tf32) staged = false;   // measured: one group beats the direct stores in fp32 mode only (its tiles take long enough)
+  }
+  if (staged && (kSmemBudget - kSmemAux - const_bytes - b_bytes - epi_groups * out_panels * stage_bytes) / stage_bytes < 3) staged = false;
+  if (!staged) { out_panels = 0; epi_groups = 1; }
+  int stages = (kSmemBudget - kSmemAux - const_bytes - b_bytes - epi_groups * out_panels * stage_bytes) / stage_bytes;
   if (stages > IT_TC_MAX_STAGES) stages = IT_TC_MAX_STAGES;
   IT_REQUIRE(stages >= 2, IT_ERR_UNSUPPORTED, "tensor-core apply: no room for two operand stages");
-  const int smem = b_bytes + stages * stage_bytes + kSmemAux + const_bytes;
+  const int smem = b_bytes + (stages + epi_groups * out_panels) * stage_bytes + kSmemAux + const_bytes;
   // fp32 mode: TMEM holds two accumulators of 2 nbc columns; what is left of its 512 columns stages the split A
   int tstages = tf32 ? (512 - 4 * nbc) / TC_TSTAGE_COLS : 0;
   if (tstages > TC_TSTAGES_MAX) tstages = TC_TSTAGES_MAX;
@@ -689,6 +902,9 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   if (a.X2) IT_TRY(make_map(&m2, a.X2, elem, a.M, K2, TC_BM));
   else m2 = m1;
   IT_TRY(make_map(&mb, B, elem, (int64_t)(tf32 ? 2 : 1) * NB, (int64_t)KB * bk, nbc));
+  CUtensorMap mo0 = m1, mo1 = m1;   // placeholders unless the epilogue is staged
+  if (staged && a.n0 > 0) IT_TRY(make_map(&mo0, a.out0, s0, a.M, a.n0, TC_BM));
+  if (staged && a.n1 > 0) IT_TRY(make_map(&mo1, a.out1, s1, a.M, a.n1, TC_BM));
 
   TcParams p;
   p.M = a.M; p.n_tiles_m = (int)((a.M + TC_BM - 1) / TC_BM); p.n_splits = n_splits; p.nbc = nbc;
@@ -697,6 +913,7 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   p.n1 = a.n1; p.out1 = a.out1; p.out1_bf16 = a.dt1 == IT_BF16;
   p.scores = scores; p.att_src = att_src; p.att_dst = att_dst; p.heads = heads; p.head_dim = head_dim > 0 ? head_dim : 1;
   p.status = status;
+  p.tma_store = staged ? 1 : 0; p.out_panels = out_panels; p.epi_groups = epi_groups;
 
   const int64_t n_tiles = (int64_t)p.n_tiles_m * n_splits;
   int64_t grid = (int64_t)(num_sms / n_splits) * n_splits;
@@ -707,10 +924,10 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   const double flops = 2.0 * (double)a.M * K * NB;
   if (tf32) {
     IT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    IT_LAUNCH(IT_K_GEMM_TC, bytes, flops, st, gemm_tc_kernel<true><<<(unsigned)grid, TC_THREADS_TF32, smem, st>>>(m1, m2, mb, p));
+    IT_LAUNCH(IT_K_GEMM_TC, bytes, flops, st, gemm_tc_kernel<true><<<(unsigned)grid, TC_THREADS_TF32, smem, st>>>(m1, m2, mb, mo0, mo1, p));
   } else {
     IT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    IT_LAUNCH(IT_K_GEMM_TC, bytes, flops, st, gemm_tc_kernel<false><<<(unsigned)grid, TC_THREADS_BF16, smem, st>>>(m1, m2, mb, p));
+    IT_LAUNCH(IT_K_GEMM_TC, bytes, flops, st, gemm_tc_kernel<false><<<(unsigned)grid, TC_THREADS_BF16, smem, st>>>(m1, m2, mb, mo0, mo1, p));
   }
   IT_CUDA_TRY(cudaGetLastError());
   return IT_OK;
