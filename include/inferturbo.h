@@ -232,6 +232,16 @@ it_status it_layer_forward_static(const it_graph *g, const it_layer_desc *layer,
  */
 it_status it_graph_check(it_graph *g, void *stream);
 
+/*
+ * it_debug_expire_wait — test hook for those bounded waits (no counterpart in the paper): launches the tensor-core
+ * apply on a 128 x 64 operand of `dtype` with its copy producer switched off and a wait limit of a few thousand polls, so
+ * that every wait inside the kernel runs out.  The kernel must then drain and return by itself; afterwards
+ * it_graph_check reports IT_ERR_TIMEOUT once, and the library goes on working.  x: device [128, 64];
+ * out: device [128, 64] (left undefined); workspace: device, 256-byte aligned, at least 64 KB.
+ */
+it_status it_debug_expire_wait(it_graph *g, it_dtype dtype, const void *x, void *out, void *workspace, size_t workspace_bytes,
+                               void *stream);
+
 /* Frees the library-owned arrays of the graph.  NULL is accepted. */
 it_status it_graph_destroy(it_graph *g);
 

@@ -25,7 +25,7 @@ IT_MAX_BUCKETS = 8
 EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspace_bytes", "it_layer_forward",
            "it_infer", "it_graph_destroy", "it_status_string", "it_last_error_message", "it_profile_begin",
            "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static", "it_graph_check",
-           "it_graph_set_edge_features"]
+           "it_graph_set_edge_features", "it_debug_expire_wait"]
 
 
 class ItError(RuntimeError):
@@ -266,6 +266,15 @@ def it_graph_check(g: Graph, stream=None):
     L.it_graph_check.restype = C.c_int
     L.it_graph_check.argtypes = [C.c_void_p, C.c_void_p]
     _check(L.it_graph_check(g.handle, _stream(stream)))
+
+
+def it_debug_expire_wait(g: Graph, x: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """Test hook: run the tensor-core apply with its producer off so that its bounded waits run out."""
+    L = lib()
+    L.it_debug_expire_wait.restype = C.c_int
+    L.it_debug_expire_wait.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    _check(L.it_debug_expire_wait(g.handle, _dt(x.dtype), _ptr(x), _ptr(out), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def it_graph_destroy(g: Graph):

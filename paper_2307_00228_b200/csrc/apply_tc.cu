@@ -50,7 +50,10 @@ constexpr int TC_THREADS_BF16 = 64 + 32 * TC_EPI_WARPS;   // warp 0 TMA, warp 1 
 #endif
 constexpr int TC_SPLIT_GROUPS = IT_TC_SPLIT_GROUPS;
 constexpr int TC_THREADS_TF32 = TC_THREADS_BF16 + 128 * TC_SPLIT_GROUPS;   // ... plus the warps splitting A into hi / lo
-constexpr int TC_TSTAGES_MAX = 4;     // fp32 mode: split A tiles in flight in TMEM
+#ifndef IT_TC_TSTAGES_MAX
+#define IT_TC_TSTAGES_MAX 4
+#endif
+constexpr int TC_TSTAGES_MAX = IT_TC_TSTAGES_MAX;     // fp32 mode: split A tiles in flight in TMEM
 constexpr int TC_TSTAGE_COLS = 64;    // TMEM columns of one split A k-block: 32 of hi, 32 of lo
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
@@ -80,8 +83,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // Bounded wait.  Returns false if the CTA is aborting (or this wait ran out and started the abort).
 // `backoff_ns` > 0: sleep between polls, for roles whose waits are long and off the critical path (their polling
 // would otherwise take issue slots from the warps that feed the tensor core).
+// abort_flag[0] is the CTA's abort flag, abort_flag[1] the number of polls after which a wait gives up.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t backoff_ns = 0) {
-  for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it) {
+  const uint32_t limit = (uint32_t)abort_flag[1];
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (backoff_ns) __nanosleep(backoff_ns);
     if ((it & 63u) == 63u && *abort_flag) return false;
@@ -209,6 +214,8 @@ struct TcParams {
   int tma_store;                  // 1: the epilogue stages each output tile in shared memory and writes it with TMA stores
   int out_panels;                 // 16 KB panels of one staging tile (128 rows x 128 bytes each)
   int epi_groups;                 // staged epilogue: 1, or 2 groups of eight warps that take alternate tiles (one staging tile each)
+  uint32_t spin_limit;            // polls after which a wait on a barrier gives up
+  int no_loads;                   // test hook: the producer issues no copies, so every wait runs out
 };
 
 template <bool TF32>
@@ -240,7 +247,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   // per-column constants of this CTA's columns, 16-byte aligned: bias (0 where none applies), GAT attention vectors
-  float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // [nbc]
+  float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 3) + 15) & ~(uintptr_t)15);   // [nbc]
   float *att_s = bias_s + p.nbc;   // [2][nbc]: source vector, destination vector (only with scores)
 
   // fp32 mode: columns [nbc, 2 nbc) of an accumulator hold A_hi * B_lo, added to the first half by the epilogue
@@ -263,7 +270,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], p.tma_store ? TC_EPI_WARPS / p.epi_groups : TC_EPI_WARPS);
     }
-    *abort_flag = 0;
+    abort_flag[0] = 0;
+    abort_flag[1] = (int)p.spin_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -289,7 +297,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && !p.no_loads) {
       // the weights of this CTA's columns, once
       mbar_arrive_expect_tx(b_full, (uint32_t)b_bytes);
       const int bk_elems = TF32 ? 32 : 64;
@@ -914,6 +922,7 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   p.scores = scores; p.att_src = att_src; p.att_dst = att_dst; p.heads = heads; p.head_dim = head_dim > 0 ? head_dim : 1;
   p.status = status;
   p.tma_store = staged ? 1 : 0; p.out_panels = out_panels; p.epi_groups = epi_groups;
+  p.spin_limit = a.spin_limit ? a.spin_limit : TC_SPIN_LIMIT; p.no_loads = a.no_loads;
 
   const int64_t n_tiles = (int64_t)p.n_tiles_m * n_splits;
   int64_t grid = (int64_t)(num_sms / n_splits) * n_splits;
@@ -931,4 +940,20 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   }
   IT_CUDA_TRY(cudaGetLastError());
   return IT_OK;
+}
+
+// Test hook for the bounded waits: a 128 x 64 product (bf16, or fp32 with its operand-splitting warps) whose producer issues no copies, with waits that give up
+// after a few thousand polls.  Every role runs out of patience, the CTA drains, frees its TMEM and returns, and the
+// status word of the graph is set, which the next it_graph_check reports as IT_ERR_TIMEOUT.
+extern "C" it_status it_debug_expire_wait(it_graph *g, it_dtype dtype, const void *x, void *out, void *workspace, size_t workspace_bytes,
+                                           void *stream) {
+  IT_REQUIRE(g != nullptr && x != nullptr && out != nullptr && workspace != nullptr, IT_ERR_INVALID_ARG, "NULL argument");
+  IT_REQUIRE(workspace_bytes >= 64 * 1024 && ((uintptr_t)workspace % 256) == 0, IT_ERR_WORKSPACE, "needs 64 KB of aligned workspace");
+  it_gemm_args a{};
+  IT_REQUIRE(dtype == IT_F32 || dtype == IT_BF16, IT_ERR_INVALID_ARG, "bad dtype");
+  a.M = 128; a.x_dtype = dtype; a.X1 = x; a.K1 = 64; a.X2 = nullptr; a.K2 = 0; a.B = nullptr; a.NB = 64;
+  a.n0 = 64; a.out0 = out; a.dt0 = dtype; a.bias0 = nullptr; a.act0 = IT_ACT_NONE;
+  a.n1 = 0; a.out1 = nullptr; a.dt1 = dtype; a.out2 = nullptr;
+  a.spin_limit = 4096; a.no_loads = 1;
+  return it_launch_gemm_tc(a, workspace, nullptr, nullptr, 1, 64, nullptr, g->num_sms, g->d_status, (cudaStream_t)stream);
 }

@@ -179,6 +179,8 @@ struct it_gemm_args {
   int n0; void *out0; it_dtype dt0; const float *bias0; it_act act0;
   int n1; void *out1; it_dtype dt1;
   void *out2;
+  uint32_t spin_limit;   // tensor-core path: polls after which a barrier wait gives up (0 = the default)
+  int no_loads;          // tensor-core path, test hook: issue no operand copies
 };
 it_status it_launch_gemm(const it_gemm_args &a, cudaStream_t stream);
 

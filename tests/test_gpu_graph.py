@@ -123,3 +123,27 @@ def test_invalid_arguments():
     assert ei.value.status_name == "IT_ERR_INVALID_ARG"
     assert B.lib().it_split_hubs(None, 4, None, None, None) == 1
     assert B.lib().it_graph_destroy(None) == 0
+
+
+@pytest.mark.parametrize("tdtype", [torch.bfloat16, torch.float32])
+def test_a_wait_that_runs_out_is_reported_and_the_library_goes_on(tdtype):
+    """The tensor-core apply waits on hardware barriers with a poll limit.  With its copy producer switched off
+    every wait runs out: the kernel must return by itself, it_graph_check must say IT_ERR_TIMEOUT once, and a
+    real layer afterwards must still be right."""
+    from gpu_util import check_against_oracle, make_sage_layer, run_device, small_workload
+    layer = make_sage_layer(1, "sum", "relu", 64, 64, "bf16")
+    w = small_workload(2, 600, 12, "bf16", [layer])
+    got, d = run_device(w)
+    check_against_oracle(w, got)
+    x = torch.zeros((128, 64), dtype=tdtype, device="cuda")
+    o = torch.empty((128, 64), dtype=tdtype, device="cuda")
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    B.it_debug_expire_wait(d.graph, x, o, ws)
+    with pytest.raises(B.ItError) as e:
+        B.it_graph_check(d.graph)
+    assert e.value.status_name == "IT_ERR_TIMEOUT"
+    B.it_graph_check(d.graph)          # reported once
+    d.infer()
+    B.it_graph_check(d.graph)
+    from gpu_util import to_numpy
+    check_against_oracle(w, to_numpy(d.out))
