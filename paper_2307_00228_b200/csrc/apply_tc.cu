@@ -83,9 +83,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // Bounded wait.  Returns false if the CTA is aborting (or this wait ran out and started the abort).
 // `backoff_ns` > 0: sleep between polls, for roles whose waits are long and off the critical path (their polling
 // would otherwise take issue slots from the warps that feed the tensor core).
-// abort_flag[0] is the CTA's abort flag, abort_flag[1] the number of polls after which a wait gives up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t backoff_ns = 0) {
-  const uint32_t limit = (uint32_t)abort_flag[1];
+// `limit`: the number of polls after which the wait gives up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit, uint32_t backoff_ns = 0) {
   for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (backoff_ns) __nanosleep(backoff_ns);
@@ -247,7 +246,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   // per-column constants of this CTA's columns, 16-byte aligned: bias (0 where none applies), GAT attention vectors
-  float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 3) + 15) & ~(uintptr_t)15);   // [nbc]
+  float *bias_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // [nbc]
   float *att_s = bias_s + p.nbc;   // [2][nbc]: source vector, destination vector (only with scores)
 
   // fp32 mode: columns [nbc, 2 nbc) of an accumulator hold A_hi * B_lo, added to the first half by the epilogue
@@ -270,8 +269,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], p.tma_store ? TC_EPI_WARPS / p.epi_groups : TC_EPI_WARPS);
     }
-    abort_flag[0] = 0;
-    abort_flag[1] = (int)p.spin_limit;
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -312,7 +310,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile / p.n_splits) * TC_BM;
         for (int kb = 0; kb < KB; ++kb) {
-          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, IT_TC_TMA_BACKOFF);
+          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.spin_limit, IT_TC_TMA_BACKOFF);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[stage], (uint32_t)a_tile_bytes);
           if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x1, kb * bk_elems, m0, &full[stage]);
@@ -334,19 +332,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
       const uint32_t fmt = TF32 ? 2u : 1u;
       const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.nbc >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
       const uint32_t idesc_wide = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)((2 * p.nbc) >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
-      bool ok = mbar_wait(b_full, 0, abort_flag);
+      bool ok = mbar_wait(b_full, 0, abort_flag, p.spin_limit);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
       uint32_t ts = 0, tphase = 0;   // fp32 mode: TMEM stage of the split A k-block
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag);
+        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, p.spin_limit);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * acc_cols;
         for (int kb = 0; kb < KB; ++kb) {
           const uint32_t b_hi = smem_u32(smem_b + (size_t)kb * (TF32 ? 2 : 1) * b_tile_bytes);
           if (TF32) {
-            ok = mbar_wait(&ready[ts], tphase, abort_flag);
+            ok = mbar_wait(&ready[ts], tphase, abort_flag, p.spin_limit);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a_hi = tmem_base + a_col0 + ts * TC_TSTAGE_COLS, a_lo = a_hi + 32;
@@ -359,7 +357,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
             tc_commit(&a_free[ts]);   // TMEM stage reusable once these MMAs have read it
             if (++ts == (uint32_t)p.tstages) { ts = 0; tphase ^= 1u; }
           } else {
-            ok = mbar_wait(&full[stage], phase, abort_flag);
+            ok = mbar_wait(&full[stage], phase, abort_flag, p.spin_limit);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a_s = smem_u32(smem_a + (size_t)stage * a_tile_bytes);
@@ -421,7 +419,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
         acc_phase = ((uint32_t)it >> 1) & 1u;
         const int m0 = (tile / p.n_splits) * TC_BM;
         const int64_t m = (int64_t)m0 + row_in_tile;
-        ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, IT_TC_EPI_BACKOFF);
+        ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.spin_limit, IT_TC_EPI_BACKOFF);
         if (issuer) tma_store_wait_read();   // the stores of this group's previous tile have read the staging tile
         // one decision for all warps of the group (they meet at named barriers below, so none may leave alone)
         __syncwarp();
@@ -532,7 +530,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const int64_t m = (int64_t)(tile / p.n_splits) * TC_BM + row_in_tile;
       const int64_t m_even = m - (odd ? 1 : 0), m_odd = m_even + 1;   // the two rows a lane pair writes together
-      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, IT_TC_EPI_BACKOFF);
+      ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.spin_limit, IT_TC_EPI_BACKOFF);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -683,14 +681,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
             if (++ts == (uint32_t)p.tstages) { ts = 0; tphase ^= 1u; }
             continue;
           }
-          ok = mbar_wait(&full[stage], phase, abort_flag);
+          ok = mbar_wait(&full[stage], phase, abort_flag, p.spin_limit);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           const unsigned char *row_base = smem_a + (size_t)stage * a_tile_bytes + (size_t)row * TC_KBLOCK_BYTES;
           float4 x[8];
 #pragma unroll
           for (int c = 0; c < 8; ++c) x[c] = *reinterpret_cast<const float4 *>(row_base + ((c ^ (row & 7)) << 4));
-          ok = mbar_wait(&a_free[ts], tphase ^ 1u, abort_flag);
+          ok = mbar_wait(&a_free[ts], tphase ^ 1u, abort_flag, p.spin_limit);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
