@@ -710,16 +710,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
             tmem_st16(t_hi + half * 16, h);
             tmem_st16(t_lo + half * 16, l);
           }
+          // the MMA issuer is waiting for this: tell it first
+          tmem_st_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&ready[ts]);
           // Every value read from the stage has been used, so the reads are complete; the proxy fence orders these
           // generic-proxy reads before the asynchronous-proxy write of the TMA copy that refills the stage.
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
           if (lane == 0) mbar_arrive(&empty[stage]);
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
-          tmem_st_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&ready[ts]);
           if (++ts == (uint32_t)p.tstages) { ts = 0; tphase ^= 1u; }
         }
       }
