@@ -64,3 +64,19 @@ def test_reference_arm_under_two_ranks_prints_one_line():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_reference_arm_prints_one_contract_line():
+    """`bench.py --impl reference` times the CPU oracle on a bounded sample and prints one JSON line with the
+    keys the benchmark contract names (also with edge features in the messages)."""
+    for extra in ([], ["--edge-dim", "8"]):
+        out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                              "--steps", "2", "--warmup", "1", "--cpu-seconds", "1"] + extra,
+                             capture_output=True, text=True, check=True, cwd=ROOT).stdout.strip().splitlines()
+        assert len(out) == 1
+        d = json.loads(out[0])
+        assert d["impl"] == "reference" and d["unit"] == "vertices/s" and d["higher_is_better"] is True
+        assert d["steps"] == 2 and d["warmup"] == 1 and d["n_gpus"] == 1 and d["value"] > 0 and d["dtype"] == "f64"
+        assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["value"] == d["value"]
+        assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+        assert d["config"]["workload"] == "tiny" and d["config"]["edge_feature_dim"] == (8 if extra else 0)
