@@ -813,15 +813,17 @@ size_t it_tc_weights_bytes(const it_layer_desc *L, int NB, int K) {
   return (size_t)NB * (K + 128) * (L->feat_dtype == IT_BF16 ? 2 : 8);   // room for the padding of both operands' K
 }
 
-// Column split of the tensor-core path: the largest columns-per-CTA count (a multiple of 16
-// that divides NB, at most 256) whose resident weights fit in 128 KB of shared memory.
+// Column split of the tensor-core path: the largest columns-per-CTA count (a multiple of 16 that divides NB, at
+// most 256) whose resident weights leave room for three operand stages (which already give the time of eight)
+// and one 32 KB staging tile of the epilogue.
+constexpr size_t kWeightBudget = kSmemBudget - kSmemAux - 1024 /*per-column constants*/ - 3 * TC_BM * TC_KBLOCK_BYTES - 32 * 1024;
 static bool tc_split(bool tf32, int NB, int KB, int *n_splits, int *nbc) {
   for (int s = 1; s <= 16; ++s) {
     if (NB % s != 0) continue;
     const int c = NB / s;
     // fp32 mode issues MMAs of 2 c columns and keeps 4 c TMEM columns of accumulators next to the split A stages
     if (c % 16 != 0 || c > (tf32 ? 64 : 256)) continue;
-    if ((size_t)(tf32 ? 2 : 1) * KB * c * TC_KBLOCK_BYTES > 128 * 1024) continue;
+    if ((size_t)(tf32 ? 2 : 1) * KB * c * TC_KBLOCK_BYTES > kWeightBudget) continue;
     *n_splits = s; *nbc = c;
     return true;
   }
