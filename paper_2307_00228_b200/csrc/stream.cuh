@@ -56,6 +56,9 @@
 #ifndef IT_SHORT_ASYNC
 #define IT_SHORT_ASYNC 1         // 1: the short-row kernel stages its slices through shared memory with cp.async (0: in registers)
 #endif
+#ifndef IT_SHORT_256
+#define IT_SHORT_256 1           // 1: 256-byte rows of at most IT_SHORT_BELOW edges take the lane-group kernel too (16 lanes per row)
+#endif
 #ifndef IT_SHORT_BELOW
 #define IT_SHORT_BELOW 32       // 128-byte rows: buckets of rows up to this long take the short-row kernel
 #endif
@@ -542,7 +545,7 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
     } else {
       // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
       int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
-      if constexpr (SB == 16 && LPR == 8) {   // 128-byte rows
+      if constexpr (SB == 16 && (LPR == 8 || (LPR == 16 && IT_SHORT_256 != 0))) {   // 128-byte rows (and 256-byte rows)
         if (bound <= IT_SHORT_BELOW) {   // one lane group per row
           const int64_t short_max = (int64_t)g->num_sms * IT_SHORT_MIN_BLOCKS * 4;
           const int64_t want = (rows + (THREADS / LPR) - 1) / (THREADS / LPR);
@@ -592,6 +595,10 @@ it_status dispatch_row_bytes(int row_bytes, bool wide, F f) {
     case 512: return f.template operator()<16, 32>(-1, ALL);
     case 256:
       if (!wide) return f.template operator()<8, 32>(-1, ALL);
+      if (IT_SHORT_256) {   // every row with edges takes 16-byte slices (short rows: the lane-group kernel); <8, 32> keeps the empty rows
+        IT_TRY((f.template operator()<16, 16>(0, ALL)));
+        return f.template operator()<8, 32>(-1, 0);
+      }
       IT_TRY((f.template operator()<16, 16>(IT_WIDE_ABOVE, ALL)));
       return f.template operator()<8, 32>(-1, IT_WIDE_ABOVE);
     case 128:
