@@ -130,11 +130,11 @@ it_status it_graph_create(int64_t n_vertices, int64_t n_edges, const void *indpt
 it_status it_graph_set_edge_features(it_graph *g, const void *edge_feat, int32_t edge_dim, it_dtype dtype);
 
 /*
- * it_split_hubs — the shadow-node rule ("divide the edges into n groups evenly ... the id
- * of each mirror is appended with the group information", Section "Optimization
- * Strategies", Shadow Nodes) applied to the in-edge segment of every vertex whose
- * in-degree d exceeds `threshold` T, so that each group can be gathered on its own and
- * the partial results combined (Partial-Gather, same section).
+ * it_split_hubs — the shadow-node rule (Section "Optimization Strategies", Shadow Nodes: the
+ * edges of a hub are cut into n groups of equal size, one mirror per group, the mirror's id
+ * being the vertex id extended by the group number) applied to the in-edge segment of every
+ * vertex whose in-degree d exceeds `threshold` T, so that each group can be gathered on its
+ * own and the partial results combined (Partial-Gather, same section).
  *   n = 1 if d <= T (or T <= 0), else ceil(d / T) groups; group g takes the next
  *   d / n + (g < d % n) consecutive edges.  Row id = owner_indptr[v] + g.
  * Also builds the degree buckets: shadow rows partitioned stably by length class
@@ -173,8 +173,8 @@ it_status it_workspace_bytes(const it_graph *g, const it_layer_desc *layers, int
  *   h_in  [n, in_dim], h_out [n, out_dim], feat_dtype, device, must not overlap.
  *   workspace: device, 256-byte aligned, >= it_workspace_bytes(g, layer, 1).
  * If allow_reorder and op is SUM, MEAN or GCN and out_dim < in_dim, the neighbour transform is
- * done before the gather (the paper's "computation flow would be reorganized", Section
- * "Inference"): Z = h_in * W[in_dim:, :] is stored in feat_dtype and gathered instead of
+ * done before the gather (Section "Inference" allows the order of a layer's computation to be
+ * rearranged for speed): Z = h_in * W[in_dim:, :] is stored in feat_dtype and gathered instead of
  * h_in; the self term h_in * W[0:in_dim, :] + bias stays fp32.
  * Asynchronous on `stream`.  Results are bit-identical from run to run.
  */
@@ -182,8 +182,8 @@ it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const 
                            void *h_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * it_infer — L layers in order ("after k iterations we get the result of a k-layer
- * model", Section "InferTurbo on Graph Processing System"): exactly the sequence of
+ * it_infer — L layers in order (Section "InferTurbo on Graph Processing System": one layer
+ * per iteration over all vertices, a k-layer model after k of them): exactly the sequence of
  * it_layer_forward calls, intermediate layer outputs double-buffered inside the
  * workspace.  x [n, layers[0].in_dim]; out [n, layers[L-1].out_dim]; layers[i].out_dim must
  * equal layers[i+1].in_dim and all feat_dtype agree.  Bit-identical to calling
@@ -213,7 +213,10 @@ it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_lay
  * during set-up.)
  *
  * The first call on each device looks up the device address of the array (with that device
- * current) and caches it; make that first call during set-up, before any stream capture.
+ * current) and caches it, and the first launch of each kernel the library holds may make the
+ * CUDA runtime load that kernel, which can allocate inside the driver.  So make one call per
+ * layer shape and dtype during set-up, before any stream capture; calls after that leave the
+ * device's memory as they found it.
  * All calls on a device share the one array.  It keeps the previous call's contents; nothing
  * in it needs to start at zero, because every kernel writes the part it later reads.  Two
  * calls whose kernels can overlap on the GPU (different streams without an ordering between

@@ -14,7 +14,7 @@
  *     does its attention-weighted reduce in apply_node.
  *   - Section "Optimization Strategies": partial-gather (aggregate what is available
  *     for one destination first, aggregate the partial results afterwards) and shadow
- *     nodes (divide the edges of a hub into n groups evenly, one mirror per group, the
+ *     nodes (the edges of a hub are cut into n equal groups, one mirror per group, the
  *     mirror id carries the group number).
  *
  * The graph is CSR by destination: the in-edges of vertex v are the entries
@@ -38,8 +38,8 @@ enum { ITO_ACT_NONE = 0, ITO_ACT_RELU = 1, ITO_ACT_ELU = 2 };
 
 /* ------------------------------------------------------------------ index side */
 
-/* Shadow-node rule applied to in-edge segments ("divide the edges into n groups
- * evenly").  A vertex with in-degree d > T is split into n = ceil(d / T) groups; group g
+/* Shadow-node rule applied to in-edge segments (the edges of a hub are cut into n groups of
+ * equal size).  A vertex with in-degree d > T is split into n = ceil(d / T) groups; group g
  * takes the next contiguous run of base + (g < rem) edges, base = d / n, rem = d % n.
  * A vertex with d <= T (including d = 0) keeps exactly one row.  T <= 0: never split. */
 static int64_t groups_of(int64_t d, int64_t T) {
@@ -156,6 +156,29 @@ void ito_aggregate_edges(int64_t n_seg, const int64_t *segptr, const double *EF,
         }
         if (op == ITO_MEAN && j1 > j0)
             for (int32_t f = 0; f < De; ++f) a[f] /= (double)(j1 - j0);
+    }
+}
+
+/* apply_edge with a learned message function (Eq. (1): m_{v,u} = M(h_v, h_u, e_{v,u}); Section "InferTurbo
+ * Abstraction", Scatter stage: apply_edge makes the message of an edge out of the source's state and the edge's
+ * features).  Here M is one dense layer on the concatenation of the two, scaled by the optional edge weight:
+ *   m_j = w_j * act( h_{u_j} W_e[0:Fi, :] + e_j W_e[Fi:Fi+De, :] + b_e ),     W_e [Fi + De, Fm] row-major.
+ * De may be 0 (no edge features; EF unused), b_e and w may be NULL.  M is [n_edges, Fm], row j for CSR entry j;
+ * the Gather stage then reduces the rows of a destination with ito_aggregate_edges. */
+static double activate(double x, int32_t act);
+void ito_edge_messages(int64_t n_edges, const int32_t *indices, const double *w, const double *H, int32_t Fi,
+                       const double *EF, int32_t De, const double *We, const double *be, int32_t Fm, int32_t act,
+                       double *M) {
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n_edges; ++j) {
+        const double *h = H + (int64_t)indices[j] * Fi;
+        double *m = M + j * Fm;
+        for (int32_t c = 0; c < Fm; ++c) m[c] = be ? be[c] : 0.0;
+        for (int32_t k = 0; k < Fi; ++k)
+            for (int32_t c = 0; c < Fm; ++c) m[c] += h[k] * We[(int64_t)k * Fm + c];
+        for (int32_t k = 0; k < De; ++k)
+            for (int32_t c = 0; c < Fm; ++c) m[c] += EF[j * De + k] * We[(int64_t)(Fi + k) * Fm + c];
+        for (int32_t c = 0; c < Fm; ++c) m[c] = (w ? w[j] : 1.0) * activate(m[c], act);
     }
 }
 

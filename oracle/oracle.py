@@ -3,8 +3,8 @@
 Thin ctypes wrappers over `it_oracle.c` plus the layer-by-layer driver that strings
 them together the way the paper does: k layers = k passes over every vertex, each
 vertex used once per layer, no sampling (Section "Alternative Backends and
-Implementation Details", Execution: "after k iterations we get the result of a k-layer
-model").  Nothing here is shared with, or imported by, the CUDA library.
+Implementation Details", Execution: one iteration per layer, the k-layer result after k
+of them).  Nothing here is shared with, or imported by, the CUDA library.
 
 Storage points.  The method itself is exact, but a deployment stores layer inputs and
 outputs in a narrow type.  `storage=None` keeps everything in fp64 (mode A).  With
@@ -170,6 +170,17 @@ def aggregate_edges(segptr, EF, op: str):
     return AE
 
 
+def edge_messages(indices, w, H, EF, We, be, act: str):
+    """m_j = w_j act(h_{u_j} We[:Fi] + e_j We[Fi:] + be) for every CSR entry j: [n_edges, Fm]."""
+    indices, w, H, EF, We, be = _i32(indices), _f64(w), _f64(H), _f64(EF), _f64(We), _f64(be)
+    Fi, De = H.shape[1], (0 if EF is None else EF.shape[1])
+    assert We.shape[0] == Fi + De
+    M = np.empty((indices.shape[0], We.shape[1]), np.float64)
+    lib().ito_edge_messages(C.c_int64(indices.shape[0]), _p(indices), _p(w), _p(H), C.c_int32(Fi), _p(EF), C.c_int32(De),
+                            _p(We), _p(be), C.c_int32(We.shape[1]), C.c_int32(ACTS[act]), _p(M))
+    return M
+
+
 def linear(X, W):
     X, W = _f64(X), _f64(W)
     out = np.empty((X.shape[0], W.shape[1]), np.float64)
@@ -247,6 +258,38 @@ def _edge_dim(layer) -> int:
     return int(getattr(layer, "edge_dim", 0) or 0)
 
 
+def _msg_dim(layer) -> int:
+    return int(getattr(layer, "msg_dim", 0) or 0)
+
+
+def _message_aggregate(indptr, indices, w, H, ef, layer, storage, threshold):
+    """Aggregate of the learned messages m_j = w_j act_e(h_u W_e[:in] + e_j W_e[in:] + b_e) of a layer with
+    msg_dim > 0, over the in-edges of every vertex of `indptr`: [n, msg_dim].
+    storage=None: the definition, edge by edge (ito_edge_messages).  With a storage type the same value is built the
+    way the layer contract stores it: the per-source part P = H W_e[:in] and the per-edge part Q = e W_e[in:] + b_e
+    are rounded where they are stored, and so is the finished message act_e(P[u] + Q[j]); without edge features the
+    rounded table act_e(P + b_e) is the message itself.  The edge weight multiplies inside the reduce."""
+    We, be = _f64(layer.W_edge), _f64(getattr(layer, "bias_edge", None))
+    act_e = getattr(layer, "act_edge", "none")
+    Fi = layer.in_dim
+    op = "sum" if layer.op == "gcn" else layer.op
+    if storage is None:
+        M = edge_messages(indices, w, H, ef, We, be, act_e)
+    else:
+        need = np.unique(_i32(indices).astype(np.int64))
+        P = np.full((H.shape[0], We.shape[1]), np.nan)
+        if ef is None:
+            P[need] = round_to(bias_act(linear(H[need], We[:Fi]), be, act_e), storage)
+            M = P[_i32(indices).astype(np.int64)]
+        else:
+            P[need] = round_to(linear(H[need], We[:Fi]), storage)
+            Q = round_to(bias_act(linear(ef, We[Fi:]), be, "none"), storage)
+            M = round_to(bias_act(P[_i32(indices).astype(np.int64)] + Q, None, act_e), storage)
+        if w is not None:
+            M = M * _f64(w)[:, None]
+    return _gathered_edges(indptr, M, op, threshold)
+
+
 def _sources_of(indptr, indices, rows):
     """Sorted unique vertex ids that `rows` read: themselves and their in-neighbours."""
     sub, idx, _ = _sub_csr(indptr, indices, None, rows)
@@ -277,6 +320,13 @@ def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=
     else:
         indptr, indices, w = _sub_csr(indptr, indices, w, rows)
         Hself = H[_i64(rows)]
+    if _msg_dim(layer):   # learned per-edge messages: W is [in + msg_dim, out]
+        if reorder:
+            raise ValueError("layers with learned messages keep the plain order")
+        assert W.shape[0] == Fi + _msg_dim(layer)
+        A = round_to(_message_aggregate(indptr, indices, w, H, ef, layer, storage, threshold), storage)
+        out = bias_act(linear(Hself, W[:Fi]) + linear(A, W[Fi:]), layer.bias, layer.act)
+        return round_to(out, storage)
     if De:
         if reorder:
             raise ValueError("layers with edge features keep the plain order")
@@ -350,6 +400,17 @@ def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0
     W = _f64(layer.W)
     w = edge_weights if layer.use_edge_weights else None
     De = _edge_dim(layer)
+    if _msg_dim(layer):   # learned per-edge messages, summed; W is [msg_dim, out]
+        if reorder:
+            raise ValueError("layers with learned messages keep the plain order")
+        ef = _f64(edge_feat) if De else None
+        if rows is not None:
+            if De:
+                indptr, indices, w, ef = _sub_csr(indptr, indices, w, rows, ef)
+            else:
+                indptr, indices, w = _sub_csr(indptr, indices, w, rows)
+        A = round_to(_message_aggregate(indptr, indices, w, H, ef, layer, storage, threshold), storage)
+        return round_to(bias_act(linear(A, W), layer.bias, layer.act), storage)
     if De:   # message [w_e h_u | e_vu], summed; W is [in + edge_dim, out]
         if reorder:
             raise ValueError("layers with edge features keep the plain order")
@@ -386,31 +447,88 @@ def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, thresho
     return sage_layer(indptr, indices, edge_weights, H, layer, storage, threshold, reorder, rows, edge_feat)
 
 
+def layer_magnitude(indptr, indices, edge_weights, H, layer, rows=None, edge_feat=None):
+    """The sum of the ABSOLUTE values of the terms that make up every output entry of `layer` (before its
+    activation): the layer evaluated on |H|, |W|, |b|, |w_e| (|e_vu|), with a max / min pooling taken as the
+    largest |w_e h_u|, and for GAT the true attention weights applied to |h| |W|.  This is the quantity D of a
+    forward error bound |computed - exact| <= c u D for any order of evaluation (the terms of the reordered and
+    of the split forms are the same terms), and D >= |exact|: it serves as the denominator floor when a device
+    result is compared with the oracle.  Plain order, fp64, no storage rounding."""
+    H = _f64(H)
+    absw = None if edge_weights is None else np.abs(_f64(edge_weights))
+    abse = None if edge_feat is None else np.abs(_f64(edge_feat))
+    if layer.op == "gat":
+        # attention weights from the true scores; messages replaced by |h| |W|
+        if rows is None:
+            need, sub_ip, sub_ix = None, indptr, indices
+        else:
+            need = _sources_of(indptr, indices, rows)
+            sub_ip, sub_ix, _ = _sub_csr(indptr, indices, None, rows)
+        sel = slice(None) if need is None else need
+        z = linear(H[sel], _f64(layer.W))
+        zabs = np.full((H.shape[0], layer.out_dim), np.nan)
+        zabs[sel] = linear(np.abs(H[sel]), np.abs(_f64(layer.W)))
+        s_src = np.full((H.shape[0], layer.heads), np.nan)
+        s_src[sel] = gat_scores(z, layer.att_src, layer.heads)
+        if rows is None:
+            s_dst = gat_scores(z, layer.att_dst, layer.heads)
+        else:
+            s_dst = gat_scores(linear(H[_i64(rows)], _f64(layer.W)), layer.att_dst, layer.heads)
+        D = gat_aggregate(sub_ip, sub_ix, zabs, s_src, s_dst, layer.heads, layer.leaky_slope)
+        return D if layer.bias is None else D + np.abs(_f64(layer.bias))[None, :]
+
+    class _Abs:   # the same layer on absolute values, no activation
+        pass
+    a = _Abs()
+    a.op = "max" if layer.op in ("max", "min") else layer.op
+    a.act = "none"
+    a.in_dim, a.out_dim = layer.in_dim, layer.out_dim
+    a.W = np.abs(_f64(layer.W))
+    a.bias = None if layer.bias is None else np.abs(_f64(layer.bias))
+    a.use_edge_weights = layer.use_edge_weights
+    a.allow_reorder = False
+    a.edge_dim = _edge_dim(layer)
+    a.heads = 1
+    a.msg_dim = _msg_dim(layer)
+    if a.msg_dim:   # |act_e(x)| <= |x| for the activations offered, so the message is bounded by its terms' sum
+        a.W_edge = np.abs(_f64(layer.W_edge))
+        be = getattr(layer, "bias_edge", None)
+        a.bias_edge = None if be is None else np.abs(_f64(be))
+        a.act_edge = "none"
+    return layer_forward(indptr, indices, absw, np.abs(H), a, storage=None, threshold=0, reorder=False, rows=rows,
+                         edge_feat=abse)
+
+
 def will_reorder(layer) -> bool:
     """The layer contract: transform first when it shrinks the rows that are gathered and
     the aggregate is linear."""
     return (bool(layer.allow_reorder) and layer.op in ("sum", "mean", "gcn") and layer.out_dim < layer.in_dim
-            and _edge_dim(layer) == 0)
+            and _edge_dim(layer) == 0 and _msg_dim(layer) == 0)
 
 
-def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, follow_reorder=False, edge_feat=None):
-    """L layers in order over the whole graph; returns the list of every layer's output."""
+def infer(indptr, indices, edge_weights, X, layers, storage=None, threshold=0, follow_reorder=False, edge_feat=None,
+          magnitudes=False):
+    """L layers in order over the whole graph; returns the list of every layer's output.  With magnitudes=True
+    also the list of every layer's term magnitudes (layer_magnitude of the input that layer was given)."""
     H = _f64(X)
-    outs = []
+    outs, mags = [], []
     for layer in layers:
+        if magnitudes:
+            mags.append(layer_magnitude(indptr, indices, edge_weights, H, layer, edge_feat=edge_feat))
         H = layer_forward(indptr, indices, edge_weights, H, layer, storage, threshold,
                           reorder=follow_reorder and will_reorder(layer), edge_feat=edge_feat)
         outs.append(H)
-    return outs
+    return (outs, mags) if magnitudes else outs
 
 
 def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, threshold=0, follow_reorder=False,
-             edge_feat=None):
+             edge_feat=None, magnitudes=False):
     """The L-layer result at the vertices `targets` only, computed from their L-hop
     in-neighbourhood (which is sufficient and necessary for an L-layer model, Section
     "K-hop Neighborhood and Sampling"): layer l is evaluated only where layer l+1 reads it.
     Everything else stays NaN, so a read outside the neighbourhood would poison the result.
-    Returns [len(targets), out_dim] in the order of `targets`."""
+    Returns [len(targets), out_dim] in the order of `targets`; with magnitudes=True also the term magnitudes of
+    the last layer at the targets (layer_magnitude)."""
     targets = _i64(targets)
     need = [None] * (len(layers) + 1)
     need[len(layers)] = np.unique(targets)
@@ -418,12 +536,16 @@ def infer_at(indptr, indices, edge_weights, X, layers, targets, storage=None, th
         need[l] = _sources_of(indptr, indices, need[l + 1])
     H = _f64(X)
     n = H.shape[0]
+    D = None
     for l, layer in enumerate(layers, start=1):
+        if magnitudes and l == len(layers):
+            D = np.full((n, layer.out_dim), np.nan)
+            D[need[l]] = layer_magnitude(indptr, indices, edge_weights, H, layer, rows=need[l], edge_feat=edge_feat)
         out_rows = layer_forward(indptr, indices, edge_weights, H, layer, storage, threshold,
                                  reorder=follow_reorder and will_reorder(layer), rows=need[l], edge_feat=edge_feat)
         H = np.full((n, layer.out_dim), np.nan)
         H[need[l]] = out_rows
-    return H[targets]
+    return (H[targets], D[targets]) if magnitudes else H[targets]
 
 
 def compact_neighbourhood(indptr, indices, edge_weights, targets, n_layers, edge_feat=None):

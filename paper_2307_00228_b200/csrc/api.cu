@@ -238,6 +238,19 @@ bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
   return x < y + nb && y < x + na;
 }
 
+// What every forward call checks about the graph and its input / output matrices before anything is launched:
+// the kernels move 16-byte slices of the rows, so a pointer that is not 16-byte aligned would fault on the device.
+it_status check_io(const it_graph *g, const void *in, size_t in_bytes, const void *out, size_t out_bytes) {
+  IT_REQUIRE(g->n == 0 || g->bucket_meta != nullptr, IT_ERR_BAD_GRAPH,
+             "the graph has no row split (an it_split_hubs call failed): call it_split_hubs again before a forward pass");
+  if (g->n == 0) return IT_OK;
+  IT_REQUIRE(in != nullptr && out != nullptr, IT_ERR_INVALID_ARG, "input / output matrix is NULL");
+  IT_REQUIRE(((uintptr_t)in % 16) == 0 && ((uintptr_t)out % 16) == 0, IT_ERR_INVALID_ARG,
+             "input and output matrices must be 16-byte aligned (got %p, %p)", in, out);
+  IT_REQUIRE(!overlaps(in, in_bytes, out, out_bytes), IT_ERR_INVALID_ARG, "input and output matrices overlap");
+  return IT_OK;
+}
+
 }  // namespace
 
 extern "C" it_status it_workspace_bytes(const it_graph *g, const it_layer_desc *layers, int32_t n_layers,
@@ -253,11 +266,12 @@ extern "C" it_status it_layer_forward(const it_graph *g, const it_layer_desc *la
                                       void *workspace, size_t workspace_bytes, void *stream) {
   IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
   IT_TRY(check_layer(g, layer));
-  IT_REQUIRE((h_in && h_out) || g->n == 0, IT_ERR_INVALID_ARG, "h_in / h_out is NULL");
   IT_REQUIRE(workspace != nullptr && ((uintptr_t)workspace % 256) == 0, IT_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
   const size_t s = (size_t)it_dtype_size(layer->feat_dtype);
-  IT_REQUIRE(g->n == 0 || !overlaps(h_in, (size_t)g->n * layer->in_dim * s, h_out, (size_t)g->n * layer->out_dim * s),
-             IT_ERR_INVALID_ARG, "h_in and h_out overlap");
+  const size_t in_bytes = (size_t)g->n * layer->in_dim * s, out_bytes = (size_t)g->n * layer->out_dim * s;
+  IT_TRY(check_io(g, h_in, in_bytes, h_out, out_bytes));
+  IT_REQUIRE(g->n == 0 || (!overlaps(h_in, in_bytes, workspace, workspace_bytes) && !overlaps(h_out, out_bytes, workspace, workspace_bytes)),
+             IT_ERR_INVALID_ARG, "h_in / h_out overlaps the workspace");
   return layer_forward_impl(g, layer, h_in, h_out, (char *)workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
@@ -292,10 +306,8 @@ extern "C" it_status it_layer_forward_static(const it_graph *g, const it_layer_d
                                              void *h_out, void *stream) {
   IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
   IT_TRY(check_layer(g, layer));
-  IT_REQUIRE((h_in && h_out) || g->n == 0, IT_ERR_INVALID_ARG, "h_in / h_out is NULL");
   const size_t s = (size_t)it_dtype_size(layer->feat_dtype);
-  IT_REQUIRE(g->n == 0 || !overlaps(h_in, (size_t)g->n * layer->in_dim * s, h_out, (size_t)g->n * layer->out_dim * s),
-             IT_ERR_INVALID_ARG, "h_in and h_out overlap");
+  IT_TRY(check_io(g, h_in, (size_t)g->n * layer->in_dim * s, h_out, (size_t)g->n * layer->out_dim * s));
   IT_REQUIRE(!it_profile_is_on(), IT_ERR_UNSUPPORTED,
              "it_layer_forward_static does not run while instrumentation is on (it would create CUDA events)");
   const size_t need = plan_layer(g, layer).bytes;
@@ -311,9 +323,13 @@ extern "C" it_status it_infer(const it_graph *g, const it_layer_desc *layers, in
                               void *workspace, size_t workspace_bytes, void *stream) {
   InferWs w;
   IT_TRY(plan_infer(g, layers, n_layers, &w));
-  IT_REQUIRE((x && out) || g->n == 0, IT_ERR_INVALID_ARG, "x / out is NULL");
   IT_REQUIRE(workspace != nullptr && ((uintptr_t)workspace % 256) == 0, IT_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
   IT_REQUIRE(workspace_bytes >= w.bytes, IT_ERR_WORKSPACE, "workspace has %zu bytes, it_infer needs %zu", workspace_bytes, w.bytes);
+  const size_t es = (size_t)it_dtype_size(layers[0].feat_dtype);
+  const size_t x_bytes = (size_t)g->n * layers[0].in_dim * es, out_bytes = (size_t)g->n * layers[n_layers - 1].out_dim * es;
+  IT_TRY(check_io(g, x, x_bytes, out, out_bytes));
+  IT_REQUIRE(g->n == 0 || (!overlaps(x, x_bytes, workspace, workspace_bytes) && !overlaps(out, out_bytes, workspace, workspace_bytes)),
+             IT_ERR_INVALID_ARG, "x / out overlaps the workspace");
   char *ws = (char *)workspace;
   void *buf[2] = {ws + w.off_buf0, ws + w.off_buf1};
   const void *cur = x;

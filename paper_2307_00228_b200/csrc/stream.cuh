@@ -30,6 +30,8 @@
 //   void end_row(float (&st)[NS], int32_t dest, int32_t owner, int64_t len);
 #pragma once
 
+#include <atomic>
+
 #include "common.cuh"
 
 #ifndef IT_GATHER_UNROLL
@@ -506,6 +508,20 @@ __global__ void __launch_bounds__(THREADS) stream_empty_kernel(StreamParams p, P
 
 namespace it_stream {
 
+// The opt-in to more than 48 KB of dynamic shared memory is an attribute of the kernel ON ONE DEVICE: it is set once
+// per device (the current one), remembered in a bit mask that any thread may update.
+template <class Kernel>
+it_status allow_dynamic_smem(Kernel kernel, int smem, std::atomic<uint64_t> &done) {
+  int dev = -1;
+  IT_CUDA_TRY(cudaGetDevice(&dev));
+  const uint64_t bit = (dev >= 0 && dev < 64) ? (uint64_t)1 << dev : 0;   // ordinals beyond 63 are configured on every launch
+  if (bit == 0 || !(done.load(std::memory_order_acquire) & bit)) {
+    IT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    done.fetch_or(bit, std::memory_order_release);
+  }
+  return IT_OK;
+}
+
 // ----------------------------------------------------------------------------- bucket dispatch
 // Longest rows first so that the tail of the launch sequence is made of short rows.
 // bytes_of(bucket, rows) gives the algorithmic bytes of a launch; kid_* the instrumentation ids.
@@ -530,11 +546,8 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
     } else if (bound > IT_GATHER_CTA_ABOVE) {
       if constexpr (RING) {
         constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
-        static bool configured = false;   // per template instance
-        if (!configured) {
-          IT_CUDA_TRY(cudaFuncSetAttribute(stream_cta_ring_kernel<T, SB, LPR, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-          configured = true;
-        }
+        static std::atomic<uint64_t> configured{0};   // per template instance: one bit per device ordinal
+        IT_TRY(allow_dynamic_smem(stream_cta_ring_kernel<T, SB, LPR, Policy>, smem, configured));
         // one CTA per row as far as the grid allows: the hardware hands out rows as CTAs retire
         unsigned blocks = (unsigned)(rows < (1 << 20) ? rows : (1 << 20));
         IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_ring_kernel<T, SB, LPR, Policy><<<blocks, THREADS, smem, st>>>(p, pol));
@@ -556,11 +569,8 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
       }
       if constexpr (RING) {   // a whole warp per batch
         constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
-        static bool configured = false;   // per template instance
-        if (!configured) {
-          IT_CUDA_TRY(cudaFuncSetAttribute(stream_rows_ring_kernel<T, SB, LPR, Policy>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-          configured = true;
-        }
+        static std::atomic<uint64_t> configured{0};   // per template instance: one bit per device ordinal
+        IT_TRY(allow_dynamic_smem(stream_rows_ring_kernel<T, SB, LPR, Policy>, smem, configured));
         p.batch_rows = br;
         const int64_t batches = (rows + br - 1) / br;
         const int64_t ring_max = (int64_t)g->num_sms * IT_RING_MIN_BLOCKS * 2;

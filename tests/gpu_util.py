@@ -11,7 +11,7 @@ from paper_2307_00228_b200 import host
 from workloads import Layer, Workload, compare
 from workloads import rng as wrng
 
-TOL = {"f32": 1e-4, "bf16": 2e-2}   # max relative error: fp32 paths / bf16 apply paths
+TOL = compare.TOL   # max relative error: fp32 paths / bf16 apply paths
 
 
 def to_numpy(t: torch.Tensor) -> np.ndarray:
@@ -81,19 +81,30 @@ def run_device(w: Workload, int32_indptr=False, threshold=None):
     return to_numpy(d.out), d
 
 
-def run_oracle(w: Workload, storage="same", threshold=None):
+def run_oracle(w: Workload, storage="same", threshold=None, magnitudes=False):
     """Oracle over all layers.  storage='same': round at the storage points like the device
-    contract (mode B); storage=None: fp64 throughout (mode A)."""
+    contract (the gate); storage=None: fp64 throughout, plain order of operations."""
     st = w.dtype if storage == "same" else storage
     thr = w.threshold if threshold is None else threshold
     return O.infer(w.indptr, w.indices, w.edge_weights, w.x_as_f32(), w.layers, storage=st, threshold=thr,
-                   follow_reorder=True, edge_feat=w.edge_feat_as_f32())
+                   follow_reorder=st is not None, edge_feat=w.edge_feat_as_f32(), magnitudes=magnitudes)
 
 
-def check_against_oracle(w: Workload, got: np.ndarray, tol=None, label=""):
-    ref = run_oracle(w)[-1]
-    err = compare.rel_error(got, ref)
-    tol = TOL[w.dtype] if tol is None else tol
-    assert err["finite"], label
-    assert err["max_rel"] <= tol, (label, err)
+def assert_close(got, ref, mag, dtype, mode="stored", tol=None, label=""):
+    """The parity gate: every entry within tol of the reference relative to max(|ref|, floor * term magnitude),
+    and the plain relative error of the entries above the reference's rms within tol as well."""
+    err = compare.rel_error(got, ref, mag, compare.FLOOR[mode])
+    tol = TOL[dtype] if tol is None else tol
+    assert err["finite"], (label, err)
+    assert err["max_rel"] <= tol, (label, mode, err)
+    assert err["max_rel_plain"] <= tol, (label, mode, err)
+    return err
+
+
+def check_against_oracle(w: Workload, got: np.ndarray, tol=None, label="", exact=True):
+    outs, mags = run_oracle(w, magnitudes=True)
+    err = assert_close(got, outs[-1], mags[-1], w.dtype, "stored", tol, label)
+    if exact:   # and against the fp64-throughout oracle, which charges the storage roundings to the device
+        outs_a, mags_a = run_oracle(w, storage=None, magnitudes=True)
+        assert_close(got, outs_a[-1], mags_a[-1], w.dtype, "exact", tol, label)
     return err

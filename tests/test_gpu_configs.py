@@ -1,9 +1,10 @@
 """The five workload shapes through it_infer, against the oracle.
 
 Tiny runs at full size with a full-graph oracle.  The others run (a) shrunk, with a full-graph
-oracle, and (b) where they fit the test budget, at full size in the launch configuration the
-benchmark times, checked on sampled vertices that the oracle evaluates from their L-hop
-in-neighbourhood.
+oracle, and (b) at full size in the launch configuration the benchmark times, checked on sampled
+vertices that the oracle evaluates from their L-hop in-neighbourhood.  The 100M-vertex workload at
+full size needs ten minutes of host time to generate and check and is left to the benchmark, which
+runs the same sampled check on the result it has just timed; here it runs when IT_RUN_LARGE is set.
 """
 import os
 
@@ -11,7 +12,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import TOL, check_against_oracle, run_device, to_numpy
+from gpu_util import assert_close, check_against_oracle, run_device, to_numpy
 from oracle import oracle as O
 from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
@@ -25,11 +26,7 @@ def test_tiny_full_size():
     w = make("tiny")
     got, d = run_device(w)
     assert d.n_split_owners > 0
-    err = check_against_oracle(w, got)
-    # mode A (no rounding at storage points) is also within the fp32 bound
-    ref_a = O.infer(w.indptr, w.indices, None, w.x_as_f32(), w.layers, follow_reorder=False)[-1]
-    assert compare.rel_error(got, ref_a)["max_rel"] <= TOL["f32"]
-    assert err["max_rel"] <= TOL["f32"]
+    check_against_oracle(w, got)   # against the storage-rounding oracle and the fp64-throughout one
 
 
 @pytest.mark.parametrize("name,scale,int32", [("medium", 0.01, False), ("gat", 0.004, False), ("extreme", 0.005, False),
@@ -52,11 +49,12 @@ def sampled_targets(w, n_top, n_random, seed=5):
 
 
 def check_sampled(w, d, targets, label):
-    ref = O.infer_at(w.indptr, w.indices, w.edge_weights, w.x_as_f32(), w.layers, targets, storage=w.dtype,
-                     threshold=w.threshold, follow_reorder=True)
     got = to_numpy(d.out[torch.from_numpy(targets).cuda()])
-    err = compare.rel_error(got, ref)
-    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], (label, err)
+    for mode, storage in (("stored", w.dtype), ("exact", None)):
+        ref, mag = O.infer_at(w.indptr, w.indices, w.edge_weights, w.x_as_f32(), w.layers, targets, storage=storage,
+                              threshold=w.threshold, follow_reorder=storage is not None, magnitudes=True)
+        err = assert_close(got, ref, mag, w.dtype, mode, label=label)
+        print(f"{label} ({mode}):", err)
     # properties that hold at any size: finite everywhere, and identical on a second run
     assert bool(torch.isfinite(d.out.float()).all())
     first = d.out.clone()
@@ -85,24 +83,22 @@ def test_extreme_hub_rows_at_scale():
     check_sampled(w, d, sampled_targets(w, 3, 200), "extreme")
 
 
-FULL = pytest.mark.skipif(not (os.environ.get("IT_RUN_FULL") or os.environ.get("IT_RUN_LARGE")),
-                          reason="set IT_RUN_FULL=1: full-size GAT and Extreme take a few minutes of host time to generate and check")
-
-
-def check_compact(w, d, targets, label):
+def check_compact(w, d, targets, label, out=None, layers=None):
     """Sampled vertices of a big workload against the oracle evaluated on their L-hop in-neighbourhood,
     relabelled to a compact graph so that no full-size fp64 array is needed."""
-    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, w.edge_weights, targets, len(w.layers))
+    layers = w.layers if layers is None else layers
+    out = d.out if out is None else out
+    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, w.edge_weights, targets, len(layers))
     xc = w.x[ids] if w.dtype == "f32" else wrng.bf16_bits_to_f32(w.x[ids])
-    ref = O.infer_at(cip, cix, cw, xc, w.layers, ct, storage=w.dtype, threshold=w.threshold, follow_reorder=True)
-    got = to_numpy(d.out[torch.from_numpy(targets).cuda()])
-    err = compare.rel_error(got, ref)
-    print(f"{label} full size:", err, "rows", d.n_rows, "split owners", d.n_split_owners, "compact vertices", len(ids))
-    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], (label, err)
-    assert bool(torch.isfinite(d.out.float()).all())
+    got = to_numpy(out[torch.from_numpy(targets).cuda()])
+    for mode, storage in (("stored", w.dtype), ("exact", None)):
+        ref, mag = O.infer_at(cip, cix, cw, xc, layers, ct, storage=storage, threshold=w.threshold,
+                              follow_reorder=storage is not None, magnitudes=True)
+        err = assert_close(got, ref, mag, w.dtype, mode, label=label)
+        print(f"{label} full size ({mode}):", err, "rows", d.n_rows, "split owners", d.n_split_owners, "compact vertices", len(ids))
+    assert bool(torch.isfinite(out.float().sum()))
 
 
-@FULL
 def test_gat_full_size_sampled():
     """5M vertices, 100M edges, bf16, two GAT layers of 4 heads, hubs split at 4096 (partial softmax states
     merged): the two largest hubs and a random sample."""
@@ -114,7 +110,6 @@ def test_gat_full_size_sampled():
     check_compact(w, d, sampled_targets(w, 2, 200), "gat")
 
 
-@FULL
 def test_extreme_full_size_sampled():
     """20M vertices, 200M edges, 100 hubs of 1M in-edges (245 shadow rows each), bf16, three max-pooling layers.
     A hub's 3-hop in-neighbourhood is the whole graph, so the final output is checked on random vertices
@@ -144,12 +139,7 @@ def test_extreme_full_size_sampled():
     o1 = torch.empty((w.n, w.layers[0].out_dim), dtype=d.x.dtype, device="cuda")
     B.it_layer_forward(d.graph, d.layers[0], d.x, o1, d.workspace)
     B.it_graph_check(d.graph)
-    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, None, h3, 1)
-    ref = O.infer_at(cip, cix, cw, wrng.bf16_bits_to_f32(w.x[ids]), w.layers[:1], ct, storage=w.dtype,
-                     threshold=w.threshold, follow_reorder=True)
-    err = compare.rel_error(to_numpy(o1[torch.from_numpy(h3).cuda()]), ref)
-    print("extreme hubs after layer 1:", err)
-    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], err
+    check_compact(w, d, h3, "extreme hubs after layer 1", out=o1, layers=w.layers[:1])
 
 
 @pytest.mark.skipif(not os.environ.get("IT_RUN_LARGE"), reason="set IT_RUN_LARGE=1: needs ~100 GB of HBM, ~60 GB of host RAM and ~10 minutes")
@@ -160,11 +150,4 @@ def test_large_full_size_sampled():
     d = host.upload(w, int32_indptr=True)
     d.infer()
     B.it_graph_check(d.graph)
-    targets = sampled_targets(w, 2, 150)
-    ids, cip, cix, cw, ct = O.compact_neighbourhood(w.indptr, w.indices, None, targets, len(w.layers))
-    xc = wrng.bf16_bits_to_f32(w.x[ids])
-    ref = O.infer_at(cip, cix, cw, xc, w.layers, ct, storage=w.dtype, threshold=w.threshold, follow_reorder=True)
-    got = to_numpy(d.out[torch.from_numpy(targets).cuda()])
-    err = compare.rel_error(got, ref)
-    print("large full size:", err, "rows", d.n_rows, "split owners", d.n_split_owners)
-    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], err
+    check_compact(w, d, sampled_targets(w, 2, 150), "large")

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import TOL, check_against_oracle, make_plain_layer, make_sage_layer, run_device, small_workload, to_numpy
+from gpu_util import TOL, assert_close, check_against_oracle, make_plain_layer, make_sage_layer, run_device, small_workload, to_numpy
 from oracle import oracle as O
 from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
@@ -76,10 +76,11 @@ def test_medium_shape_with_edge_features_sampled():
                                         np.random.default_rng(5).choice(w.n, size=200, replace=False)]))
     ids, cip, cix, cw, ct, cef = O.compact_neighbourhood(w.indptr, w.indices, w.edge_weights, targets, len(w.layers),
                                                          edge_feat=w.edge_feat)
-    ref = O.infer_at(cip, cix, cw, w.x[ids], w.layers, ct, storage=w.dtype, threshold=w.threshold, follow_reorder=True,
-                     edge_feat=cef)
-    err = compare.rel_error(to_numpy(d.out[torch.from_numpy(targets).cuda()]), ref)
-    assert err["finite"] and err["max_rel"] <= TOL[w.dtype], err
+    got = to_numpy(d.out[torch.from_numpy(targets).cuda()])
+    for mode, storage in (("stored", w.dtype), ("exact", None)):
+        ref, mag = O.infer_at(cip, cix, cw, w.x[ids], w.layers, ct, storage=storage, threshold=w.threshold,
+                              follow_reorder=storage is not None, edge_feat=cef, magnitudes=True)
+        assert_close(got, ref, mag, w.dtype, mode)
     first = d.out.clone()
     d.infer()
     torch.cuda.synchronize()

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import (TOL, check_against_oracle, make_gat_layer, make_plain_layer, make_sage_layer, run_device, run_oracle,
+from gpu_util import (TOL, assert_close, check_against_oracle, make_gat_layer, make_plain_layer, make_sage_layer, run_device, run_oracle,
                       small_workload, to_numpy)
 from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
@@ -79,13 +79,19 @@ def test_gat_head_shapes(heads, hd):
 
 
 def test_gat_large_scores_do_not_overflow():
+    """Attention logits of +-100 and more: exp() of them overflows fp32, the running maximum keeps the softmax
+    finite.  The logits are fp32 by contract, so a softmax weight carries a relative error of about
+    |logit| * 2^-23 (1e-5 here): the plain fp32 tolerance still holds."""
     layer = make_gat_layer(9, "none", 16, 2, 8, "f32")
-    layer.att_src *= 200.0
-    layer.att_dst *= 200.0
+    layer.att_src *= 60.0
+    layer.att_dst *= 60.0
     w = small_workload(10, 400, 25, "f32", [layer], hubs=(300,))
+    z = w.x_as_f32() @ layer.W
+    logits = np.abs(z.reshape(w.n, 2, 8) * layer.att_src[None]).sum(-1)
+    assert logits.max() > 100.0, "the case must reach logits whose exp overflows fp32"
     got, _ = run_device(w)
     assert np.isfinite(got).all()
-    check_against_oracle(w, got, tol=1e-3)   # exp of large score differences: looser than the plain fp32 bound
+    check_against_oracle(w, got)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -234,6 +240,20 @@ def test_error_statuses():
     assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], d.x, d.x, d.workspace)) == "IT_ERR_INVALID_ARG"
     misaligned = d.workspace[1:]
     assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], d.x, out, misaligned)) == "IT_ERR_WORKSPACE"
+    # matrices that are not 16-byte aligned are refused on the host (the kernels move 16-byte slices)
+    flat = torch.empty(w.n * 16 + 4, device="cuda")
+    off4 = flat[1:1 + w.n * 16].view(w.n, 16)
+    assert off4.data_ptr() % 16 == 4
+    assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], off4, out, d.workspace)) == "IT_ERR_INVALID_ARG"
+    assert status_of(lambda: B.it_layer_forward(d.graph, d.layers[0], d.x, off4, d.workspace)) == "IT_ERR_INVALID_ARG"
+    assert status_of(lambda: B.it_layer_forward_static(d.graph, d.layers[0], off4, out)) == "IT_ERR_INVALID_ARG"
+    assert status_of(lambda: B.it_infer(d.graph, d.layers, off4, out, d.workspace)) == "IT_ERR_INVALID_ARG"
+    assert status_of(lambda: B.it_infer(d.graph, d.layers, d.x, off4, d.workspace)) == "IT_ERR_INVALID_ARG"
+    # input or output inside the workspace, or on top of each other
+    inside = d.workspace[:w.n * 16 * 4].view(torch.float32).view(w.n, 16)
+    assert status_of(lambda: B.it_infer(d.graph, d.layers, inside, out, d.workspace)) == "IT_ERR_INVALID_ARG"
+    assert status_of(lambda: B.it_infer(d.graph, d.layers, d.x, inside, d.workspace)) == "IT_ERR_INVALID_ARG"
+    assert status_of(lambda: B.it_infer(d.graph, d.layers, d.x, d.x, d.workspace)) == "IT_ERR_INVALID_ARG"
     bad = host.layer_to_device(make_sage_layer(29, "sum", "relu", 6, 16, "f32"), "f32")   # 24-byte rows
     assert status_of(lambda: B.it_workspace_bytes(d.graph, [bad])) == "IT_ERR_INVALID_ARG"
     mism = [d.layers[0], host.layer_to_device(make_sage_layer(30, "sum", "relu", 32, 16, "f32"), "f32")]
@@ -244,15 +264,13 @@ def test_error_statuses():
     assert torch.ones(4, device="cuda").sum().item() == 4
 
 
-def test_mode_a_error_is_reported_and_bounded():
-    """Against the exact fp64 oracle (no rounding at storage points) the bf16 path stays within a few bf16 ulps per layer."""
-    layers = [make_sage_layer(31, "mean", "relu", 64, 64, "bf16"), make_sage_layer(32, "mean", "none", 64, 32, "bf16")]
-    w = small_workload(33, 2000, 20, "bf16", layers, hubs=(700,), threshold=256)
-    got, _ = run_device(w)
-    err = compare.rel_error(got, run_oracle(w, storage=None)[-1])
-    assert err["max_rel"] < 5e-2
-    # and the fp32 path is far tighter
-    layers = [make_sage_layer(31, "mean", "relu", 64, 64, "f32"), make_sage_layer(32, "mean", "none", 64, 32, "f32")]
-    w = small_workload(33, 2000, 20, "f32", layers, hubs=(700,), threshold=256)
-    got, _ = run_device(w)
-    assert compare.rel_error(got, run_oracle(w, storage=None)[-1])["max_rel"] < TOL["f32"]
+def test_exact_oracle_bounds_both_storage_types():
+    """Against the fp64-throughout oracle (no rounding at storage points, plain order of operations) a two-layer
+    pass stays within the tolerance of its storage type, entry by entry."""
+    for dtype in ("bf16", "f32"):
+        layers = [make_sage_layer(31, "mean", "relu", 64, 64, dtype), make_sage_layer(32, "mean", "none", 64, 32, dtype)]
+        w = small_workload(33, 2000, 20, dtype, layers, hubs=(700,), threshold=256)
+        got, _ = run_device(w)
+        outs, mags = run_oracle(w, storage=None, magnitudes=True)
+        err = assert_close(got, outs[-1], mags[-1], dtype, "exact", label=dtype)
+        print(dtype, err)

@@ -15,9 +15,16 @@ GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "w5.json
 
 
 def L(op="sum", act="none", W=None, bias=None, heads=1, att_src=None, att_dst=None, slope=0.2,
-      use_edge_weights=False, allow_reorder=True, edge_dim=0):
+      use_edge_weights=False, allow_reorder=True, edge_dim=0, W_edge=None, bias_edge=None, act_edge="none"):
     W = np.asarray(W, dtype=np.float64)
     in_dim = (W.shape[0] - edge_dim) if op in ("gat", "dense", "gcn") else (W.shape[0] - edge_dim) // 2
+    if W_edge is not None:   # learned messages: W_edge is [in + edge_dim, msg_dim], W is [in + msg_dim, out] (GCN: [msg_dim, out])
+        W_edge = np.asarray(W_edge, dtype=np.float64)
+        in_dim = W_edge.shape[0] - edge_dim
+        return NS(op=op, act=act, in_dim=in_dim, out_dim=W.shape[1], W=W, edge_dim=edge_dim, msg_dim=W_edge.shape[1],
+                  W_edge=W_edge, bias_edge=None if bias_edge is None else np.asarray(bias_edge, dtype=np.float64),
+                  act_edge=act_edge, bias=None if bias is None else np.asarray(bias, dtype=np.float64), heads=1,
+                  att_src=None, att_dst=None, leaky_slope=slope, use_edge_weights=use_edge_weights, allow_reorder=allow_reorder)
     return NS(op=op, act=act, in_dim=in_dim, out_dim=W.shape[1], W=W, edge_dim=edge_dim,
               bias=None if bias is None else np.asarray(bias, dtype=np.float64), heads=heads,
               att_src=None if att_src is None else np.asarray(att_src, dtype=np.float64),
@@ -130,9 +137,17 @@ def tree_eval(v, depth, ip, ix, w, x, layers, memo=None, ef=None):
                         out[hd * D + c] += p / tot * z[hd * D + c]
         return [py_act(out[c] + (lay.bias[c] if lay.bias is not None else 0.0), lay.act) for c in range(Fo)]
     De = getattr(lay, "edge_dim", 0)
-    Fm = Fi + De   # length of a message: [w_e h_u | e_vu]
-    full = [[wj * h[f] for f in range(Fi)] + [float(ef[j][f]) for f in range(De)]
-            for j, (_, wj), h in zip(range(ip[v], ip[v + 1]), nb, hn)]
+    if getattr(lay, "msg_dim", 0):   # learned message: w_e act_e([h_u | e_vu] W_e + b_e)
+        Fm = lay.msg_dim
+        full = []
+        for j, (_, wj), h in zip(range(ip[v], ip[v + 1]), nb, hn):
+            cat = list(h) + [float(ef[j][f]) for f in range(De)]
+            full.append([wj * py_act(sum(cat[k] * lay.W_edge[k][c] for k in range(Fi + De)) +
+                                     (lay.bias_edge[c] if lay.bias_edge is not None else 0.0), lay.act_edge) for c in range(Fm)])
+    else:
+        Fm = Fi + De   # length of a message: [w_e h_u | e_vu]
+        full = [[wj * h[f] for f in range(Fi)] + [float(ef[j][f]) for f in range(De)]
+                for j, (_, wj), h in zip(range(ip[v], ip[v + 1]), nb, hn)]
     agg = [0.0] * Fm
     if full:
         for f in range(Fm):
@@ -728,3 +743,96 @@ def test_compact_neighbourhood_carries_edge_features():
     ids, cip, cix, cw, ct, cef = O.compact_neighbourhood(ip, ix, None, targets, 2, edge_feat=ef)
     got = O.infer_at(cip, cix, cw, x[ids], layers, ct, edge_feat=cef)
     assert np.allclose(got, full[targets], rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------ learned messages (apply_edge)
+
+class TestW5EdgeMessages:
+    g = GOLD["edge_messages"]
+    ip = np.array(GOLD["indptr"], np.int64)
+    ix = np.array(GOLD["indices"], np.int32)
+    x = np.array(GOLD["x"], np.float64)
+    w = np.array(GOLD["w"], np.float64)
+    ef = np.array(GOLD["edge_features"]["ef"], np.float64)
+
+    def test_messages(self):
+        g = self.g
+        assert O.edge_messages(self.ix, None, self.x, self.ef, g["W_e"], g["b_e"], g["act_e"]).tolist() == g["messages"]
+        assert O.edge_messages(self.ix, self.w, self.x, self.ef, g["W_e"], g["b_e"], g["act_e"]).tolist() == g["weighted_messages"]
+
+    @pytest.mark.parametrize("op", ["sum", "mean", "max"])
+    def test_aggregates_of_messages(self, op):
+        M = np.array(self.g["messages"], np.float64)
+        assert O.aggregate_edges(self.ip, M, op).tolist() == self.g[op]
+        sp, _, owner = O.split_hubs(self.ip, GOLD["split_T"])
+        P = O.aggregate_edges(sp, M, "sum" if op == "mean" else op)
+        if op == "sum":
+            assert P[:2].tolist() == self.g["partial_sum_v0"]
+        assert O.combine(owner, self.ip, P, op).tolist() == self.g[op]
+
+    def test_layer(self):
+        g = self.g
+        lay = L("sum", g["act"], g["W"], g["b"], edge_dim=1, W_edge=g["W_e"], bias_edge=g["b_e"], act_edge=g["act_e"])
+        for thr in (0, 2):
+            for storage in (None, "f32"):
+                out = O.layer_forward(self.ip, self.ix, None, self.x, lay, storage=storage, threshold=thr, edge_feat=self.ef)
+                assert out.tolist() == g["sage_sum_out"], (thr, storage)
+        wl = L("sum", "none", [[0, 0], [0, 0], [1, 0], [0, 1]], None, edge_dim=1, W_edge=g["W_e"], bias_edge=g["b_e"],
+               act_edge=g["act_e"], use_edge_weights=True)
+        assert O.layer_forward(self.ip, self.ix, self.w, self.x, wl, edge_feat=self.ef).tolist() == g["weighted_sum"]
+
+
+@pytest.mark.parametrize("op", ["sum", "mean", "max", "min", "gcn"])
+@pytest.mark.parametrize("depth", [1, 2])
+@pytest.mark.parametrize("De", [0, 2])
+def test_message_layers_equal_computation_tree(op, depth, De):
+    rng = np.random.default_rng(400 + depth + 10 * De)
+    n, Fm = 12, 3
+    ip, ix = random_graph(rng, n, 3)
+    w = rng.random(ix.shape[0])
+    ef = rng.standard_normal((ix.shape[0], De)) if De else None
+    dims = [3, 4, 2][:depth + 1]
+    x = rng.standard_normal((n, dims[0]))
+    layers = []
+    for i in range(depth):
+        fi, fo = dims[i], dims[i + 1]
+        rows = Fm if op == "gcn" else fi + Fm
+        layers.append(L(op, ["relu", "none"][i % 2], rng.standard_normal((rows, fo)), rng.standard_normal(fo),
+                        use_edge_weights=(op != "mean"), edge_dim=De, W_edge=rng.standard_normal((fi + De, Fm)),
+                        bias_edge=rng.standard_normal(Fm), act_edge=["elu", "relu"][i % 2]))
+    full = O.infer(ip, ix, w, x, layers, edge_feat=ef)[-1]
+    split = O.infer(ip, ix, w, x, layers, threshold=2, edge_feat=ef)[-1]
+    at = O.infer_at(ip, ix, w, x, layers, np.arange(n), threshold=2, edge_feat=ef)
+    stored = O.infer(ip, ix, w, x, layers, storage="f32", threshold=2, edge_feat=ef)[-1]
+    for v in range(n):
+        ref = np.array(tree_eval(v, depth, ip, ix, w, x, layers, ef=ef))
+        assert np.allclose(full[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+        assert np.allclose(split[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+        assert np.allclose(at[v], ref, rtol=1e-11, atol=1e-12), (op, depth, v)
+        assert np.allclose(stored[v], ref, rtol=2e-5, atol=2e-5), (op, depth, v)
+
+
+def test_linear_messages_reduce_to_the_plain_aggregates():
+    """Without an activation the sum of the messages is a closed form of the plain aggregates:
+    sum_j w_j ([h_u | e_j] W_e + b_e) = (sum_j w_j h_u) W_e[:in] + (sum_j w_j e_j) W_e[in:] + (sum_j w_j) b_e."""
+    rng = np.random.default_rng(41)
+    n, Fi, De, Fm = 40, 3, 2, 4
+    ip, ix = random_graph(rng, n, 6)
+    x = rng.standard_normal((n, Fi))
+    ef = rng.standard_normal((ix.shape[0], De))
+    w = rng.random(ix.shape[0])
+    We, be = rng.standard_normal((Fi + De, Fm)), rng.standard_normal(Fm)
+    M = O.edge_messages(ix, w, x, ef, We, be, "none")
+    got = O.aggregate_edges(ip, M, "sum")
+    wsum = np.add.reduceat(np.concatenate([w, [0.0]]), np.minimum(ip[:-1], w.size)) * (np.diff(ip) > 0)
+    want = O.aggregate(ip, ix, w, x, "sum") @ We[:Fi] + O.aggregate_edges(ip, ef * w[:, None], "sum") @ We[Fi:] + wsum[:, None] * be
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    # no edge features: the message depends on the source alone, so the aggregate is a plain gather of a table
+    M0 = O.edge_messages(ix, None, x, None, We[:Fi], be, "relu")
+    table = np.maximum(x @ We[:Fi] + be, 0.0)
+    assert np.allclose(O.aggregate_edges(ip, M0, "max"), O.aggregate(ip, ix, None, table, "max"), rtol=1e-13, atol=1e-13)
+    # the source part and the edge part of W_e are not swapped
+    We2 = We.copy()
+    We2[Fi] += 1.0
+    d = O.edge_messages(ix, None, x, ef, We2, be, "none") - O.edge_messages(ix, None, x, ef, We, be, "none")
+    assert np.allclose(d, np.repeat(ef[:, :1], Fm, axis=1), rtol=1e-12, atol=1e-12)

@@ -52,6 +52,30 @@ def test_static_variant_matches_the_workspace_variant_on_two_calls_in_a_row(case
         assert torch.equal(o, ref)     # same kernels, same order: the tests' bar here is equality
 
 
+def test_a_repeated_call_leaves_device_memory_as_it_found_it():
+    """What the entry point is for: after the set-up call of a layer shape (which loads the kernels it needs and
+    looks up the array), further calls neither take nor return device memory — seen from the driver (free bytes of
+    the device) and from torch's caching allocator (bytes reserved, allocation count)."""
+    layer = make_sage_layer(54, "sum", "relu", 64, 64, "f32", weights=True)
+    w = small_workload(55, 4000, 20, "f32", [layer], hubs=(3000, 700), weights=True, threshold=128)
+    d = host.upload(w)
+    assert d.n_split_owners > 0
+    out = torch.empty((w.n, 64), device="cuda")
+    B.it_layer_forward_static(d.graph, d.layers[0], d.x, out)     # set-up call
+    torch.cuda.synchronize()
+    first = out.clone()
+    free0 = torch.cuda.mem_get_info()[0]
+    stats0 = torch.cuda.memory_stats()
+    for _ in range(3):
+        B.it_layer_forward_static(d.graph, d.layers[0], d.x, out)
+    torch.cuda.synchronize()
+    stats1 = torch.cuda.memory_stats()
+    assert torch.cuda.mem_get_info()[0] == free0
+    for key in ("reserved_bytes.all.current", "allocation.all.allocated", "segment.all.allocated"):
+        assert stats1[key] == stats0[key], key
+    assert torch.equal(out, first)
+
+
 def test_calls_of_different_layers_share_the_array_safely():
     """Back-to-back calls with different layouts of the scratch array: each call rewrites what it reads."""
     l1 = make_sage_layer(47, "max", "relu", 32, 32, "f32")

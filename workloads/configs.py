@@ -32,6 +32,10 @@ class Layer:
     use_edge_weights: bool = False
     allow_reorder: bool = True
     edge_dim: int = 0        # > 0: the message carries the edge's feature vector; W has edge_dim more neighbour rows
+    msg_dim: int = 0         # > 0: learned message m = w_e act_edge([h_u | e_vu] W_edge + bias_edge); W is [in + msg_dim, out] (GCN: [msg_dim, out])
+    W_edge: np.ndarray | None = None      # float32 [in + edge_dim, msg_dim]
+    bias_edge: np.ndarray | None = None   # float32 [msg_dim]
+    act_edge: str = "none"
 
 
 @dataclass
