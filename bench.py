@@ -293,13 +293,14 @@ def sampled_parity(w, d, n_top: int, n_random: int) -> dict:
     for key, storage in (("stored", w.dtype), ("exact", None)):
         ref, mag = O.infer_at(cip, cix, cw, xc, w.layers, ct, storage=storage, threshold=w.threshold,
                               follow_reorder=storage is not None, edge_feat=cef, magnitudes=True)
-        err = compare.rel_error(got, ref, mag, compare.FLOOR[key])
+        err = compare.rel_error(got, ref, mag, compare.floor_for(key, w.dtype, len(w.layers)))
         out[key] = {k: err[k] for k in ("max_rel", "max_rel_plain", "max_over_mag", "max_abs", "rms")}
         out[key]["finite"] = bool(err["finite"])
-    out["ok"] = all(out[k]["finite"] and out[k]["max_rel"] <= out["tolerance"] and out[k]["max_rel_plain"] <= out["tolerance"]
-                    for k in ("stored", "exact"))
-    out["metric"] = ("max |got - ref| / max(|ref|, floor * sum of |terms| of the entry), floor 2^-7 (stored) / 2^-4 (exact); "
-                     "max_rel_plain = plain relative error over entries with |ref| > rms(ref)")
+    out["floor"] = {k: compare.floor_for(k, w.dtype, len(w.layers)) for k in ("stored", "exact")}
+    out["ok"] = bool(all(out[k]["finite"] and out[k]["max_rel"] <= out["tolerance"] for k in ("stored", "exact"))
+                     and out["stored"]["max_rel_plain"] <= out["tolerance"])
+    out["metric"] = ("max |got - ref| / max(|ref|, floor * sum of |terms| of the entry); max_rel_plain = plain relative error "
+                     "over entries with |ref| > rms(ref)")
     out["oracle"] = ("stored = fp64 accumulation, rounded where the layer contract stores a tensor (the gate); "
                      "exact = fp64 throughout, plain order of operations")
     out["seconds"] = time.perf_counter() - t0

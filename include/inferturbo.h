@@ -86,6 +86,15 @@ typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
  *   Every message function that is linear in (h_u, e_{v,u}) and is followed by a sum or mean and a dense update
  *   folds into this form.  The vectors come from it_graph_set_edge_features; such layers are never reordered.
  *
+ * Learned messages (msg_dim > 0; pooling layers and GCN): the general apply_edge of the Scatter stage (Section
+ *   "InferTurbo Abstraction"; M of Eq. (1)) as one dense layer on the source state and the edge's features,
+ *       m_{v,u} = w_e * act_edge( h_u * W_edge[0:in_dim] + e_{v,u} * W_edge[in_dim:in_dim+edge_dim] + bias_edge ),
+ *   msg_dim entries, reduced entry by entry with the layer's op (w_e = 1 without edge weights; edge_dim may be 0), then
+ *       GraphSAGE: h'_v = act( h_v * W[0:in_dim] + a_v * W[in_dim : in_dim + msg_dim] + bias ),  W is [in_dim + msg_dim, out_dim]
+ *       GCN:       h'_v = act( a_v * W + bias ),                                             W is [msg_dim, out_dim]
+ *   The source part h_u * W_edge[0:in_dim] is computed once per vertex and the edge part once per edge, both by the dense
+ *   transform; they, and the finished messages, are stored in feat_dtype.  Never reordered.
+ *
  * Storage contract: h_in, h_out (and the internal Z / aggregate tensors) are feat_dtype,
  * rounded to nearest even when written; all accumulation is fp32.  W is weight_dtype and
  * must equal feat_dtype.  bias, att_src, att_dst are fp32.  All are device pointers.
@@ -102,6 +111,10 @@ typedef struct {
   int32_t use_edge_weights;             /* 0/1; needs a graph created with edge weights */
   int32_t allow_reorder;                /* 0/1: allow transform-before-aggregate (see it_layer_forward) */
   int32_t edge_dim;                     /* 0, or the length of the edge-feature vectors the messages carry (see below) */
+  int32_t msg_dim;                      /* 0, or the length of a learned message (see "Learned messages") */
+  it_act act_edge;                      /* learned messages: activation of the message function */
+  const void *W_edge;                   /* learned messages: [in_dim + edge_dim, msg_dim], weight_dtype */
+  const float *bias_edge;               /* learned messages: [msg_dim], may be NULL */
 } it_layer_desc;
 
 /*
@@ -191,6 +204,79 @@ it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const 
  */
 it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, const void *x,
                    void *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * it_graph_create_part — one worker's part of a vertex-partitioned graph (Section "InferTurbo on Graph Processing
+ * System": vertices are partitioned over the workers together with their edges, one layer per superstep, messages
+ * exchanged in between).  The part holds the in-edges of `n_vertices` local destinations as a CSR of its own
+ * (indptr has n_vertices + 1 entries); source ids name rows of a table of `n_sources` rows that the caller assembles
+ * (all vertices of the graph for a destination partition; the local vertices for a source partition, see
+ * it_layer_gather).  Validation, borrowing and errors as it_graph_create, with 0 <= source < n_sources.
+ * it_layer_forward / it_infer take such a graph only when n_sources == n_vertices; otherwise use the stage calls.
+ */
+it_status it_graph_create_part(int64_t n_vertices, int64_t n_sources, int64_t n_edges, const void *indptr,
+                               it_itype indptr_type, const int32_t *indices, const float *edge_weights, void *stream,
+                               it_graph **out);
+
+/*
+ * The three stages of one layer as calls of their own, for callers that exchange data between them: several GPUs
+ * that each own a range of the vertices, or one GPU that walks over parts of a graph too large to hold at once.
+ * The names follow Section "InferTurbo Abstraction": what a vertex hands to its out-edges is produced by
+ * it_layer_transform (the apply_edge half of Scatter, done once per source), it_layer_gather is the Gather stage
+ * (gather_nbrs + aggregate; for GAT and transform-first layers it also finishes the vertex), it_layer_update is
+ * apply_node.  it_layer_forward is exactly transform, gather, update on one graph with every table in the workspace.
+ *
+ * it_layer_stages tells what the layer exchanges:
+ *   table_dim / table_dtype  one row per SOURCE vertex that the gather reads (the layer input itself when
+ *                            table_is_input = 1: then it_layer_transform has nothing to do and need not be called)
+ *   score_dim                fp32 values per vertex that travel with the table (GAT: 2 * heads, source scores
+ *                            then destination scores), else 0
+ *   agg_dim                  entries of the aggregate row that it_layer_gather hands to it_layer_update; 0 when the
+ *                            gather writes the layer output itself and there is no update call
+ */
+typedef struct {
+  int32_t table_dim;
+  it_dtype table_dtype;
+  int32_t score_dim;
+  int32_t table_is_input;
+  int32_t agg_dim;
+} it_stage_desc;
+it_status it_layer_stages(const it_graph *g, const it_layer_desc *layer, it_stage_desc *out);
+
+/*
+ * it_layer_transform — per local vertex, what its out-edges will carry: h_self [n, in_dim] -> table_out [n, table_dim]
+ * (and scores_out [n, score_dim]).  Terms of the layer that stay with the vertex (the self term of a transform-first
+ * layer) are kept in the workspace for it_layer_gather, so the same workspace must be passed to all three calls.
+ */
+it_status it_layer_transform(const it_graph *g, const it_layer_desc *layer, const void *h_self, void *table_out,
+                             float *scores_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * it_layer_gather — the Gather stage over the in-edges of the local destinations.  table [n_sources, table_dim] is
+ * indexed by the source ids of the graph; scores [n_sources, score_dim] likewise (GAT), the destination scores of
+ * local vertex v being row first_vertex + v of it.  out is the aggregate [n, agg_dim] in feat_dtype, or the layer
+ * output [n, out_dim] when agg_dim = 0.
+ * raw_partial = 1 (layers with agg_dim > 0 whose table is the input, no edge features): the partial-gather of
+ * Section "Optimization Strategies" for a partition of the SOURCES: out is fp32 [n, agg_dim] and holds the plain
+ * sum (for mean too), max or min over the edges this part has, with the identity of the reduce (0, -inf, +inf)
+ * where it has none; the caller reduces the parts' results (sum / max / min) and finishes with it_aggregate_finish.
+ */
+it_status it_layer_gather(const it_graph *g, const it_layer_desc *layer, const void *table, const float *scores,
+                          int64_t first_vertex, int32_t raw_partial, void *out, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+/* it_layer_update — apply_node: h_self [n, in_dim] and agg [n, agg_dim] -> h_out [n, out_dim]. */
+it_status it_layer_update(const it_graph *g, const it_layer_desc *layer, const void *h_self, const void *agg,
+                          void *h_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * it_aggregate_finish — the receiver's side of a partial-gather over source partitions: raw [n, dim] fp32 (the
+ * reduced partial results) -> out [n, dim] of `dtype`, out[v, :] = raw[v, :] * scale[v], and 0 where scale[v] = 0
+ * (a vertex without in-edges, whose raw row still holds the identity of the reduce).  scale: fp32 [n]; 1 / in-degree
+ * for mean, 1 otherwise.
+ */
+it_status it_aggregate_finish(int64_t n, int32_t dim, it_dtype dtype, const float *raw, const float *scale, void *out,
+                              void *stream);
 
 /*
  * it_layer_forward_static — it_layer_forward for callers that must not allocate device

@@ -25,7 +25,8 @@ IT_MAX_BUCKETS = 8
 EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspace_bytes", "it_layer_forward",
            "it_infer", "it_graph_destroy", "it_status_string", "it_last_error_message", "it_profile_begin",
            "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static", "it_graph_check",
-           "it_graph_set_edge_features", "it_debug_expire_wait"]
+           "it_graph_set_edge_features", "it_debug_expire_wait", "it_graph_create_part", "it_layer_stages",
+           "it_layer_transform", "it_layer_gather", "it_layer_update", "it_aggregate_finish"]
 
 
 class ItError(RuntimeError):
@@ -41,7 +42,13 @@ class it_layer_desc(C.Structure):
                 ("feat_dtype", C.c_int), ("weight_dtype", C.c_int),
                 ("W", C.c_void_p), ("bias", C.c_void_p), ("att_src", C.c_void_p), ("att_dst", C.c_void_p),
                 ("leaky_slope", C.c_float), ("use_edge_weights", C.c_int32), ("allow_reorder", C.c_int32),
-                ("edge_dim", C.c_int32)]
+                ("edge_dim", C.c_int32), ("msg_dim", C.c_int32), ("act_edge", C.c_int),
+                ("W_edge", C.c_void_p), ("bias_edge", C.c_void_p)]
+
+
+class it_stage_desc(C.Structure):
+    _fields_ = [("table_dim", C.c_int32), ("table_dtype", C.c_int), ("score_dim", C.c_int32),
+                ("table_is_input", C.c_int32), ("agg_dim", C.c_int32)]
 
 
 _lib = None
@@ -63,6 +70,15 @@ def lib() -> C.CDLL:
         L.it_layer_forward.argtypes = [vp, C.POINTER(it_layer_desc), vp, vp, vp, C.c_size_t, vp]
         L.it_infer.argtypes = [vp, C.POINTER(it_layer_desc), i32, vp, vp, vp, C.c_size_t, vp]
         L.it_graph_destroy.argtypes = [vp]
+        L.it_graph_create_part.argtypes = [i64, i64, i64, vp, C.c_int, vp, vp, vp, C.POINTER(vp)]
+        L.it_layer_stages.argtypes = [vp, C.POINTER(it_layer_desc), C.POINTER(it_stage_desc)]
+        L.it_layer_transform.argtypes = [vp, C.POINTER(it_layer_desc), vp, vp, vp, vp, C.c_size_t, vp]
+        L.it_layer_gather.argtypes = [vp, C.POINTER(it_layer_desc), vp, vp, i64, i32, vp, vp, C.c_size_t, vp]
+        L.it_layer_update.argtypes = [vp, C.POINTER(it_layer_desc), vp, vp, vp, vp, C.c_size_t, vp]
+        L.it_aggregate_finish.argtypes = [i64, i32, C.c_int, vp, vp, vp, vp]
+        for name in ("it_graph_create_part", "it_layer_stages", "it_layer_transform", "it_layer_gather", "it_layer_update",
+                     "it_aggregate_finish"):
+            getattr(L, name).restype = C.c_int
         for name in EXPORTS[:7]:
             getattr(L, name).restype = C.c_int
         L.it_status_string.argtypes = [C.c_int]
@@ -110,12 +126,17 @@ class LayerDesc:
     use_edge_weights: bool = False
     allow_reorder: bool = True
     edge_dim: int = 0
+    msg_dim: int = 0
+    W_edge: torch.Tensor | None = None
+    bias_edge: torch.Tensor | None = None
+    act_edge: str = "none"
 
     def to_c(self) -> it_layer_desc:
-        for t in (self.W, self.bias, self.att_src, self.att_dst):
+        for t in (self.W, self.bias, self.att_src, self.att_dst, self.W_edge, self.bias_edge):
             assert t is None or (t.is_cuda and t.is_contiguous())
-        for t in (self.bias, self.att_src, self.att_dst):
+        for t in (self.bias, self.att_src, self.att_dst, self.bias_edge):
             assert t is None or t.dtype == torch.float32
+        assert self.W_edge is None or self.W_edge.dtype == self.W.dtype
         d = it_layer_desc()
         d.op, d.act = GATHER_OPS[self.op], ACTS[self.act]
         d.in_dim, d.out_dim, d.heads = self.in_dim, self.out_dim, self.heads
@@ -128,6 +149,10 @@ class LayerDesc:
         d.use_edge_weights = int(self.use_edge_weights)
         d.allow_reorder = int(self.allow_reorder)
         d.edge_dim = int(self.edge_dim)
+        d.msg_dim = int(self.msg_dim)
+        d.act_edge = ACTS[self.act_edge]
+        d.W_edge = None if self.W_edge is None else self.W_edge.data_ptr()
+        d.bias_edge = None if self.bias_edge is None else self.bias_edge.data_ptr()
         return d
 
 
@@ -162,6 +187,56 @@ def it_graph_create(indptr: torch.Tensor, indices: torch.Tensor, edge_weights: t
     _check(lib().it_graph_create(n, e, _ptr(indptr), IT_I64 if indptr.dtype == torch.int64 else IT_I32,
                                  _ptr(indices), _ptr(edge_weights), _stream(stream), C.byref(out)))
     return Graph(out, n, e, (indptr, indices, edge_weights))
+
+
+def it_graph_create_part(indptr: torch.Tensor, indices: torch.Tensor, n_sources: int, edge_weights: torch.Tensor | None = None,
+                         stream=None) -> Graph:
+    """One part of a vertex-partitioned graph: the in-edges of len(indptr) - 1 local destinations, source ids
+    naming rows of a table of n_sources rows."""
+    assert indptr.is_cuda and indptr.is_contiguous() and indptr.dtype in (torch.int32, torch.int64)
+    assert indices.dtype == torch.int32 and indices.is_contiguous() and (indices.is_cuda or indices.numel() == 0)
+    assert edge_weights is None or (edge_weights.is_cuda and edge_weights.dtype == torch.float32 and edge_weights.is_contiguous())
+    n, e = indptr.numel() - 1, indices.numel()
+    out = C.c_void_p()
+    _check(lib().it_graph_create_part(n, n_sources, e, _ptr(indptr), IT_I64 if indptr.dtype == torch.int64 else IT_I32,
+                                      _ptr(indices), _ptr(edge_weights), _stream(stream), C.byref(out)))
+    g = Graph(out, n, e, (indptr, indices, edge_weights))
+    g.n_sources = n_sources
+    return g
+
+
+def it_layer_stages(g: Graph, layer) -> dict:
+    """What the stage calls of this layer exchange: table_dim, table_dtype, score_dim, table_is_input, agg_dim."""
+    d = it_stage_desc()
+    _check(lib().it_layer_stages(g.handle, _c_layers([layer]), C.byref(d)))
+    return {"table_dim": d.table_dim, "table_dtype": torch.float32 if d.table_dtype == IT_F32 else torch.bfloat16,
+            "score_dim": d.score_dim, "table_is_input": bool(d.table_is_input), "agg_dim": d.agg_dim}
+
+
+def _nbytes(t):
+    return t.numel() * t.element_size()
+
+
+def it_layer_transform(g: Graph, layer, h_self, table_out, scores_out, workspace, stream=None):
+    _check(lib().it_layer_transform(g.handle, _c_layers([layer]), _ptr(h_self), _ptr(table_out), _ptr(scores_out),
+                                    _ptr(workspace), _nbytes(workspace), _stream(stream)))
+
+
+def it_layer_gather(g: Graph, layer, table, scores, first_vertex: int, raw_partial: bool, out, workspace, stream=None):
+    _check(lib().it_layer_gather(g.handle, _c_layers([layer]), _ptr(table), _ptr(scores), first_vertex, int(raw_partial),
+                                 _ptr(out), _ptr(workspace), _nbytes(workspace), _stream(stream)))
+
+
+def it_layer_update(g: Graph, layer, h_self, agg, h_out, workspace, stream=None):
+    _check(lib().it_layer_update(g.handle, _c_layers([layer]), _ptr(h_self), _ptr(agg), _ptr(h_out), _ptr(workspace),
+                                 _nbytes(workspace), _stream(stream)))
+
+
+def it_aggregate_finish(raw: torch.Tensor, scale: torch.Tensor, out: torch.Tensor, stream=None):
+    """out[v, :] = raw[v, :] * scale[v] (0 where scale[v] = 0); raw fp32 [n, dim], scale fp32 [n]."""
+    assert raw.dtype == torch.float32 and scale.dtype == torch.float32 and raw.is_contiguous() and out.is_contiguous()
+    _check(lib().it_aggregate_finish(raw.shape[0], raw.shape[1], _dt(out.dtype), _ptr(raw), _ptr(scale), _ptr(out), _stream(stream)))
+    return out
 
 
 def it_graph_set_edge_features(g: Graph, edge_feat: torch.Tensor | None):

@@ -42,6 +42,7 @@ void it_set_error(const char *fmt, ...);
 enum it_kernel_id {
   IT_K_VALIDATE = 0, IT_K_SPLIT_SCAN, IT_K_SPLIT_FILL, IT_K_BUCKET_SCAN, IT_K_PREP, IT_K_GATHER_CTA, IT_K_GATHER_FLAT,
   IT_K_GATHER_EMPTY, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY,
+  IT_K_EDGE_MSG, IT_K_AGG_FINISH,
   IT_K_COUNT
 };
 // Wraps one kernel launch: counts it and, while profiling is on, brackets it with events on `st`.
@@ -69,6 +70,7 @@ struct __align__(16) it_row_meta {
 
 struct it_graph {
   int64_t n = 0, e = 0;
+  int64_t n_src = 0;   // rows of the table the source ids name (= n unless the graph is one part of a partition)
   const void *indptr = nullptr;
   it_itype indptr_type = IT_I64;
   const int32_t *indices = nullptr;
@@ -126,7 +128,9 @@ static inline int it_dtype_size(it_dtype t) { return t == IT_F32 ? 4 : 2; }
 enum it_epilogue_kind {
   IT_EPI_STORE = 0,      // dst[v, :] = agg                      (feat dtype)
   IT_EPI_ADD_ACT = 1,    // dst[v, :] = act(self[v, :] + agg)    (self fp32, dst feat dtype)
-  IT_EPI_BIAS_ACT = 2    // dst[v, :] = act(bias + agg)          (bias fp32 [dim] or NULL)
+  IT_EPI_BIAS_ACT = 2,   // dst[v, :] = act(bias + agg)          (bias fp32 [dim] or NULL)
+  IT_EPI_RAW_F32 = 3     // dst[v, :] = the raw reduce in fp32: plain sum (mean undivided), max or min, and the identity of
+                         // the reduce (0, -inf, +inf) for a row without edges: one part's share of a partial-gather
 };
 
 struct it_gather_args {
@@ -155,7 +159,8 @@ struct it_gat_args {
   it_dtype dtype;
   int heads, head_dim;
   const void *z;          // [n, heads*head_dim] messages
-  const float *scores;    // [n, 2*heads]: source scores of the vertex, then its destination scores
+  const float *scores;    // [n_src, 2*heads]: source scores of the vertex, then its destination scores
+  const float *scores_dst;   // the same layout, row v = local destination v (scores + first_vertex * 2*heads for a part; NULL: scores)
   float *partials;        // it_gat_partial_bytes() of fp32 scratch for the groups of split vertices (may be NULL if none)
   float slope;
   const float *bias;      // may be NULL
@@ -202,3 +207,10 @@ it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *laye
                                     cudaStream_t stream);
 it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *att_src, const float *att_dst,
                             int heads, int head_dim, float *scores, int num_sms, int *status, cudaStream_t stream);
+
+// ----------------------------------------------------------------------------- message.cu
+// Learned messages, edge by edge: M[j, :] = act(P[indices[j], :] + M[j, :]) in place (M arrives holding the per-edge
+// part Q), rows of `dim` elements of `dtype` (a multiple of 16 bytes).
+it_status it_launch_edge_messages(const it_graph *g, it_dtype dtype, int dim, const void *P, void *M, it_act act, cudaStream_t stream);
+// out[v, :] = raw[v, :] * scale[v] (0 where scale[v] = 0), fp32 -> dtype.
+it_status it_launch_aggregate_finish(int64_t n, int dim, it_dtype dtype, const float *raw, const float *scale, void *out, cudaStream_t stream);

@@ -19,7 +19,8 @@ struct GatPolicy {
   static constexpr int VEC = Slice::VEC;
   static constexpr int NS = VEC + 2;   // accumulators, running max, running sum
   static constexpr bool WEIGHTED = false, HAS_EXTRA = true, NEEDS_OWNER = true;
-  const float *__restrict__ scores;    // [n, 2*heads]: source scores of the vertex, then its destination scores
+  const float *__restrict__ scores;    // [n_src, 2*heads]: source scores of the vertex, then its destination scores
+  const float *__restrict__ scores_dst;   // the same rows, counted from the first local destination
   const float *__restrict__ bias;
   void *__restrict__ dst;
   float *__restrict__ partials;        // [n_partial_rows, stride]: acc[dim], m[heads], l[heads]
@@ -61,7 +62,7 @@ struct GatPolicy {
     st[VEC] = m_new;
   }
   __device__ __forceinline__ void begin_row(int32_t, int32_t owner) {
-    s_dst = __ldg(scores + (int64_t)owner * (2 * heads) + heads + head);
+    s_dst = __ldg(scores_dst + (int64_t)owner * (2 * heads) + heads + head);
   }
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t) const {
     if (dest < 0) {   // a group of a split vertex: its state goes to the partial buffer
@@ -136,7 +137,7 @@ __global__ void __launch_bounds__(THREADS) gat_combine_kernel(GatCombineParams p
 template <typename T, int SB, int LPR>
 it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   GatPolicy<T, SB> pol;
-  pol.scores = a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
+  pol.scores = a.scores; pol.scores_dst = a.scores_dst ? a.scores_dst : a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
   pol.dim = a.heads * a.head_dim; pol.heads = a.heads; pol.head_dim = a.head_dim; pol.act = a.act; pol.slope = a.slope;
   pol.col = 0; pol.head = 0; pol.s_dst = 0.f;
   const it_graph *g = a.g;

@@ -52,12 +52,16 @@ struct SagePolicy {
     if (epi == IT_EPI_ADD_ACT && dest >= 0) load_floats_stream<VEC>(self_term + (int64_t)dest * self_ld + col, self);
   }
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t len) const {
-    if (RED != RED_SUM && len == 0) {
+    if (RED != RED_SUM && len == 0 && epi != IT_EPI_RAW_F32) {
 #pragma unroll
       for (int i = 0; i < VEC; ++i) st[i] = 0.f;
     }
     if (dest < 0) {  // a group of a split vertex: raw partial, finished by the combine kernel
       store_floats<VEC>(partials + (int64_t)(~dest) * dim + col, st);
+      return;
+    }
+    if (epi == IT_EPI_RAW_F32) {   // one part's share of a partial-gather: the reduce as it is (its identity for an empty row)
+      store_floats<VEC>(reinterpret_cast<float *>(dst) + (int64_t)dest * dst_ld + col, st);
       return;
     }
     if (is_mean && len > 0) {
@@ -125,6 +129,10 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
       for (; g < n; ++g) fold(__ldg(reinterpret_cast<const float4 *>(p.partials + (p0 + g) * p.dim + c)));
       float o[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
       const int64_t doff = v * p.dst_ld + c;
+      if (p.epi == IT_EPI_RAW_F32) {
+        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.dst) + doff) = make_float4(o[0], o[1], o[2], o[3]);
+        continue;
+      }
       if (p.epi == IT_EPI_ADD_ACT) {
         float4 s = __ldg(reinterpret_cast<const float4 *>(p.self_term + v * p.self_ld + c));
         o[0] = act_apply(o[0] + s.x, p.act); o[1] = act_apply(o[1] + s.y, p.act);
@@ -149,7 +157,7 @@ template <typename T, int SB, int LPR, int RED, bool WEIGHTED>
 it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   SagePolicy<T, SB, RED, WEIGHTED> pol;
   pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim; pol.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; pol.self_ld = a.self_ld > 0 ? a.self_ld : a.dim;
-  pol.is_mean = a.op == IT_GATHER_MEAN; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
+  pol.is_mean = a.op == IT_GATHER_MEAN && a.epi != IT_EPI_RAW_F32; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
   const it_graph *g = a.g;
   // algorithmic bytes: per edge the index, the optional weight and one source row; per row its
   // metadata and one output row (plus the self row it is added to)
@@ -188,7 +196,7 @@ static it_status launch_gather_chunk(const it_gather_args &a, cudaStream_t st) {
     c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.shadow_indptr = g->shadow_indptr;
     c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.bias = a.bias; c.n_split_owners = g->n_split_owners;
     c.dim = a.dim; c.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; c.self_ld = a.self_ld > 0 ? a.self_ld : a.dim;
-    c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN; c.epi = a.epi; c.act = a.act;
+    c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN && a.epi != IT_EPI_RAW_F32; c.epi = a.epi; c.act = a.act;
     int64_t want = (g->n_split_owners + 7) / 8;
     int64_t cap = (int64_t)g->num_sms * 8;
     unsigned blocks = (unsigned)(want < cap ? want : cap);
@@ -222,7 +230,7 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
     c.dim = bytes / es;
     c.src = (const char *)a.src + (size_t)c0 * es;
     c.src_ld = a.src_ld > 0 ? a.src_ld : full;
-    c.dst = (char *)a.dst + (size_t)c0 * es;
+    c.dst = (char *)a.dst + (size_t)c0 * (a.epi == IT_EPI_RAW_F32 ? 4 : es);
     c.dst_ld = a.dst_ld > 0 ? a.dst_ld : full;
     c.self_term = a.self_term ? a.self_term + c0 : nullptr;
     c.self_ld = a.self_ld > 0 ? a.self_ld : full;

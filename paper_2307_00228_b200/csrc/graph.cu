@@ -395,12 +395,13 @@ extern "C" it_status it_graph_set_edge_features(it_graph *g, const void *edge_fe
   return IT_OK;
 }
 
-extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, it_itype indptr_type,
-                                     const int32_t *indices, const float *edge_weights, void *stream,
-                                     it_graph **out) {
+static it_status create_impl(int64_t n, int64_t n_src, int64_t e, const void *indptr, it_itype indptr_type,
+                             const int32_t *indices, const float *edge_weights, void *stream, it_graph **out) {
   IT_REQUIRE(out != nullptr, IT_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
   IT_REQUIRE(n >= 0 && n <= (int64_t)INT32_MAX - 1, IT_ERR_INVALID_ARG, "n_vertices %lld outside [0, 2^31-2]", (long long)n);
+  IT_REQUIRE(n_src >= 0 && n_src <= (int64_t)INT32_MAX - 1, IT_ERR_INVALID_ARG, "n_sources %lld outside [0, 2^31-2]", (long long)n_src);
+  IT_REQUIRE(e == 0 || n_src > 0, IT_ERR_INVALID_ARG, "edges need at least one source vertex");
   IT_REQUIRE(e >= 0, IT_ERR_INVALID_ARG, "n_edges is negative");
   IT_REQUIRE(indptr != nullptr, IT_ERR_INVALID_ARG, "indptr is NULL");
   IT_REQUIRE(indices != nullptr || e == 0, IT_ERR_INVALID_ARG, "indices is NULL");
@@ -422,7 +423,7 @@ extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, i
   if (ce == cudaSuccess && h_flags == 0 && e > 0) {
     int64_t want = (e + 255) / 256;
     unsigned blocks = (unsigned)(want < 148 * 16 ? want : 148 * 16);
-    IT_LAUNCH(IT_K_VALIDATE, 0, 0, st, validate_indices_kernel<<<blocks, 256, 0, st>>>(indices, e, n, d_flags));
+    IT_LAUNCH(IT_K_VALIDATE, 0, 0, st, validate_indices_kernel<<<blocks, 256, 0, st>>>(indices, e, n_src, d_flags));
     ce = cudaMemcpyAsync(&h_flags, d_flags, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
   }
@@ -433,13 +434,13 @@ extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, i
   }
   if (h_flags != 0) {
     it_set_error("bad CSR:%s%s%s%s", (h_flags & 1) ? " indptr[0] != 0;" : "", (h_flags & 2) ? " indptr decreases;" : "",
-                 (h_flags & 4) ? " indptr[n] != n_edges;" : "", (h_flags & 8) ? " a source id is outside [0, n);" : "");
+                 (h_flags & 4) ? " indptr[n] != n_edges;" : "", (h_flags & 8) ? " a source id is outside [0, n_sources);" : "");
     return IT_ERR_BAD_GRAPH;
   }
 
   it_graph *g = new (std::nothrow) it_graph();
   IT_REQUIRE(g != nullptr, IT_ERR_OOM, "host allocation failed");
-  g->n = n; g->e = e; g->indptr = indptr; g->indptr_type = indptr_type;
+  g->n = n; g->n_src = n_src; g->e = e; g->indptr = indptr; g->indptr_type = indptr_type;
   g->indices = indices; g->edge_weights = edge_weights;
   cudaGetDevice(&g->device);
   int sms = 0;
@@ -454,6 +455,18 @@ extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, i
   if (rc != IT_OK) { cudaFree(g->d_status); delete g; return rc; }
   *out = g;
   return IT_OK;
+}
+
+extern "C" it_status it_graph_create(int64_t n, int64_t e, const void *indptr, it_itype indptr_type,
+                                     const int32_t *indices, const float *edge_weights, void *stream,
+                                     it_graph **out) {
+  return create_impl(n, n, e, indptr, indptr_type, indices, edge_weights, stream, out);
+}
+
+extern "C" it_status it_graph_create_part(int64_t n, int64_t n_sources, int64_t e, const void *indptr, it_itype indptr_type,
+                                          const int32_t *indices, const float *edge_weights, void *stream,
+                                          it_graph **out) {
+  return create_impl(n, n_sources, e, indptr, indptr_type, indices, edge_weights, stream, out);
 }
 
 extern "C" it_status it_split_hubs(it_graph *g, int64_t threshold, void *stream, int64_t *out_n_rows,

@@ -29,7 +29,9 @@ def layer_to_device(layer, dtype: str, device="cuda") -> B.LayerDesc:
                        W=param_to_device(layer.W, dtype, device), bias=f32(layer.bias), heads=layer.heads,
                        att_src=f32(layer.att_src), att_dst=f32(layer.att_dst), leaky_slope=float(layer.leaky_slope),
                        use_edge_weights=bool(layer.use_edge_weights), allow_reorder=bool(layer.allow_reorder),
-                       edge_dim=int(getattr(layer, "edge_dim", 0) or 0))
+                       edge_dim=int(getattr(layer, "edge_dim", 0) or 0), msg_dim=int(getattr(layer, "msg_dim", 0) or 0),
+                       W_edge=None if getattr(layer, "W_edge", None) is None else param_to_device(layer.W_edge, dtype, device),
+                       bias_edge=f32(getattr(layer, "bias_edge", None)), act_edge=getattr(layer, "act_edge", "none"))
 
 
 @dataclass

@@ -63,6 +63,17 @@ def make_plain_layer(seed, op, act, fi, fo, dtype, weights=False, allow_reorder=
                  use_edge_weights=weights, allow_reorder=allow_reorder, edge_dim=edge_dim)
 
 
+def make_msg_layer(seed, op, act, fi, fm, fo, dtype, act_edge="relu", weights=False, edge_dim=0, bias=True) -> Layer:
+    """A layer with learned messages m = w_e act_edge([h_u | e_vu] W_edge + b_edge) of length fm; op may be "gcn"."""
+    rng = np.random.default_rng(seed)
+    k = fm if op == "gcn" else fi + fm
+    lim, lim_e = np.sqrt(6.0 / (k + fo)), np.sqrt(6.0 / (fi + edge_dim + fm))
+    return Layer(op=op, act=act, in_dim=fi, out_dim=fo, W=storage_exact(rng.uniform(-lim, lim, (k, fo)), dtype),
+                 bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None, use_edge_weights=weights,
+                 edge_dim=edge_dim, msg_dim=fm, W_edge=storage_exact(rng.uniform(-lim_e, lim_e, (fi + edge_dim, fm)), dtype),
+                 bias_edge=rng.uniform(-0.1, 0.1, fm).astype(np.float32) if bias else None, act_edge=act_edge)
+
+
 def make_gat_layer(seed, act, fi, heads, hd, dtype, bias=True) -> Layer:
     rng = np.random.default_rng(seed)
     fo = heads * hd
@@ -90,21 +101,45 @@ def run_oracle(w: Workload, storage="same", threshold=None, magnitudes=False):
                    follow_reorder=st is not None, edge_feat=w.edge_feat_as_f32(), magnitudes=magnitudes)
 
 
-def assert_close(got, ref, mag, dtype, mode="stored", tol=None, label=""):
-    """The parity gate: every entry within tol of the reference relative to max(|ref|, floor * term magnitude),
-    and the plain relative error of the entries above the reference's rms within tol as well."""
-    err = compare.rel_error(got, ref, mag, compare.FLOOR[mode])
+def assert_close(got, ref, mag, dtype, mode="stored", tol=None, label="", n_layers=1):
+    """The parity gate: every entry within tol of the reference relative to max(|ref|, floor * term magnitude); against
+    the storage-rounding oracle, for up to three layers, also the plain relative error of the entries above the
+    reference's rms.  (Against the fp64-throughout oracle, and at the end of a deep pipeline, an entry above the rms may
+    still be a small remainder of large terms, each carrying the rounding of a stored tensor, so only the floored form is
+    a bound there.)"""
+    err = compare.rel_error(got, ref, mag, compare.floor_for(mode, dtype, n_layers))
     tol = TOL[dtype] if tol is None else tol
     assert err["finite"], (label, err)
-    assert err["max_rel"] <= tol, (label, mode, err)
-    assert err["max_rel_plain"] <= tol, (label, mode, err)
+    assert err["max_rel"] <= tol, (label, mode, n_layers, err)
+    if mode == "stored" and n_layers <= 3:
+        assert err["max_rel_plain"] <= tol, (label, mode, n_layers, err)
     return err
 
 
 def check_against_oracle(w: Workload, got: np.ndarray, tol=None, label="", exact=True):
+    """The result of all layers against the oracle run from the raw inputs."""
+    L = len(w.layers)
     outs, mags = run_oracle(w, magnitudes=True)
-    err = assert_close(got, outs[-1], mags[-1], w.dtype, "stored", tol, label)
+    err = assert_close(got, outs[-1], mags[-1], w.dtype, "stored", tol, label, n_layers=L)
     if exact:   # and against the fp64-throughout oracle, which charges the storage roundings to the device
         outs_a, mags_a = run_oracle(w, storage=None, magnitudes=True)
-        assert_close(got, outs_a[-1], mags_a[-1], w.dtype, "exact", tol, label)
+        assert_close(got, outs_a[-1], mags_a[-1], w.dtype, "exact", tol, label, n_layers=L)
     return err
+
+
+def check_each_layer(w: Workload, d, label=""):
+    """Every layer on its own: the device runs layer l on ITS OWN output of layer l - 1, and the oracle is given exactly
+    those values, so nothing compounds and each layer is held to the single-layer floors."""
+    h = d.x
+    for l, (lay, src) in enumerate(zip(d.layers, w.layers)):
+        o = torch.empty((w.n, src.out_dim), dtype=d.x.dtype, device=d.x.device)
+        B.it_layer_forward(d.graph, lay, h, o, d.workspace)
+        B.it_graph_check(d.graph)
+        H = to_numpy(h)
+        for mode, storage in (("stored", w.dtype), ("exact", None)):
+            ref = O.layer_forward(w.indptr, w.indices, w.edge_weights, H, src, storage=storage, threshold=w.threshold,
+                                  reorder=storage is not None and O.will_reorder(src), edge_feat=w.edge_feat_as_f32())
+            mag = O.layer_magnitude(w.indptr, w.indices, w.edge_weights, H, src, edge_feat=w.edge_feat_as_f32())
+            assert_close(to_numpy(o), ref, mag, w.dtype, mode, label=(label, "layer", l))
+        h = o
+    return h

@@ -122,7 +122,7 @@ def test_rounding_noise_passes_and_planted_mistakes_fail_the_fp32_gate():
     ip, ix, X, lay = sage_case()
     ref = O.layer_forward(ip, ix, None, X, lay)
     D = O.layer_magnitude(ip, ix, None, X, lay)
-    tol, floor = compare.TOL["f32"], compare.FLOOR["stored"]
+    tol, floor = compare.TOL["f32"], compare.FLOOR["stored"]["f32"]
     # an fp32 evaluation of the same layer: every product and sum rounded to fp32
     A = O.aggregate(ip, ix, None, X, "sum").astype(np.float32)
     pre = (X.astype(np.float32) @ lay.W[:64].astype(np.float32) + A @ lay.W[64:].astype(np.float32) + lay.bias.astype(np.float32))
@@ -137,8 +137,8 @@ def test_rounding_noise_passes_and_planted_mistakes_fail_the_fp32_gate():
         wrong = O.layer_forward(ip, ix, None, X, bad)
         e = compare.rel_error(wrong, ref, D, floor)
         assert e["max_rel"] > 100 * tol, e
-        # the bf16 gate sees them too
-        assert e["max_rel"] > compare.TOL["bf16"], e
+        # the bf16 gate (its own floor and tolerance) sees them too
+        assert compare.rel_error(wrong, ref, D, compare.FLOOR["stored"]["bf16"])["max_rel"] > compare.TOL["bf16"], e
 
 
 def test_entries_that_cancelled_are_held_to_the_floor_not_to_their_own_size():
@@ -163,5 +163,5 @@ def test_bf16_storage_rounding_stays_inside_the_bf16_gate_against_the_exact_orac
     ref = O.layer_forward(ip, ix, None, Xb, lay)
     D = O.layer_magnitude(ip, ix, None, Xb, lay)
     got = O.layer_forward(ip, ix, None, Xb, lay, storage="bf16")
-    e = compare.rel_error(got, ref, D, compare.FLOOR["exact"])
+    e = compare.rel_error(got, ref, D, compare.FLOOR["exact"]["bf16"])
     assert e["max_rel"] <= compare.TOL["bf16"], e

@@ -53,7 +53,7 @@ def check_sampled(w, d, targets, label):
     for mode, storage in (("stored", w.dtype), ("exact", None)):
         ref, mag = O.infer_at(w.indptr, w.indices, w.edge_weights, w.x_as_f32(), w.layers, targets, storage=storage,
                               threshold=w.threshold, follow_reorder=storage is not None, magnitudes=True)
-        err = assert_close(got, ref, mag, w.dtype, mode, label=label)
+        err = assert_close(got, ref, mag, w.dtype, mode, label=label, n_layers=len(w.layers))
         print(f"{label} ({mode}):", err)
     # properties that hold at any size: finite everywhere, and identical on a second run
     assert bool(torch.isfinite(d.out.float()).all())
@@ -94,7 +94,7 @@ def check_compact(w, d, targets, label, out=None, layers=None):
     for mode, storage in (("stored", w.dtype), ("exact", None)):
         ref, mag = O.infer_at(cip, cix, cw, xc, layers, ct, storage=storage, threshold=w.threshold,
                               follow_reorder=storage is not None, magnitudes=True)
-        err = assert_close(got, ref, mag, w.dtype, mode, label=label)
+        err = assert_close(got, ref, mag, w.dtype, mode, label=label, n_layers=len(layers))
         print(f"{label} full size ({mode}):", err, "rows", d.n_rows, "split owners", d.n_split_owners, "compact vertices", len(ids))
     assert bool(torch.isfinite(out.float().sum()))
 

@@ -80,7 +80,7 @@ def test_medium_shape_with_edge_features_sampled():
     for mode, storage in (("stored", w.dtype), ("exact", None)):
         ref, mag = O.infer_at(cip, cix, cw, w.x[ids], w.layers, ct, storage=storage, threshold=w.threshold,
                               follow_reorder=storage is not None, edge_feat=cef, magnitudes=True)
-        assert_close(got, ref, mag, w.dtype, mode)
+        assert_close(got, ref, mag, w.dtype, mode, n_layers=len(w.layers))
     first = d.out.clone()
     d.infer()
     torch.cuda.synchronize()

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import (TOL, assert_close, check_against_oracle, make_gat_layer, make_plain_layer, make_sage_layer, run_device, run_oracle,
+from gpu_util import (TOL, assert_close, check_against_oracle, check_each_layer, make_gat_layer, make_plain_layer, make_sage_layer, run_device, run_oracle,
                       small_workload, to_numpy)
 from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
@@ -141,8 +141,9 @@ def test_embed_gnn_predict_pipeline():
                   make_plain_layer(46, "gcn", "relu", 64, 32, dtype, weights=True),
                   make_plain_layer(47, "dense", "none", 32, 8, dtype)]
         w = small_workload(48, 2500, 18, dtype, layers, hubs=HUBS, weights=True, threshold=200)
-        got, _ = run_device(w)
+        got, d = run_device(w)
         check_against_oracle(w, got, label=dtype)
+        check_each_layer(w, d, label=dtype)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -152,6 +153,7 @@ def test_multi_layer_infer_matches_layer_by_layer_and_oracle(dtype):
     w = small_workload(14, 2100, 16, dtype, layers, hubs=HUBS, weights=True, threshold=100)
     got, d = run_device(w)
     check_against_oracle(w, got)
+    check_each_layer(w, d, label=dtype)
     # exactly the sequence of it_layer_forward calls: bit-identical
     h = d.x
     for lay, src in zip(d.layers, w.layers):
