@@ -15,7 +15,7 @@ the same metric through the C ABI from page-locked host buffers (host->device co
 and features and the device->host read of the result inside the timed region); `parity` = the
 result the timed steps left, at sampled vertices, against the CPU oracle.  A step whose kernels
 gave up a bounded wait, a non-finite result or a parity failure sets `rejected` and the exit code.
-With N > 1 every rank runs an independent replica of the workload.
+With N > 1 the ONE workload is partitioned over the ranks (vertex ranges, one NCCL exchange per layer): strong scaling.
 """
 from __future__ import annotations
 
@@ -52,6 +52,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-parity", action="store_true", help="skip the sampled check of the timed result against the CPU oracle")
     ap.add_argument("--no-others", action="store_true", help="headline workload only: no sub-records of the other workloads")
+    ap.add_argument("--layout", choices=["gather", "partial"], default=None,
+                    help="N > 1: partition destinations and all-gather the gathered table per layer (gather, the default), or partition "
+                         "sources and reduce-scatter partial results (partial).  Given with N = 1 it runs the partitioned code path on one rank")
     return ap.parse_args()
 
 
@@ -514,6 +517,148 @@ def measure(name: str, args, steps: int, world: int, rank: int, dev, full: bool)
     return rec
 
 
+def shared_workload(args, rank: int, world: int, barrier):
+    """The workload's host arrays on every rank of one node without generating them N times: rank 0 generates and
+    writes them to shared memory, the others map them read-only."""
+    from workloads import make
+    from workloads.configs import Workload
+    tag = os.environ.get("MASTER_PORT", "0")
+    root = f"/dev/shm/inferturbo_bench_{tag}"
+    if rank == 0:
+        w = make(args.workload, args.scale)
+        os.makedirs(root, exist_ok=True)
+        np.save(os.path.join(root, "indptr.npy"), w.indptr)
+        np.save(os.path.join(root, "indices.npy"), w.indices)
+        np.save(os.path.join(root, "x.npy"), w.x)
+        if w.edge_weights is not None:
+            np.save(os.path.join(root, "w.npy"), w.edge_weights)
+    barrier()
+    if rank != 0:
+        w0 = make(args.workload, min(args.scale, 1e-4))   # the model (layers, threshold, dtype) is the same at every size
+        ld = lambda f: np.load(os.path.join(root, f), mmap_mode="r")
+        ip = ld("indptr.npy")
+        ew = ld("w.npy") if os.path.exists(os.path.join(root, "w.npy")) else None
+        w = Workload(w0.name, ip.shape[0] - 1, int(ip[-1]), ip, ld("indices.npy"), ew, w0.dtype, ld("x.npy"), w0.layers, w0.threshold)
+    return w, root
+
+
+def measure_sharded(args, rank: int, world: int, dev):
+    """N > 1: ONE workload partitioned over the ranks (strong scaling): every rank owns a range of the vertices, one
+    exchange per layer over NCCL (all-gather of what the layer gathers, or reduce-scatter of partial results)."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2307_00228_b200 import binding as B
+    from paper_2307_00228_b200 import host, sharded
+
+    barrier = dist.barrier
+    w, root = shared_workload(args, rank, world, barrier)
+    if args.threshold is not None:
+        w.threshold = args.threshold
+    v0, v1 = sharded.vertex_ranges(w.n, world)[rank]
+    eng = sharded.CudaEngine(threshold=w.threshold, device=dev)
+    x_local = host.features_to_device(np.ascontiguousarray(w.x[v0:v1]), w.dtype, dev)
+    worker = sharded.Worker(rank, world, np.asarray(w.indptr), np.asarray(w.indices),
+                            None if w.edge_weights is None else np.asarray(w.edge_weights), x_local, w.layers, w.dtype, eng,
+                            layout=args.layout)
+    warmup = max(3, args.warmup)
+    for _ in range(warmup):
+        sharded.run_spmd(worker)
+    torch.cuda.synchronize()
+    problems = []
+
+    def check(label):
+        try:
+            B.it_graph_check(worker.part)
+        except B.ItError as e:
+            problems.append(f"rank {rank} {label}: {e}")
+
+    sampler = ClockSampler(None) if rank == 0 else None
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    launches0 = B.it_kernel_launch_count()
+    ev0.record()
+    for _ in range(args.steps):
+        out = sharded.run_spmd(worker)
+    ev1.record()
+    torch.cuda.synchronize()
+    barrier()
+    launches = B.it_kernel_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    check("timed steps")
+    ms_per_step = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / args.steps
+    finite = bool(torch.isfinite(out.float().sum()).item())
+    if not finite:
+        problems.append(f"rank {rank}: the result holds non-finite values")
+
+    # per-kernel breakdown of this rank's share (instrumented second loop)
+    B.it_profile_begin()
+    for _ in range(args.steps):
+        sharded.run_spmd(worker)
+    torch.cuda.synchronize()
+    stats = B.it_profile_end()
+    tot_ms = sum(s_["total_ms"] for s_ in stats) or 1.0
+    peak, peak_src = hbm_peak()
+    kernels = [{"name": s_["name"], "launches": s_["launches"], "ms_per_step": s_["total_ms"] / args.steps, "share": s_["total_ms"] / tot_ms,
+                "algo_GBps": (s_["algo_bytes"] / 1e9) / (s_["total_ms"] * 1e-3) if s_["total_ms"] > 0 else 0.0}
+               for s_ in sorted(stats, key=lambda s_: -s_["total_ms"])]
+    top = max(stats, key=lambda s_: s_["total_ms"])
+    achieved = (top["algo_bytes"] / 1e9) / (top["total_ms"] * 1e-3)
+
+    # end to end: every step copies this rank's features and its part of the CSR in and its rows of the result out
+    keep = worker.part._keep
+    host_arrays = [np.ascontiguousarray(w.x[v0:v1]) if w.dtype == "f32" else np.ascontiguousarray(w.x[v0:v1]).view(np.int16)]
+    dev_in = [worker.x0[:worker.n_loc].view(torch.int16) if w.dtype == "bf16" else worker.x0[:worker.n_loc]]
+    e0, e1 = int(w.indptr[v0]), int(w.indptr[v1])
+    host_arrays.append(np.ascontiguousarray(w.indices[e0:e1])); dev_in.append(keep[1])
+    if w.edge_weights is not None:
+        host_arrays.append(np.ascontiguousarray(w.edge_weights[e0:e1])); dev_in.append(keep[2])
+    host_in = [torch.from_numpy(a).pin_memory() for a in host_arrays]
+    host_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    h2d = sum(t_.numel() * t_.element_size() for t_ in host_in)
+    d2h = host_out.numel() * host_out.element_size()
+
+    def e2e_step():
+        for src_t, dst_t in zip(host_in, dev_in):
+            dst_t.copy_(src_t, non_blocking=True)
+        host_out.copy_(sharded.run_spmd(worker), non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    k = max(3, min(args.steps, 5))
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    a.record()
+    for _ in range(k):
+        e2e_step()
+    b.record()
+    torch.cuda.synchronize()
+    check("e2e steps")
+    e2e_ms = max_over_ranks(a.elapsed_time(b) / k, world, dev)
+    tot = torch.tensor([float(h2d), float(d2h), float(len(problems))], dtype=torch.float64, device=dev)
+    dist.all_reduce(tot)
+    barrier()
+    if rank == 0:
+        import shutil
+        shutil.rmtree(root, ignore_errors=True)
+        cfg = workload_config(w, args)
+        cfg["parallelism"] = f"{world} vertex ranges, one exchange per layer ({'all-gather' if args.layout == 'gather' else 'reduce-scatter of partial results'}, NCCL)"
+        line = {
+            "metric": METRIC, "value": w.n / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": w.dtype,
+            "data": "synthetic", "config": cfg, "clocks": clocks,
+            "e2e": {"value": w.n / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(tot[0].item()), "d2h_bytes_per_step": int(tot[1].item()),
+                    "ms_per_step": e2e_ms, "steps": k},
+            "gpu_launches": int(launches) * world,
+            "roofline": {"bound": "hbm", "kernel": top["name"], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": peak_src, "traffic": None, "note": "rank 0's share of the partitioned workload"},
+            "kernels": kernels, "cpu_baseline": None, "result_check": {"finite": finite},
+            "rejected": bool(tot[2].item() > 0), "problems": problems}
+        print(json.dumps(line))
+    return int(tot[2].item())
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -524,31 +669,36 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if world > 1 or args.layout_forced:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29531")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local))
     B.lib()
     dev = torch.device("cuda", local)
+    if world > 1 or args.layout_forced:
+        bad = measure_sharded(args, rank, world, dev)
+        dist.destroy_process_group()
+        if bad:
+            sys.exit(3)
+        return
 
-    main = measure(args.workload, args, args.steps, world, rank, dev, full=True)
+    main = measure(args.workload, args, args.steps, 1, 0, dev, full=True)
     others = {}
-    if args.workload == "large" and args.scale == 1.0 and world == 1 and not args.no_others:
+    if args.workload == "large" and args.scale == 1.0 and not args.no_others:
         for name in OTHER_WORKLOADS:
-            r = measure(name, args, min(args.steps, 10), world, rank, dev, full=False)
+            r = measure(name, args, min(args.steps, 10), 1, 0, dev, full=False)
             top = r["roofline"]
             others[name] = {"ms_per_step": r["ms_per_step"], "value": r["value"], "unit": UNIT, "steps": r["steps"],
                             "edges_per_sec_per_layer": r["edges_per_sec_per_layer"],
                             "dominant_kernel": {k: top[k] for k in ("kernel", "achieved", "frac", "dram_GBps", "dram_frac", "traffic_scaled_from")},
                             "kernels": [{k: v for k, v in kk.items() if k in ("name", "ms_per_step", "algo_GBps", "dram_frac")} for kk in r["kernels"][:4]],
                             "parity": r.get("parity"), "problems": r["problems"], "config": r["config"]["layers"], "dtype": r["dtype"]}
-    if world > 1:
-        dist.destroy_process_group()
-    if rank != 0:
-        return
-
     problems = list(main["problems"]) + [f"{n}: {p}" for n, r in others.items() for p in r["problems"]]
     line = {
-        "metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
-        "ms_per_step": main["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": main["ms_per_step"], "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
         "dtype": main["dtype"], "data": "synthetic", "config": main["config"],
         "edges_per_sec_per_layer": main["edges_per_sec_per_layer"], "clocks": main.get("clocks"), "e2e": main.get("e2e"),
         "gpu_launches": main["gpu_launches"], "roofline": main["roofline"], "kernels": main["kernels"],
@@ -563,6 +713,8 @@ def run_ours(args):
 
 def main():
     args = parse_args()
+    args.layout_forced = args.layout is not None
+    args.layout = args.layout or "gather"
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -279,14 +279,17 @@ void ito_gat_scores(int64_t n, const double *Z, int32_t heads, int32_t D, const 
 
 /* GAT reduce (done in apply_node because it is not associative): per destination v and
  * head k,
- *   e_j     = LeakyReLU_slope( s_src[u_j, k] + s_dst[v, k] )
+ *   e_j     = LeakyReLU_slope( s_src[u_j, k] + s_dst[v, k] + c[j, k] )      (c: see below; 0 when absent)
  *   alpha_j = exp(e_j - max_j e_j) / sum_j exp(e_j - max_j e_j)
  *   o_v^k   = sum_j alpha_j z_{u_j}^k
  * Empty in-neighbourhood: o_v = 0.  Z is the message table [n_src, heads*D] (it may be a
- * rounded copy of the z the scores were computed from); O is [n, heads*D]. */
+ * rounded copy of the z the scores were computed from); O is [n, heads*D].
+ * edge_logit (may be NULL) is [n_edges, heads]: the share of the edge's own features in the attention
+ * logit, c[j, k] = att_edge[k] . e_j (Eq. (1): the message function may read e_{v,u}; with attention
+ * the edge features enter the logit next to the two vertex terms). */
 void ito_gat_aggregate(int64_t n, const int64_t *indptr, const int32_t *indices, const double *Z,
                        const double *s_src, const double *s_dst, int32_t heads, int32_t D,
-                       double slope, double *O) {
+                       double slope, const double *edge_logit, double *O) {
     int32_t F = heads * D;
 #pragma omp parallel for schedule(dynamic, 256)
     for (int64_t v = 0; v < n; ++v) {
@@ -296,18 +299,18 @@ void ito_gat_aggregate(int64_t n, const int64_t *indptr, const int32_t *indices,
         for (int32_t k = 0; k < heads; ++k) {
             double emax = -INFINITY;
             for (int64_t j = j0; j < j1; ++j) {
-                double e = s_src[(int64_t)indices[j] * heads + k] + s_dst[v * heads + k];
+                double e = s_src[(int64_t)indices[j] * heads + k] + s_dst[v * heads + k] + (edge_logit ? edge_logit[j * heads + k] : 0.0);
                 e = e > 0.0 ? e : slope * e;
                 if (e > emax) emax = e;
             }
             double denom = 0.0;
             for (int64_t j = j0; j < j1; ++j) {
-                double e = s_src[(int64_t)indices[j] * heads + k] + s_dst[v * heads + k];
+                double e = s_src[(int64_t)indices[j] * heads + k] + s_dst[v * heads + k] + (edge_logit ? edge_logit[j * heads + k] : 0.0);
                 e = e > 0.0 ? e : slope * e;
                 denom += exp(e - emax);
             }
             for (int64_t j = j0; j < j1; ++j) {
-                double e = s_src[(int64_t)indices[j] * heads + k] + s_dst[v * heads + k];
+                double e = s_src[(int64_t)indices[j] * heads + k] + s_dst[v * heads + k] + (edge_logit ? edge_logit[j * heads + k] : 0.0);
                 e = e > 0.0 ? e : slope * e;
                 double alpha = exp(e - emax) / denom;
                 const double *z = Z + (int64_t)indices[j] * F + k * D;

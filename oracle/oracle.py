@@ -213,12 +213,14 @@ def gat_scores(Z, att, heads: int):
     return s
 
 
-def gat_aggregate(indptr, indices, Z, s_src, s_dst, heads: int, slope: float):
+def gat_aggregate(indptr, indices, Z, s_src, s_dst, heads: int, slope: float, edge_logit=None):
     indptr, indices, Z, s_src, s_dst = _i64(indptr), _i32(indices), _f64(Z), _f64(s_src), _f64(s_dst)
+    edge_logit = _f64(edge_logit)
     n, F = indptr.shape[0] - 1, Z.shape[1]
+    assert edge_logit is None or edge_logit.shape == (indices.shape[0], heads)
     O = np.empty((n, F), np.float64)
     lib().ito_gat_aggregate(C.c_int64(n), _p(indptr), _p(indices), _p(Z), _p(s_src), _p(s_dst),
-                            C.c_int32(heads), C.c_int32(F // heads), C.c_double(slope), _p(O))
+                            C.c_int32(heads), C.c_int32(F // heads), C.c_double(slope), _p(edge_logit), _p(O))
     return O
 
 
@@ -357,26 +359,36 @@ def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=
     return round_to(out, storage)
 
 
-def gat_layer(indptr, indices, H, layer, storage=None, rows=None):
+def gat_layer(indptr, indices, H, layer, storage=None, rows=None, edge_feat=None):
     """One GAT layer: z = h W; additive attention per head with LeakyReLU; softmax over the
     in-edges of each destination; heads concatenated; bias; activation.  `rows` as in
-    sage_layer."""
+    sage_layer.  layer.edge_dim > 0: the edge's features enter its attention logit through
+    att_edge [heads, edge_dim], e = LeakyReLU(a_src . z_u + a_dst . z_v + a_edge . e_vu)."""
     H = _f64(H)
+    De = _edge_dim(layer)
+    ef = _f64(edge_feat) if De else None
     if rows is None:
         z = linear(H, _f64(layer.W))
         s_src = gat_scores(z, layer.att_src, layer.heads)
         s_dst = gat_scores(z, layer.att_dst, layer.heads)
     else:
         need = _sources_of(indptr, indices, rows)
-        indptr, indices, _ = _sub_csr(indptr, indices, None, rows)
+        if De:
+            indptr, indices, _, ef = _sub_csr(indptr, indices, None, rows, ef)
+        else:
+            indptr, indices, _ = _sub_csr(indptr, indices, None, rows)
         z = np.full((H.shape[0], layer.out_dim), np.nan)
         z[need] = linear(H[need], _f64(layer.W))
         s_src = np.full((H.shape[0], layer.heads), np.nan)
         s_src[need] = gat_scores(z[need], layer.att_src, layer.heads)
         s_dst = gat_scores(z[_i64(rows)], layer.att_dst, layer.heads)
+    c = linear(ef, _f64(layer.att_edge).T) if De else None   # [n_edges, heads]
     if storage is not None:
         s_src, s_dst = round_f32(s_src), round_f32(s_dst)
-    O = gat_aggregate(indptr, indices, round_to(z, storage), s_src, s_dst, layer.heads, layer.leaky_slope)
+        if De:   # the contract stores ONE fp32 logit term per edge and head: source score + the edge's share
+            c = round_f32(s_src[_i32(indices).astype(np.int64)] + round_f32(c))
+            s_src = np.zeros_like(s_src)
+    O = gat_aggregate(indptr, indices, round_to(z, storage), s_src, s_dst, layer.heads, layer.leaky_slope, edge_logit=c)
     return round_to(bias_act(O, layer.bias, layer.act), storage)
 
 
@@ -439,7 +451,7 @@ def gcn_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=0
 def layer_forward(indptr, indices, edge_weights, H, layer, storage=None, threshold=0, reorder=False, rows=None,
                   edge_feat=None):
     if layer.op == "gat":
-        return gat_layer(indptr, indices, H, layer, storage, rows)
+        return gat_layer(indptr, indices, H, layer, storage, rows, edge_feat)
     if layer.op == "dense":
         return dense_layer(H, layer, storage, rows)
     if layer.op == "gcn":
@@ -474,7 +486,13 @@ def layer_magnitude(indptr, indices, edge_weights, H, layer, rows=None, edge_fea
             s_dst = gat_scores(z, layer.att_dst, layer.heads)
         else:
             s_dst = gat_scores(linear(H[_i64(rows)], _f64(layer.W)), layer.att_dst, layer.heads)
-        D = gat_aggregate(sub_ip, sub_ix, zabs, s_src, s_dst, layer.heads, layer.leaky_slope)
+        c = None
+        if _edge_dim(layer):
+            ef = _f64(edge_feat)
+            if rows is not None:
+                ef = _sub_csr(indptr, indices, None, rows, ef)[3]
+            c = linear(ef, _f64(layer.att_edge).T)
+        D = gat_aggregate(sub_ip, sub_ix, zabs, s_src, s_dst, layer.heads, layer.leaky_slope, edge_logit=c)
         return D if layer.bias is None else D + np.abs(_f64(layer.bias))[None, :]
 
     class _Abs:   # the same layer on absolute values, no activation

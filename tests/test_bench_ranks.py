@@ -1,8 +1,8 @@
 """The multi-rank side of bench.py on CPU: world_size-2 gloo ranks.
 
-The layer pass does not shard without an exchange step, so N > 1 means N independent replicas; what the
-ranks share is the timing protocol (the slowest rank's time, the whole-job value) and the rule that rank 0
-alone reports.
+With N > 1 the benchmark partitions one workload over the ranks (tests/test_sharded_cpu.py covers the partition and
+the exchanges); what is checked here is the timing protocol the ranks share (the slowest rank's time, the whole-job
+value) and the rule that rank 0 alone reports.
 """
 import json
 import os

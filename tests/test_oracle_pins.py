@@ -15,9 +15,9 @@ GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "w5.json
 
 
 def L(op="sum", act="none", W=None, bias=None, heads=1, att_src=None, att_dst=None, slope=0.2,
-      use_edge_weights=False, allow_reorder=True, edge_dim=0, W_edge=None, bias_edge=None, act_edge="none"):
+      use_edge_weights=False, allow_reorder=True, edge_dim=0, W_edge=None, bias_edge=None, act_edge="none", att_edge=None):
     W = np.asarray(W, dtype=np.float64)
-    in_dim = (W.shape[0] - edge_dim) if op in ("gat", "dense", "gcn") else (W.shape[0] - edge_dim) // 2
+    in_dim = W.shape[0] if op == "gat" else ((W.shape[0] - edge_dim) if op in ("dense", "gcn") else (W.shape[0] - edge_dim) // 2)
     if W_edge is not None:   # learned messages: W_edge is [in + edge_dim, msg_dim], W is [in + msg_dim, out] (GCN: [msg_dim, out])
         W_edge = np.asarray(W_edge, dtype=np.float64)
         in_dim = W_edge.shape[0] - edge_dim
@@ -29,7 +29,8 @@ def L(op="sum", act="none", W=None, bias=None, heads=1, att_src=None, att_dst=No
               bias=None if bias is None else np.asarray(bias, dtype=np.float64), heads=heads,
               att_src=None if att_src is None else np.asarray(att_src, dtype=np.float64),
               att_dst=None if att_dst is None else np.asarray(att_dst, dtype=np.float64),
-              leaky_slope=slope, use_edge_weights=use_edge_weights, allow_reorder=allow_reorder)
+              leaky_slope=slope, use_edge_weights=use_edge_weights, allow_reorder=allow_reorder,
+              att_edge=None if att_edge is None else np.asarray(att_edge, dtype=np.float64))
 
 
 def random_graph(rng, n, max_deg, p_zero=0.2):
@@ -125,8 +126,10 @@ def tree_eval(v, depth, ip, ix, w, x, layers, memo=None, ef=None):
         for hd in range(lay.heads):
             sd = sum(lay.att_dst[hd][c] * zv[hd * D + c] for c in range(D))
             es = []
-            for z in zn:
+            for jj, z in zip(range(ip[v], ip[v + 1]), zn):
                 e = sum(lay.att_src[hd][c] * z[hd * D + c] for c in range(D)) + sd
+                if getattr(lay, "edge_dim", 0):
+                    e += sum(lay.att_edge[hd][f] * float(ef[jj][f]) for f in range(lay.edge_dim))
                 es.append(e if e > 0 else lay.leaky_slope * e)
             if es:
                 m = max(es)
@@ -836,3 +839,67 @@ def test_linear_messages_reduce_to_the_plain_aggregates():
     We2[Fi] += 1.0
     d = O.edge_messages(ix, None, x, ef, We2, be, "none") - O.edge_messages(ix, None, x, ef, We, be, "none")
     assert np.allclose(d, np.repeat(ef[:, :1], Fm, axis=1), rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------ GAT with edge features in the logits
+
+def gat_edge_layer(rng, fi, heads, hd, De, act="none"):
+    return L("gat", act, rng.standard_normal((fi, heads * hd)), rng.standard_normal(heads * hd), heads=heads,
+             att_src=rng.standard_normal((heads, hd)), att_dst=rng.standard_normal((heads, hd)), edge_dim=De,
+             att_edge=rng.standard_normal((heads, De)))
+
+
+@pytest.mark.parametrize("depth", [1, 2])
+def test_gat_with_edge_logits_equals_computation_tree(depth):
+    rng = np.random.default_rng(500 + depth)
+    n, De = 12, 3
+    ip, ix = random_graph(rng, n, 4)
+    ef = rng.standard_normal((ix.shape[0], De))
+    x = rng.standard_normal((n, 4))
+    layers = [gat_edge_layer(rng, 4, 2, 2, De, act="elu"), gat_edge_layer(rng, 4, 1, 3, De)][:depth]
+    full = O.infer(ip, ix, None, x, layers, edge_feat=ef)[-1]
+    at = O.infer_at(ip, ix, None, x, layers, np.arange(n), edge_feat=ef)
+    stored = O.infer(ip, ix, None, x, layers, storage="f32", edge_feat=ef)[-1]
+    for v in range(n):
+        ref = np.array(tree_eval(v, depth, ip, ix, None, x, layers, ef=ef))
+        assert np.allclose(full[v], ref, rtol=1e-11, atol=1e-12), (depth, v)
+        assert np.allclose(at[v], ref, rtol=1e-11, atol=1e-12), (depth, v)
+        assert np.allclose(stored[v], ref, rtol=2e-5, atol=2e-5), (depth, v)
+
+
+def test_gat_edge_logit_special_cases():
+    rng = np.random.default_rng(51)
+    n, De = 30, 2
+    ip, ix = random_graph(rng, n, 5)
+    x = rng.standard_normal((n, 4))
+    ef = rng.standard_normal((ix.shape[0], De))
+    lay = gat_edge_layer(rng, 4, 2, 3, De)
+    plain = L("gat", "none", lay.W, lay.bias, heads=2, att_src=lay.att_src, att_dst=lay.att_dst)
+    base = O.gat_layer(ip, ix, x, plain)
+    # zero edge features, or a zero attention vector for them: the plain GAT layer
+    assert np.array_equal(O.gat_layer(ip, ix, x, lay, edge_feat=np.zeros_like(ef)), base)
+    zero_att = L("gat", "none", lay.W, lay.bias, heads=2, att_src=lay.att_src, att_dst=lay.att_dst, edge_dim=De, att_edge=np.zeros((2, De)))
+    assert np.array_equal(O.gat_layer(ip, ix, x, zero_att, edge_feat=ef), base)
+    # a softmax is unchanged by a shift of all its logits: with positive logits throughout (where the LeakyReLU is
+    # the identity) an edge term that is the same for all in-edges of a destination changes nothing
+    pos = L("gat", "none", lay.W, lay.bias, heads=2, att_src=np.zeros((2, 3)), att_dst=np.zeros((2, 3)), edge_dim=1, att_edge=np.ones((2, 1)))
+    const = np.repeat(rng.random(n) + 1.0, np.diff(ip))[:, None]     # one value per destination
+    flat = L("gat", "none", lay.W, lay.bias, heads=2, att_src=np.zeros((2, 3)), att_dst=np.zeros((2, 3)))
+    assert np.allclose(O.gat_layer(ip, ix, x, pos, edge_feat=const), O.gat_layer(ip, ix, x, flat), rtol=1e-12, atol=1e-12)
+    # two in-edges, logits from the edge features alone: alpha = sigmoid of their difference
+    ip2, ix2 = np.array([0, 2, 2], np.int64), np.array([0, 1], np.int32)
+    x2 = np.array([[1.0, 2.0], [3.0, -1.0]])
+    lay2 = L("gat", "none", np.eye(2), None, heads=1, att_src=[[0, 0]], att_dst=[[0, 0]], edge_dim=1, att_edge=[[1.0]])
+    e = np.array([[0.7], [1.9]])
+    a0 = 1.0 / (1.0 + math.exp(1.9 - 0.7))
+    out = O.gat_layer(ip2, ix2, x2, lay2, edge_feat=e)
+    assert np.allclose(out[0], a0 * x2[0] + (1 - a0) * x2[1], rtol=1e-14)
+    # a hugely negative edge term removes the edge from the softmax: the graph without that edge
+    ef_big = np.zeros((ix.shape[0], 1))
+    v = int(np.argmax(np.diff(ip)))
+    ef_big[ip[v]] = -1e4
+    drop = L("gat", "none", lay.W, lay.bias, heads=2, att_src=lay.att_src, att_dst=lay.att_dst, edge_dim=1, att_edge=np.ones((2, 1)))
+    got = O.gat_layer(ip, ix, x, drop, edge_feat=ef_big)[v]
+    ip3 = ip.copy(); ip3[v + 1:] -= 1
+    ix3 = np.delete(ix, ip[v])
+    assert np.allclose(got, O.gat_layer(ip3, ix3, x, plain)[v], rtol=1e-12, atol=1e-12)

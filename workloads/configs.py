@@ -29,6 +29,7 @@ class Layer:
     att_src: np.ndarray | None = None   # float32 [heads, out/heads]
     att_dst: np.ndarray | None = None
     leaky_slope: float = 0.2
+    att_edge: np.ndarray | None = None  # GAT with edge features: float32 [heads, edge_dim]
     use_edge_weights: bool = False
     allow_reorder: bool = True
     edge_dim: int = 0        # > 0: the message carries the edge's feature vector; W has edge_dim more neighbour rows
