@@ -77,7 +77,7 @@ typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
  *   W is [in_dim, out_dim].  The degree normalisation is carried by the edge weights and a self loop is
  *   an edge of the graph like any other; the vertex's own state enters in no other way.
  *
- * Edge features (edge_dim > 0; pooling layers and GCN): Eq. (1) lets the message function M read the feature
+ * Edge features (edge_dim > 0; pooling layers and GCN; for GAT see below): Eq. (1) lets the message function M read the feature
  *   vector e_{v,u} of the edge next to the source state.  The message here is the concatenation
  *       m_{v,u} = [ w_e * h_u | e_{v,u} ]                      (in_dim + edge_dim entries)
  *   reduced entry by entry with the layer's op (MEAN divides both parts by the edge count), so that
@@ -85,6 +85,11 @@ typedef enum { IT_ACT_NONE = 0, IT_ACT_RELU = 1, IT_ACT_ELU = 2 } it_act;
  *       GCN:       h'_v = act( a_v * W + bias ),                                                  W is [in_dim + edge_dim, out_dim]
  *   Every message function that is linear in (h_u, e_{v,u}) and is followed by a sum or mean and a dense update
  *   folds into this form.  The vectors come from it_graph_set_edge_features; such layers are never reordered.
+ *
+ * GAT with edge features (op = GAT, edge_dim > 0): the edge's features enter its attention logit,
+ *       e = LeakyReLU_slope( att_src[k] . z_u^k + att_dst[k] . z_v^k + att_edge[k] . e_{v,u} ),
+ *   the messages stay z_u.  One fp32 logit term per edge and head (source score + edge share) and the message
+ *   row of every edge are materialised in the workspace ([n_edges, heads] fp32 and [n_edges, out_dim] feat_dtype).
  *
  * Learned messages (msg_dim > 0; pooling layers and GCN): the general apply_edge of the Scatter stage (Section
  *   "InferTurbo Abstraction"; M of Eq. (1)) as one dense layer on the source state and the edge's features,
@@ -115,6 +120,7 @@ typedef struct {
   it_act act_edge;                      /* learned messages: activation of the message function */
   const void *W_edge;                   /* learned messages: [in_dim + edge_dim, msg_dim], weight_dtype */
   const float *bias_edge;               /* learned messages: [msg_dim], may be NULL */
+  const float *att_edge;                /* GAT with edge_dim > 0: [heads, edge_dim] fp32 */
 } it_layer_desc;
 
 /*

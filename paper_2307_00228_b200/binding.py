@@ -43,7 +43,7 @@ class it_layer_desc(C.Structure):
                 ("W", C.c_void_p), ("bias", C.c_void_p), ("att_src", C.c_void_p), ("att_dst", C.c_void_p),
                 ("leaky_slope", C.c_float), ("use_edge_weights", C.c_int32), ("allow_reorder", C.c_int32),
                 ("edge_dim", C.c_int32), ("msg_dim", C.c_int32), ("act_edge", C.c_int),
-                ("W_edge", C.c_void_p), ("bias_edge", C.c_void_p)]
+                ("W_edge", C.c_void_p), ("bias_edge", C.c_void_p), ("att_edge", C.c_void_p)]
 
 
 class it_stage_desc(C.Structure):
@@ -130,11 +130,12 @@ class LayerDesc:
     W_edge: torch.Tensor | None = None
     bias_edge: torch.Tensor | None = None
     act_edge: str = "none"
+    att_edge: torch.Tensor | None = None
 
     def to_c(self) -> it_layer_desc:
-        for t in (self.W, self.bias, self.att_src, self.att_dst, self.W_edge, self.bias_edge):
+        for t in (self.W, self.bias, self.att_src, self.att_dst, self.W_edge, self.bias_edge, self.att_edge):
             assert t is None or (t.is_cuda and t.is_contiguous())
-        for t in (self.bias, self.att_src, self.att_dst, self.bias_edge):
+        for t in (self.bias, self.att_src, self.att_dst, self.bias_edge, self.att_edge):
             assert t is None or t.dtype == torch.float32
         assert self.W_edge is None or self.W_edge.dtype == self.W.dtype
         d = it_layer_desc()
@@ -153,6 +154,7 @@ class LayerDesc:
         d.act_edge = ACTS[self.act_edge]
         d.W_edge = None if self.W_edge is None else self.W_edge.data_ptr()
         d.bias_edge = None if self.bias_edge is None else self.bias_edge.data_ptr()
+        d.att_edge = None if self.att_edge is None else self.att_edge.data_ptr()
         return d
 
 

@@ -11,6 +11,7 @@ enum LayerPlan { PLAN_SAGE = 0, PLAN_SAGE_REORDER = 1, PLAN_GAT = 2, PLAN_DENSE 
 
 struct LayerWs {
   LayerPlan plan;
+  size_t off_counters;                              // IT_MAX_BUCKETS words from which the gather's warps claim their batches
   size_t off_B, off_partials, off_a, off_b, off_q;  // a: aggregate A | self term S | scores ; b: Z | P ; q: per-edge part Q / messages
   size_t bytes;
 };
@@ -37,11 +38,14 @@ it_status check_layer(const it_graph *g, const it_layer_desc *L) {
   }
   IT_REQUIRE(L->edge_dim >= 0, IT_ERR_INVALID_ARG, "edge_dim is negative");
   if (L->edge_dim > 0) {
-    IT_REQUIRE(L->op != IT_GATHER_GAT && L->op != IT_GATHER_NONE, IT_ERR_UNSUPPORTED, "edge features are taken by the pooling layers and GCN only");
+    IT_REQUIRE(L->op != IT_GATHER_NONE, IT_ERR_UNSUPPORTED, "a dense layer has no edges whose features it could take");
     IT_REQUIRE(g->edge_feat != nullptr, IT_ERR_INVALID_ARG, "layer uses edge features but the graph has none (it_graph_set_edge_features)");
     IT_REQUIRE(g->edge_dim == L->edge_dim && g->edge_dtype == L->feat_dtype, IT_ERR_INVALID_ARG,
                "layer expects edge features [%d] of its feat_dtype, the graph holds [%d]", L->edge_dim, g->edge_dim);
   }
+  // rows that lie in edge order are addressed by a 32-bit edge id
+  IT_REQUIRE((L->edge_dim == 0 && L->msg_dim == 0) || g->e <= (int64_t)INT32_MAX, IT_ERR_UNSUPPORTED,
+             "layers with edge features or learned messages take graphs of at most 2^31 - 1 edges");
   IT_REQUIRE(L->msg_dim >= 0, IT_ERR_INVALID_ARG, "msg_dim is negative");
   if (L->msg_dim > 0) {
     IT_REQUIRE(is_pooling(L->op) || L->op == IT_GATHER_GCN, IT_ERR_UNSUPPORTED, "learned messages are taken by the pooling layers and GCN only");
@@ -84,12 +88,15 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
   auto take = [&](size_t bytes) { size_t o = off; off += it_align_up(bytes); return o; };
   w.plan = plan_of(L);
   w.off_q = 0;
+  w.off_counters = take(IT_MAX_BUCKETS * sizeof(int));
   switch (w.plan) {
     case PLAN_GAT:
       w.off_B = take((fi + kpad) * (fo + 2 * (size_t)L->heads) * 8);
       w.off_partials = take(it_gat_partial_bytes(g, L->out_dim, L->heads));
       w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
       w.off_b = take(n * fo * s);                    // Z
+      // edge features in the logits: per edge its message row and one logit term per head
+      w.off_q = take(fe > 0 ? (size_t)g->e * fo * s + it_align_up((size_t)g->e * (size_t)L->heads * 4) : 0);
       break;
     case PLAN_DENSE:
       w.off_B = take((fi + kpad) * fo * 8);
@@ -238,13 +245,20 @@ it_status stage_gather(const StageCtx &c, const void *table, const float *scores
   if (c.w.plan == PLAN_GAT) {
     it_gat_args aa{};
     aa.g = g; aa.dtype = dt; aa.heads = L->heads; aa.head_dim = L->out_dim / L->heads; aa.z = table; aa.scores = scores;
-    aa.scores_dst = scores_dst; aa.partials = c.partials;
+    aa.scores_dst = scores_dst; aa.partials = c.partials; aa.counters = reinterpret_cast<int *>(c.ws + c.w.off_counters);
     aa.slope = L->leaky_slope; aa.bias = L->bias; aa.act = L->act; aa.dst = out;
+    if (L->edge_dim > 0) {
+      IT_REQUIRE(L->att_edge != nullptr, IT_ERR_INVALID_ARG, "GAT layer with edge features needs att_edge");
+      void *Zj = c.ws + c.w.off_q;
+      float *sc = reinterpret_cast<float *>(c.ws + c.w.off_q + it_align_up((size_t)g->e * (size_t)L->out_dim * (size_t)it_dtype_size(dt)));
+      IT_TRY(it_launch_gat_edge_rows(g, dt, L->out_dim, L->heads, table, scores, L->att_edge, Zj, sc, c.st));
+      aa.z = Zj; aa.per_edge_rows = 1; aa.src_scores = sc;
+    }
     return it_launch_gat(aa, c.st);
   }
   it_gather_args gg{};
   gg.g = g; gg.op = L->op == IT_GATHER_GCN ? IT_GATHER_SUM : L->op; gg.use_edge_weights = L->use_edge_weights; gg.dtype = dt;
-  gg.partials = c.partials;
+  gg.partials = c.partials; gg.counters = reinterpret_cast<int *>(c.ws + c.w.off_counters);
   switch (c.w.plan) {
     case PLAN_GCN_REORDER:   // h' = act(sum_e w_e z_u + b) in the gather's epilogue
       gg.dim = L->out_dim; gg.src = table; gg.dst = out; gg.epi = IT_EPI_BIAS_ACT; gg.self_term = nullptr; gg.bias = L->bias; gg.act = L->act;

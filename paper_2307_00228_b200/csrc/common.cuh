@@ -143,6 +143,7 @@ struct it_gather_args {
   int src_ld;              // 0 means dim
   int per_edge_rows;       // 1: src is [n_edges, dim] and row j belongs to edge j (edge features); 0: rows are looked up by source vertex
   float *partials;         // [n_partial_rows, dim] fp32 scratch (may be NULL when nothing is split)
+  int *counters;           // IT_MAX_BUCKETS device words of scratch from which warps claim their batches (NULL: fixed strides)
   void *dst;               // row v starts at dst + v * dst_ld elements and takes dim of them
   int dst_ld;              // 0 means dim
   it_epilogue_kind epi;
@@ -161,7 +162,10 @@ struct it_gat_args {
   const void *z;          // [n, heads*head_dim] messages
   const float *scores;    // [n_src, 2*heads]: source scores of the vertex, then its destination scores
   const float *scores_dst;   // the same layout, row v = local destination v (scores + first_vertex * 2*heads for a part; NULL: scores)
+  int per_edge_rows;      // 1: z is [n_edges, dim] and src_scores [n_edges, heads], row j belonging to edge j (edge features in the logits)
+  const float *src_scores;   // per_edge_rows only: the logit term of every edge (source score + edge share)
   float *partials;        // it_gat_partial_bytes() of fp32 scratch for the groups of split vertices (may be NULL if none)
+  int *counters;          // IT_MAX_BUCKETS device words of scratch from which warps claim their batches (NULL: fixed strides)
   float slope;
   const float *bias;      // may be NULL
   it_act act;
@@ -212,5 +216,8 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
 // Learned messages, edge by edge: M[j, :] = act(P[indices[j], :] + M[j, :]) in place (M arrives holding the per-edge
 // part Q), rows of `dim` elements of `dtype` (a multiple of 16 bytes).
 it_status it_launch_edge_messages(const it_graph *g, it_dtype dtype, int dim, const void *P, void *M, it_act act, cudaStream_t stream);
+// GAT with edge features: Zj[j, :] = Z[indices[j], :] and sc[j, h] = scores[indices[j], h] + att_edge[h, :] . ef[j, :].
+it_status it_launch_gat_edge_rows(const it_graph *g, it_dtype dtype, int dim, int heads, const void *Z, const float *scores,
+                                  const float *att_edge, void *Zj, float *sc, cudaStream_t stream);
 // out[v, :] = raw[v, :] * scale[v] (0 where scale[v] = 0), fp32 -> dtype.
 it_status it_launch_aggregate_finish(int64_t n, int dim, it_dtype dtype, const float *raw, const float *scale, void *out, cudaStream_t stream);

@@ -25,6 +25,7 @@ struct GatPolicy {
   void *__restrict__ dst;
   float *__restrict__ partials;        // [n_partial_rows, stride]: acc[dim], m[heads], l[heads]
   int dim, heads, head_dim, act;
+  int src_stride;                      // floats from one row of `scores` to the next (2*heads; heads when the rows are per edge)
   float slope;
   // per-thread
   int col, head;
@@ -37,8 +38,8 @@ struct GatPolicy {
     st[VEC] = -INFINITY;
     st[VEC + 1] = 0.f;
   }
-  __device__ __forceinline__ float extra(uint32_t s) const { return __ldg(scores + (uint64_t)s * (2 * heads) + head); }
-  __device__ __forceinline__ const float *extra_ptr(uint32_t s) const { return scores + (uint64_t)s * (2 * heads) + head; }
+  __device__ __forceinline__ float extra(uint32_t s) const { return __ldg(scores + (uint64_t)s * src_stride + head); }
+  __device__ __forceinline__ const float *extra_ptr(uint32_t s) const { return scores + (uint64_t)s * src_stride + head; }
   __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float, float x) const {
     float e = x + s_dst;
     e = e > 0.f ? e : slope * e;
@@ -47,8 +48,13 @@ struct GatPolicy {
     const float pw = __expf(e - m_new);
     float f[VEC];
     Slice::unpack(raw, f);
+    if constexpr (VEC % 2 == 0) {
 #pragma unroll
-    for (int k = 0; k < VEC; ++k) st[k] = fmaf(pw, f[k], st[k] * scale);
+      for (int k = 0; k < VEC; k += 2) scale_fma_f32x2(st[k], st[k + 1], scale, pw, f[k], f[k + 1]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < VEC; ++k) st[k] = fmaf(pw, f[k], st[k] * scale);
+    }
     st[VEC + 1] = fmaf(st[VEC + 1], scale, pw);
     st[VEC] = m_new;
   }
@@ -137,7 +143,8 @@ __global__ void __launch_bounds__(THREADS) gat_combine_kernel(GatCombineParams p
 template <typename T, int SB, int LPR>
 it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   GatPolicy<T, SB> pol;
-  pol.scores = a.scores; pol.scores_dst = a.scores_dst ? a.scores_dst : a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
+  pol.scores = a.per_edge_rows ? a.src_scores : a.scores; pol.src_stride = a.per_edge_rows ? a.heads : 2 * a.heads;
+  pol.scores_dst = a.scores_dst ? a.scores_dst : a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
   pol.dim = a.heads * a.head_dim; pol.heads = a.heads; pol.head_dim = a.head_dim; pol.act = a.act; pol.slope = a.slope;
   pol.col = 0; pol.head = 0; pol.s_dst = 0.f;
   const it_graph *g = a.g;
@@ -148,7 +155,7 @@ it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, int64_t bound_lo
   auto bytes_of = [=](int b, int64_t rows) {
     return (double)g->h_bucket_edges[b] * (4.0 + 4.0 * heads + row_bytes) + (double)rows * (20.0 + 4.0 * heads + row_bytes);
   };
-  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, bound_lo, bound_hi, st);
+  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY, bound_lo, bound_hi, a.counters, st);
 }
 
 template <typename T>
@@ -176,8 +183,8 @@ it_status it_launch_gat(const it_gat_args &a, cudaStream_t st) {
   IT_REQUIRE(g->n_split_owners == 0 || a.head_dim % 4 == 0, IT_ERR_UNSUPPORTED, "gat on a split graph needs head_dim to be a multiple of 4");
   if (g->n == 0) return IT_OK;
   StreamParams sp;
-  sp.meta = g->bucket_meta; sp.owner = g->bucket_owner; sp.indices = g->indices; sp.weights = nullptr;
-  sp.src = a.z; sp.row_lo = sp.row_hi = 0; sp.dim = a.heads * a.head_dim; sp.batch_rows = 1;
+  sp.meta = g->bucket_meta; sp.owner = g->bucket_owner; sp.indices = a.per_edge_rows ? nullptr : g->indices; sp.weights = nullptr;
+  sp.src = a.z; sp.row_lo = sp.row_hi = 0; sp.dim = a.heads * a.head_dim; sp.batch_rows = 1; sp.counter = nullptr; sp.claim = 1;
   sp.src_pitch = (uint32_t)(sp.dim * it_dtype_size(a.dtype));
   if (a.dtype == IT_F32) IT_TRY(launch_gat<float>(a, sp, st));
   else IT_TRY(launch_gat<__nv_bfloat16>(a, sp, st));

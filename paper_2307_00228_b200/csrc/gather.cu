@@ -36,11 +36,16 @@ struct SagePolicy {
   __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float w, float) const {
     float f[VEC];
     Slice::unpack(raw, f);
+    if constexpr (RED == RED_SUM && !WEIGHTED && VEC % 2 == 0) {   // two accumulators per instruction (measured: 1 % on the
+#pragma unroll                                                      // 128-byte rows; with a weight the pair set-up eats the gain)
+      for (int k = 0; k < VEC; k += 2) add_f32x2(st[k], st[k + 1], f[k], f[k + 1]);
+    } else {
 #pragma unroll
-    for (int k = 0; k < VEC; ++k) {
-      if (RED == RED_MAX) st[k] = fmaxf(st[k], WEIGHTED ? w * f[k] : f[k]);
-      else if (RED == RED_MIN) st[k] = fminf(st[k], WEIGHTED ? w * f[k] : f[k]);
-      else st[k] = WEIGHTED ? fmaf(w, f[k], st[k]) : st[k] + f[k];
+      for (int k = 0; k < VEC; ++k) {
+        if (RED == RED_MAX) st[k] = fmaxf(st[k], WEIGHTED ? w * f[k] : f[k]);
+        else if (RED == RED_MIN) st[k] = fminf(st[k], WEIGHTED ? w * f[k] : f[k]);
+        else st[k] = WEIGHTED ? fmaf(w, f[k], st[k]) : st[k] + f[k];
+      }
     }
   }
   __device__ __forceinline__ void merge(float (&st)[NS], const float (&o)[NS]) const {
@@ -166,7 +171,7 @@ it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_
     return (double)g->h_bucket_edges[b] * ((a.per_edge_rows ? 0.0 : 4.0) + (WEIGHTED ? 4.0 : 0.0) + row_bytes) +
            (double)rows * (16.0 + row_bytes + (a.epi == IT_EPI_ADD_ACT ? 4.0 * a.dim : 0.0));
   };
-  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, bound_lo, bound_hi, st);
+  return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, bound_lo, bound_hi, a.counters, st);
 }
 
 template <typename T>
@@ -187,7 +192,7 @@ static it_status launch_gather_chunk(const it_gather_args &a, cudaStream_t st) {
   const it_graph *g = a.g;
   StreamParams sp;
   sp.meta = g->bucket_meta; sp.owner = nullptr; sp.indices = a.per_edge_rows ? nullptr : g->indices; sp.weights = g->edge_weights;
-  sp.src = a.src; sp.row_lo = sp.row_hi = 0; sp.dim = a.dim; sp.batch_rows = 1;
+  sp.src = a.src; sp.row_lo = sp.row_hi = 0; sp.dim = a.dim; sp.batch_rows = 1; sp.counter = nullptr; sp.claim = 1;
   sp.src_pitch = (uint32_t)((a.src_ld > 0 ? a.src_ld : a.dim) * it_dtype_size(a.dtype));
   if (a.dtype == IT_F32) IT_TRY(launch_lpr<float>(a, sp, st));
   else IT_TRY(launch_lpr<__nv_bfloat16>(a, sp, st));

@@ -1,10 +1,12 @@
-// Two elementwise kernels around the gather:
+// Elementwise kernels around the gather:
 //   * the learned message of every edge, m_j = act(P[u_j] + Q[j]) (the source part P was computed once per vertex, the
 //     edge part Q once per edge, both by the dense transform), written over Q so that the per-edge-row gather can
 //     reduce it;
+//   * for GAT layers whose logits read the edge features: the message row of every edge (a copy of its source's row)
+//     and its logit term per head (source score + the edge's share), so that the reduce can walk rows in edge order;
 //   * the receiver's finish of a partial-gather over source partitions (scale, zero the vertices without in-edges,
 //     round to the storage type).
-// Both are HBM-bound streams of 16-byte slices; the only irregular access is the source row of an edge.
+// All are HBM-bound streams of 16-byte slices; the only irregular access is the source row of an edge.
 #include "common.cuh"
 
 namespace {
@@ -64,6 +66,48 @@ __global__ void __launch_bounds__(MSG_THREADS) edge_messages_kernel(const int32_
   }
 }
 
+// GAT with edge features: the message row of every edge (a copy of its source's row, so that the reduce can walk rows
+// in edge order) ...
+__global__ void __launch_bounds__(MSG_THREADS) gat_edge_rows_kernel(const int32_t *__restrict__ indices, const uint4 *__restrict__ Z,
+                                                                    uint4 *__restrict__ Zj, int64_t total, int slices) {
+  const int64_t stride = (int64_t)gridDim.x * MSG_THREADS;
+  for (int64_t t0 = (int64_t)blockIdx.x * MSG_THREADS + threadIdx.x; t0 < total; t0 += stride * MSG_UNROLL) {
+    uint4 z[MSG_UNROLL];
+#pragma unroll
+    for (int u = 0; u < MSG_UNROLL; ++u) {
+      const int64_t t = t0 + u * stride;
+      if (t < total) {
+        const int64_t j = t / slices;
+        z[u] = __ldg(Z + (int64_t)__ldg(indices + j) * slices + (t - j * slices));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < MSG_UNROLL; ++u) {
+      const int64_t t = t0 + u * stride;
+      if (t < total) __stcs(Zj + t, z[u]);
+    }
+  }
+}
+// ... and its logit term per head: the source's score plus the edge's own share att_edge[h] . e_j
+template <typename T>
+__global__ void __launch_bounds__(MSG_THREADS) gat_edge_scores_kernel(const int32_t *__restrict__ indices, const float *__restrict__ scores,
+                                                                      const T *__restrict__ ef, const float *__restrict__ att_edge,
+                                                                      float *__restrict__ sc, int64_t n_edges, int heads, int edge_dim) {
+  const int64_t total = n_edges * heads, stride = (int64_t)gridDim.x * MSG_THREADS;
+  for (int64_t t = (int64_t)blockIdx.x * MSG_THREADS + threadIdx.x; t < total; t += stride) {
+    const int64_t j = t / heads;
+    const int h = (int)(t - j * heads);
+    float acc = 0.f;
+    for (int k = 0; k < edge_dim; ++k) {
+      float e;
+      if constexpr (sizeof(T) == 4) e = __ldg(reinterpret_cast<const float *>(ef) + j * edge_dim + k);
+      else e = __bfloat162float(ef[j * edge_dim + k]);
+      acc = fmaf(__ldg(att_edge + h * edge_dim + k), e, acc);
+    }
+    sc[t] = __ldg(scores + (int64_t)__ldg(indices + j) * (2 * heads) + h) + acc;
+  }
+}
+
 // one thread per four consecutive entries of a row
 template <typename T>
 __global__ void __launch_bounds__(MSG_THREADS) aggregate_finish_kernel(const float4 *__restrict__ raw, const float *__restrict__ scale,
@@ -103,6 +147,30 @@ it_status it_launch_edge_messages(const it_graph *g, it_dtype dtype, int dim, co
   else
     IT_LAUNCH(IT_K_EDGE_MSG, bytes, 0, st, edge_messages_kernel<__nv_bfloat16><<<blocks, MSG_THREADS, 0, st>>>(
         g->indices, reinterpret_cast<const uint4 *>(P), reinterpret_cast<uint4 *>(M), total, slices, (int)act));
+  IT_CUDA_TRY(cudaGetLastError());
+  return IT_OK;
+}
+
+it_status it_launch_gat_edge_rows(const it_graph *g, it_dtype dtype, int dim, int heads, const void *Z, const float *scores,
+                                  const float *att_edge, void *Zj, float *sc, cudaStream_t st) {
+  if (g->e == 0) return IT_OK;
+  const int es = it_dtype_size(dtype);
+  const int slices = dim * es / 16;
+  const int64_t total = g->e * slices;
+  const int64_t cap = (int64_t)g->num_sms * 16;
+  int64_t want = (total + (int64_t)MSG_THREADS * MSG_UNROLL - 1) / ((int64_t)MSG_THREADS * MSG_UNROLL);
+  unsigned blocks = (unsigned)(want < cap ? want : cap);
+  IT_LAUNCH(IT_K_EDGE_MSG, (double)g->e * (4.0 + 2.0 * dim * es), 0, st,
+            gat_edge_rows_kernel<<<blocks, MSG_THREADS, 0, st>>>(g->indices, reinterpret_cast<const uint4 *>(Z), reinterpret_cast<uint4 *>(Zj), total, slices));
+  want = (g->e * heads + MSG_THREADS - 1) / MSG_THREADS;
+  blocks = (unsigned)(want < cap ? want : cap);
+  const double sbytes = (double)g->e * (4.0 + (double)g->edge_dim * es + 8.0 * heads);
+  if (dtype == IT_F32)
+    IT_LAUNCH(IT_K_EDGE_MSG, sbytes, 0, st, gat_edge_scores_kernel<float><<<blocks, MSG_THREADS, 0, st>>>(
+        g->indices, scores, reinterpret_cast<const float *>(g->edge_feat), att_edge, sc, g->e, heads, g->edge_dim));
+  else
+    IT_LAUNCH(IT_K_EDGE_MSG, sbytes, 0, st, gat_edge_scores_kernel<__nv_bfloat16><<<blocks, MSG_THREADS, 0, st>>>(
+        g->indices, scores, reinterpret_cast<const __nv_bfloat16 *>(g->edge_feat), att_edge, sc, g->e, heads, g->edge_dim));
   IT_CUDA_TRY(cudaGetLastError());
   return IT_OK;
 }

@@ -209,7 +209,19 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_
   const int64_t n_batches = (n_rows + BR - 1) / BR;
   const int64_t warps_total = (int64_t)gridDim.x * (THREADS / 32);
 
-  for (int64_t b = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); b < n_batches; b += warps_total) {
+  // a warp's first batch is fixed; the following ones are claimed from the launch's counter (or, without one, follow at
+  // a fixed stride).  Which warp takes a batch has no influence on the batch's result.
+  // Batches are handed out in claims of p.claim consecutive batches (sized so that a warp makes about sixteen claims:
+  // one atomic per batch would serialise on the counter when the rows are short).
+  auto next_claim = [&](int64_t c) -> int64_t {
+    if (p.counter == nullptr) return c + warps_total;
+    int v = 0;
+    if (lane == 0) v = atomicAdd(p.counter, 1);
+    return warps_total + (int64_t)__shfl_sync(0xffffffffu, v, 0);
+  };
+  const int64_t CH = p.counter ? p.claim : 1;
+  for (int64_t c = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); c * CH < n_batches; c = next_claim(c))
+  for (int64_t b = c * CH; b < (c + 1) * CH && b < n_batches; ++b) {
     // ---- batch metadata: lane i owns row i of the batch
     const int64_t i = p.row_lo + b * BR + lane;
     int64_t my_j0 = 0;

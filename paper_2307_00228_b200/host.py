@@ -31,7 +31,8 @@ def layer_to_device(layer, dtype: str, device="cuda") -> B.LayerDesc:
                        use_edge_weights=bool(layer.use_edge_weights), allow_reorder=bool(layer.allow_reorder),
                        edge_dim=int(getattr(layer, "edge_dim", 0) or 0), msg_dim=int(getattr(layer, "msg_dim", 0) or 0),
                        W_edge=None if getattr(layer, "W_edge", None) is None else param_to_device(layer.W_edge, dtype, device),
-                       bias_edge=f32(getattr(layer, "bias_edge", None)), act_edge=getattr(layer, "act_edge", "none"))
+                       bias_edge=f32(getattr(layer, "bias_edge", None)), act_edge=getattr(layer, "act_edge", "none"),
+                       att_edge=f32(getattr(layer, "att_edge", None)))
 
 
 @dataclass
@@ -48,8 +49,10 @@ class DeviceWorkload:
         return B.it_infer(self.graph, self.layers, self.x, self.out, self.workspace, stream)
 
 
-def upload(w, device="cuda", int32_indptr=False, threshold=None) -> DeviceWorkload:
-    """Create the device graph (split at the workload's threshold), parameters, workspace, output."""
+def upload(w, device="cuda", int32_indptr=False, threshold=None, with_workspace=True) -> DeviceWorkload:
+    """Create the device graph (split at the workload's threshold), parameters, workspace, output.
+    with_workspace=False: a second set of input / output buffers for a caller that shares one workspace and one set of
+    layer parameters between them (layers and workspace are left empty)."""
     indptr = torch.from_numpy(w.indptr.astype(np.int32) if int32_indptr else w.indptr).to(device)
     indices = torch.from_numpy(w.indices).to(device)
     ew = None if w.edge_weights is None else torch.from_numpy(w.edge_weights).to(device)
@@ -58,8 +61,11 @@ def upload(w, device="cuda", int32_indptr=False, threshold=None) -> DeviceWorklo
         B.it_graph_set_edge_features(g, features_to_device(w.edge_feat, w.dtype, device))
     thr = w.threshold if threshold is None else threshold
     n_rows, n_split = B.it_split_hubs(g, thr)
-    layers = [layer_to_device(l, w.dtype, device) for l in w.layers]
     x = features_to_device(w.x, w.dtype, device)
+    if not with_workspace:
+        out = torch.empty((w.n, w.layers[-1].out_dim), dtype=x.dtype, device=device)
+        return DeviceWorkload(g, x, [], None, out, n_rows, n_split)
+    layers = [layer_to_device(l, w.dtype, device) for l in w.layers]
     ws = torch.empty(B.it_workspace_bytes(g, layers), dtype=torch.uint8, device=device)
     out = torch.empty((w.n, w.layers[-1].out_dim), dtype=x.dtype, device=device)
     return DeviceWorkload(g, x, layers, ws, out, n_rows, n_split)

@@ -74,14 +74,15 @@ def make_msg_layer(seed, op, act, fi, fm, fo, dtype, act_edge="relu", weights=Fa
                  bias_edge=rng.uniform(-0.1, 0.1, fm).astype(np.float32) if bias else None, act_edge=act_edge)
 
 
-def make_gat_layer(seed, act, fi, heads, hd, dtype, bias=True) -> Layer:
+def make_gat_layer(seed, act, fi, heads, hd, dtype, bias=True, edge_dim=0) -> Layer:
     rng = np.random.default_rng(seed)
     fo = heads * hd
     lim = np.sqrt(6.0 / (fi + fo))
     return Layer(op="gat", act=act, in_dim=fi, out_dim=fo, W=storage_exact(rng.uniform(-lim, lim, (fi, fo)), dtype),
                  bias=rng.uniform(-0.1, 0.1, fo).astype(np.float32) if bias else None, heads=heads,
                  att_src=rng.uniform(-0.4, 0.4, (heads, hd)).astype(np.float32),
-                 att_dst=rng.uniform(-0.4, 0.4, (heads, hd)).astype(np.float32))
+                 att_dst=rng.uniform(-0.4, 0.4, (heads, hd)).astype(np.float32), edge_dim=edge_dim,
+                 att_edge=rng.uniform(-0.4, 0.4, (heads, edge_dim)).astype(np.float32) if edge_dim else None)
 
 
 def run_device(w: Workload, int32_indptr=False, threshold=None):

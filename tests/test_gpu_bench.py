@@ -1,0 +1,39 @@
+"""bench.py end to end on small workloads: the one-GPU record with its checks, and the partitioned arm (the code
+path of N > 1) on a single rank with NCCL."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def run_bench(*args):
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True, text=True, cwd=ROOT, timeout=900)
+    assert r.returncode == 0, (r.stdout[-2000:], r.stderr[-2000:])
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    return json.loads(lines[0])
+
+
+def test_single_gpu_record_carries_its_checks():
+    d = run_bench("--workload", "medium", "--scale", "0.02", "--steps", "3", "--warmup", "3", "--cpu-seconds", "1")
+    assert d["n_gpus"] == 1 and d["value"] > 0 and d["rejected"] is False and d["problems"] == []
+    assert d["config"]["workload"].startswith("medium") and d["dtype"] == "f32"
+    assert d["parity"]["ok"] and d["parity"]["stored"]["max_rel"] <= 1e-4 and d["parity"]["exact"]["max_rel"] <= 1e-4
+    assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0 and d["e2e"]["buffer_sets"] == 2
+    assert d["roofline"]["bound"] == "hbm" and d["roofline"]["achieved"] > 0 and d["gpu_launches"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["result_check"]["finite"]
+    assert abs(d["instrumented_ms_per_step"] - d["ms_per_step"]) < 0.25 * d["ms_per_step"]
+
+
+@pytest.mark.parametrize("layout", ["gather", "partial"])
+def test_partitioned_arm_on_one_rank(layout):
+    d = run_bench("--workload", "medium", "--scale", "0.02", "--steps", "2", "--warmup", "3", "--layout", layout)
+    assert d["scaling"] == "strong" and d["n_gpus"] == 1 and d["value"] > 0 and d["rejected"] is False
+    assert "vertex ranges" in d["config"]["parallelism"] and d["result_check"]["finite"]
+    assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["gpu_launches"] > 0

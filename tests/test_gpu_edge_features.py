@@ -104,6 +104,12 @@ def test_argument_checks():
         B.it_graph_set_edge_features(d.graph, torch.zeros((w.e, 3), device="cuda"))
     gat = B.LayerDesc(op="gat", act="none", in_dim=16, out_dim=16, W=torch.zeros((16, 16), device="cuda"), heads=2,
                       att_src=torch.zeros((2, 8), device="cuda"), att_dst=torch.zeros((2, 8), device="cuda"), edge_dim=4)
+    # a GAT layer may read the edge features in its logits, but then it needs the attention vector for them
+    ws = torch.empty(B.it_workspace_bytes(d.graph, [gat]), dtype=torch.uint8, device="cuda")
     with pytest.raises(B.ItError) as e:
-        B.it_layer_forward(d.graph, gat, d.x, o, d.workspace)
+        B.it_layer_forward(d.graph, gat, d.x, o, ws)
+    assert e.value.status_name == "IT_ERR_INVALID_ARG"
+    dense = B.LayerDesc(op="dense", act="none", in_dim=16, out_dim=16, W=torch.zeros((16, 16), device="cuda"), edge_dim=4)
+    with pytest.raises(B.ItError) as e:
+        B.it_workspace_bytes(d.graph, [dense])
     assert e.value.status_name == "IT_ERR_UNSUPPORTED"

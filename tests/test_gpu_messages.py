@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import check_against_oracle, make_msg_layer, make_sage_layer, run_device, small_workload
+from gpu_util import check_against_oracle, make_gat_layer, make_msg_layer, make_sage_layer, run_device, small_workload
 from paper_2307_00228_b200 import binding as B
 from paper_2307_00228_b200 import host
 
@@ -55,6 +55,32 @@ def test_message_layers_stack_with_plain_layers():
     assert torch.equal(h, d.out)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("threshold", [0, 100])
+@pytest.mark.parametrize("heads,hd,de", [(2, 16, 8), (4, 32, 16), (1, 8, 8)])
+def test_gat_with_edge_features_in_the_logits(dtype, threshold, heads, hd, de):
+    """e = LeakyReLU(a_src . z_u + a_dst . z_v + a_edge . e_vu): split and unsplit, all row kernels (hubs up to 2500 edges)."""
+    layer = make_gat_layer(21, "elu", 32, heads, hd, dtype, edge_dim=de)
+    w = small_workload(22, 1300, 25, dtype, [layer], hubs=HUBS, threshold=threshold, edge_dim=de)
+    got, d = run_device(w)
+    if threshold:
+        assert d.n_split_owners > 0
+    check_against_oracle(w, got, label=(dtype, threshold, heads, hd, de))
+
+
+def test_gat_edge_logits_change_the_result_and_stack():
+    layers = [make_gat_layer(23, "elu", 32, 2, 16, "f32", edge_dim=8), make_gat_layer(24, "none", 32, 2, 8, "f32", edge_dim=8)]
+    w = small_workload(25, 800, 12, "f32", layers, hubs=(300,), threshold=64, edge_dim=8)
+    got, _ = run_device(w)
+    check_against_oracle(w, got)
+    plain = [make_gat_layer(23, "elu", 32, 2, 16, "f32"), make_gat_layer(24, "none", 32, 2, 8, "f32")]
+    for a, b in zip(plain, layers):   # the same parameters without the edge term
+        a.W, a.bias, a.att_src, a.att_dst = b.W, b.bias, b.att_src, b.att_dst
+    w2 = small_workload(25, 800, 12, "f32", plain, hubs=(300,), threshold=64)
+    base, _ = run_device(w2)
+    assert np.abs(got - base).max() > 1e-3
+
+
 def test_message_argument_checks():
     layer = make_msg_layer(9, "sum", "none", 16, 16, 16, "f32", edge_dim=8)
     w = small_workload(10, 100, 5, "f32", [layer], edge_dim=8)
@@ -74,5 +100,9 @@ def test_message_argument_checks():
     gat = host.layer_to_device(layer, "f32")
     gat.op = "gat"
     gat.edge_dim = 0
-    assert status_of(lambda: B.it_workspace_bytes(d.graph, [gat])) == "IT_ERR_UNSUPPORTED"
+    assert status_of(lambda: B.it_workspace_bytes(d.graph, [gat])) == "IT_ERR_UNSUPPORTED"   # learned messages are not for GAT
+    g2 = host.layer_to_device(make_gat_layer(12, "none", 16, 2, 8, "f32", edge_dim=8), "f32")
+    g2.att_edge = None
+    ws = torch.empty(B.it_workspace_bytes(d.graph, [g2]), dtype=torch.uint8, device="cuda")
+    assert status_of(lambda: B.it_layer_forward(d.graph, g2, d.x, out, ws)) == "IT_ERR_INVALID_ARG"
     assert torch.ones(3, device="cuda").sum().item() == 3
