@@ -194,7 +194,7 @@ it_status it_workspace_bytes(const it_graph *g, const it_layer_desc *layers, int
  * If allow_reorder and op is SUM, MEAN or GCN and out_dim < in_dim, the neighbour transform is
  * done before the gather (Section "Inference" allows the order of a layer's computation to be
  * rearranged for speed): Z = h_in * W[in_dim:, :] is stored in feat_dtype and gathered instead of
- * h_in; the self term h_in * W[0:in_dim, :] + bias stays fp32.
+ * h_in; the self term h_in * W[0:in_dim, :] + bias is stored in feat_dtype as well.
  * Asynchronous on `stream`.  Results are bit-identical from run to run.
  */
 it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const void *h_in,

@@ -10,9 +10,9 @@ Storage points.  The method itself is exact, but a deployment stores layer input
 outputs in a narrow type.  `storage=None` keeps everything in fp64 (mode A).  With
 `storage='f32'|'bf16'` (mode B) the oracle still accumulates in fp64 but rounds to the
 storage type (nearest even) at the points where the layer contract says a tensor is
-stored: the aggregate handed to apply, the transformed rows Z (GAT and
-transform-before-aggregate) and the layer output.  The self term of a reordered layer
-and the GAT scores are contract-fp32 and are rounded to fp32.
+stored: the aggregate handed to apply, the transformed rows Z and the self term (GAT and
+transform-before-aggregate) and the layer output.  The GAT scores are contract-fp32 and
+are rounded to fp32.
 """
 from __future__ import annotations
 
@@ -350,8 +350,7 @@ def sage_layer(indptr, indices, edge_weights, H, layer, storage=None, threshold=
         S = linear(Hself, W[:Fi])
         if layer.bias is not None:
             S = S + _f64(layer.bias)[None, :]
-        if storage is not None:
-            S = round_f32(S)
+        S = round_to(S, storage)   # the contract stores the self term like every other vertex table
         out = bias_act(S + _gathered(indptr, indices, w, Z, layer.op, threshold), None, layer.act)
     else:
         A = round_to(_gathered(indptr, indices, w, H, layer.op, threshold), storage)

@@ -117,7 +117,7 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
     case PLAN_SAGE_REORDER:
       w.off_B = take((fi + kpad) * 2 * fo * 8);
       w.off_partials = take((size_t)g->n_partial_rows * fo * 4);
-      w.off_a = take(n * fo * 4);  // S (fp32)
+      w.off_a = take(n * fo * s);  // S (the self term, stored like the rows)
       w.off_b = take(n * fo * s);  // Z
       break;
     case PLAN_SAGE:
@@ -220,9 +220,9 @@ it_status stage_transform(const StageCtx &c, const void *h_self, void *table_out
       ga.n0 = 0; ga.out0 = nullptr; ga.dt0 = dt; ga.bias0 = nullptr; ga.act0 = IT_ACT_NONE;
       ga.n1 = L->out_dim; ga.out1 = table_out; ga.dt1 = dt; ga.out2 = nullptr;
       return run_apply(g, L, IT_PREP_DENSE, ga, c.B, nullptr, c.st);
-    case PLAN_SAGE_REORDER:  // S = H W_self + b (fp32, stays with the vertex), Z = H W_neigh
+    case PLAN_SAGE_REORDER:  // S = H W_self + b (stays with the vertex), Z = H W_neigh
       ga.NB = 2 * L->out_dim;
-      ga.n0 = L->out_dim; ga.out0 = c.ws + c.w.off_a; ga.dt0 = IT_F32; ga.bias0 = L->bias; ga.act0 = IT_ACT_NONE;
+      ga.n0 = L->out_dim; ga.out0 = c.ws + c.w.off_a; ga.dt0 = dt; ga.bias0 = L->bias; ga.act0 = IT_ACT_NONE;
       ga.n1 = L->out_dim; ga.out1 = table_out; ga.dt1 = dt; ga.out2 = nullptr;
       return run_apply(g, L, IT_PREP_SAGE_REORDER, ga, c.B, nullptr, c.st);
     case PLAN_MSG:
@@ -265,7 +265,7 @@ it_status stage_gather(const StageCtx &c, const void *table, const float *scores
       return it_launch_gather(gg, c.st);
     case PLAN_SAGE_REORDER:
       gg.dim = L->out_dim; gg.src = table; gg.dst = out; gg.epi = IT_EPI_ADD_ACT;
-      gg.self_term = reinterpret_cast<const float *>(c.ws + c.w.off_a); gg.act = L->act;
+      gg.self_term = c.ws + c.w.off_a; gg.self_dtype = dt; gg.act = L->act;
       return it_launch_gather(gg, c.st);
     case PLAN_MSG:
       gg.dim = L->msg_dim; gg.dst = out; gg.dst_ld = L->msg_dim; gg.epi = IT_EPI_STORE; gg.act = IT_ACT_NONE;

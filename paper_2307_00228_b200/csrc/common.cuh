@@ -127,7 +127,7 @@ static inline int it_dtype_size(it_dtype t) { return t == IT_F32 ? 4 : 2; }
 // What a gather / combine kernel does with the finished aggregate of vertex v.
 enum it_epilogue_kind {
   IT_EPI_STORE = 0,      // dst[v, :] = agg                      (feat dtype)
-  IT_EPI_ADD_ACT = 1,    // dst[v, :] = act(self[v, :] + agg)    (self fp32, dst feat dtype)
+  IT_EPI_ADD_ACT = 1,    // dst[v, :] = act(self[v, :] + agg)    (self fp32 or feat dtype, dst feat dtype)
   IT_EPI_BIAS_ACT = 2,   // dst[v, :] = act(bias + agg)          (bias fp32 [dim] or NULL)
   IT_EPI_RAW_F32 = 3     // dst[v, :] = the raw reduce in fp32: plain sum (mean undivided), max or min, and the identity of
                          // the reduce (0, -inf, +inf) for a row without edges: one part's share of a partial-gather
@@ -147,7 +147,8 @@ struct it_gather_args {
   void *dst;               // row v starts at dst + v * dst_ld elements and takes dim of them
   int dst_ld;              // 0 means dim
   it_epilogue_kind epi;
-  const float *self_term;  // fp32, IT_EPI_ADD_ACT only: row v starts at self_term + v * self_ld
+  const void *self_term;   // IT_EPI_ADD_ACT only: row v starts at self_term + v * self_ld elements of self_dtype
+  it_dtype self_dtype;     // IT_F32, or the dtype of the rows (the self term of a transform-first layer is stored like the rows)
   int self_ld;             // 0 means dim
   const float *bias;       // [dim] fp32 or NULL, IT_EPI_BIAS_ACT only
   it_act act;              // IT_EPI_ADD_ACT and IT_EPI_BIAS_ACT

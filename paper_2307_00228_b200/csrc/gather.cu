@@ -19,9 +19,10 @@ struct SagePolicy {
   static constexpr bool WEIGHTED = WEIGHTED_, HAS_EXTRA = false, NEEDS_OWNER = false;
   float *__restrict__ partials;
   void *__restrict__ dst;
-  const float *__restrict__ self_term;
+  const void *__restrict__ self_term;
   const float *__restrict__ bias;
   int dim, dst_ld, self_ld, is_mean, epi, act;   // dim: width of this column chunk; *_ld: row lengths of dst / the self term
+  int self_is_t;                                 // the self term is stored in T (else fp32)
   // per-thread
   int col;
   float self[VEC];
@@ -54,7 +55,12 @@ struct SagePolicy {
   }
   // the matching slice of the self term is fetched when the row starts, so that end_row does not wait for it
   __device__ __forceinline__ void begin_row(int32_t dest, int32_t) {
-    if (epi == IT_EPI_ADD_ACT && dest >= 0) load_floats_stream<VEC>(self_term + (int64_t)dest * self_ld + col, self);
+    if (epi == IT_EPI_ADD_ACT && dest >= 0) {
+      if (sizeof(T) == 2 && self_is_t)
+        Slice::unpack(Slice::load(reinterpret_cast<const char *>(self_term) + ((int64_t)dest * self_ld + col) * (int64_t)sizeof(T)), self);
+      else
+        load_floats_stream<VEC>(reinterpret_cast<const float *>(self_term) + (int64_t)dest * self_ld + col, self);
+    }
   }
   __device__ __forceinline__ void end_row(float (&st)[NS], int32_t dest, int32_t, int64_t len) const {
     if (RED != RED_SUM && len == 0 && epi != IT_EPI_RAW_F32) {
@@ -94,10 +100,10 @@ struct CombineParams {
   const int64_t *__restrict__ shadow_indptr;
   const float *__restrict__ partials;
   void *__restrict__ dst;
-  const float *__restrict__ self_term;
+  const void *__restrict__ self_term;
   const float *__restrict__ bias;
   int64_t n_split_owners;
-  int dim, dst_ld, self_ld;
+  int dim, dst_ld, self_ld, self_is_t;
   int red, is_mean, epi, act;   // red: RED_SUM / RED_MAX / RED_MIN
 };
 
@@ -139,7 +145,14 @@ __global__ void __launch_bounds__(GATHER_THREADS) combine_kernel(CombineParams p
         continue;
       }
       if (p.epi == IT_EPI_ADD_ACT) {
-        float4 s = __ldg(reinterpret_cast<const float4 *>(p.self_term + v * p.self_ld + c));
+        float4 s;
+        if (sizeof(T) == 2 && p.self_is_t) {
+          const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const T *>(p.self_term) + v * p.self_ld + c));
+          s = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u), __uint_as_float(raw.y << 16),
+                          __uint_as_float(raw.y & 0xffff0000u));
+        } else {
+          s = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(p.self_term) + v * p.self_ld + c));
+        }
         o[0] = act_apply(o[0] + s.x, p.act); o[1] = act_apply(o[1] + s.y, p.act);
         o[2] = act_apply(o[2] + s.z, p.act); o[3] = act_apply(o[3] + s.w, p.act);
       } else if (p.epi == IT_EPI_BIAS_ACT) {
@@ -163,13 +176,14 @@ it_status launch_policy(const it_gather_args &a, StreamParams sp, int64_t bound_
   SagePolicy<T, SB, RED, WEIGHTED> pol;
   pol.partials = a.partials; pol.dst = a.dst; pol.self_term = a.self_term; pol.bias = a.bias; pol.dim = a.dim; pol.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; pol.self_ld = a.self_ld > 0 ? a.self_ld : a.dim;
   pol.is_mean = a.op == IT_GATHER_MEAN && a.epi != IT_EPI_RAW_F32; pol.epi = a.epi; pol.act = a.act; pol.col = 0;
+  pol.self_is_t = a.self_dtype != IT_F32;
   const it_graph *g = a.g;
   // algorithmic bytes: per edge the index, the optional weight and one source row; per row its
   // metadata and one output row (plus the self row it is added to)
   const double row_bytes = (double)a.dim * sizeof(T);
   auto bytes_of = [=](int b, int64_t rows) {
     return (double)g->h_bucket_edges[b] * ((a.per_edge_rows ? 0.0 : 4.0) + (WEIGHTED ? 4.0 : 0.0) + row_bytes) +
-           (double)rows * (16.0 + row_bytes + (a.epi == IT_EPI_ADD_ACT ? 4.0 * a.dim : 0.0));
+           (double)rows * (16.0 + row_bytes + (a.epi == IT_EPI_ADD_ACT ? (a.self_dtype == IT_F32 ? 4.0 : (double)sizeof(T)) * a.dim : 0.0));
   };
   return launch_buckets<T, SB, LPR>(g, sp, pol, bytes_of, IT_K_GATHER_CTA, IT_K_GATHER_FLAT, IT_K_GATHER_EMPTY, bound_lo, bound_hi, a.counters, st);
 }
@@ -201,7 +215,7 @@ static it_status launch_gather_chunk(const it_gather_args &a, cudaStream_t st) {
     c.split_owners = g->split_owners; c.owner_indptr = g->owner_indptr; c.shadow_indptr = g->shadow_indptr;
     c.partials = a.partials; c.dst = a.dst; c.self_term = a.self_term; c.bias = a.bias; c.n_split_owners = g->n_split_owners;
     c.dim = a.dim; c.dst_ld = a.dst_ld > 0 ? a.dst_ld : a.dim; c.self_ld = a.self_ld > 0 ? a.self_ld : a.dim;
-    c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN && a.epi != IT_EPI_RAW_F32; c.epi = a.epi; c.act = a.act;
+    c.red = a.op == IT_GATHER_MAX ? RED_MAX : (a.op == IT_GATHER_MIN ? RED_MIN : RED_SUM); c.is_mean = a.op == IT_GATHER_MEAN && a.epi != IT_EPI_RAW_F32; c.epi = a.epi; c.act = a.act; c.self_is_t = a.self_dtype != IT_F32;
     int64_t want = (g->n_split_owners + 7) / 8;
     int64_t cap = (int64_t)g->num_sms * 8;
     unsigned blocks = (unsigned)(want < cap ? want : cap);
@@ -237,7 +251,7 @@ it_status it_launch_gather(const it_gather_args &a, cudaStream_t st) {
     c.src_ld = a.src_ld > 0 ? a.src_ld : full;
     c.dst = (char *)a.dst + (size_t)c0 * (a.epi == IT_EPI_RAW_F32 ? 4 : es);
     c.dst_ld = a.dst_ld > 0 ? a.dst_ld : full;
-    c.self_term = a.self_term ? a.self_term + c0 : nullptr;
+    c.self_term = a.self_term ? (const char *)a.self_term + (size_t)c0 * (a.self_dtype == IT_F32 ? 4 : es) : nullptr;
     c.self_ld = a.self_ld > 0 ? a.self_ld : full;
     c.bias = a.bias ? a.bias + c0 : nullptr;
     IT_TRY(launch_gather_chunk(c, st));

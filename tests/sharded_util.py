@@ -69,7 +69,7 @@ class OracleEngine:
         else:
             self._store(table_out, O.linear(H, W[Fi:]), part.n)
             S = O.linear(H, W[:Fi]) + (0 if layer.bias is None else np.asarray(layer.bias, np.float64)[None, :])
-            ws["S"] = O.round_f32(S)
+            ws["S"] = O.round_to(S, self.dtype)
 
     def gather(self, part, layer, table, scores, first, raw, out, ws):
         T = self._np(table)
