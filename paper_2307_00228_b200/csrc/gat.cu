@@ -43,9 +43,13 @@ struct GatPolicy {
   __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float, float x) const {
     float e = x + s_dst;
     e = e > 0.f ? e : slope * e;
-    const float m_new = fmaxf(st[VEC], e);
-    const float scale = __expf(st[VEC] - m_new);   // exp(-inf) = 0 for the first edge; m_new is finite
-    const float pw = __expf(e - m_new);
+    // One exponential per edge: of the two factors exp(m - m_new) and exp(e - m_new) one is exp(0) = 1 and the other is
+    // exp(-|e - m|).  (First edge: m = -inf, the old state is scaled by exp(-inf) = 0.)
+    const float d = e - st[VEC];
+    const float t = __expf(-fabsf(d));
+    const bool up = d > 0.f;
+    const float scale = up ? t : 1.f, pw = up ? 1.f : t;
+    const float m_new = up ? e : st[VEC];
     float f[VEC];
     Slice::unpack(raw, f);
     if constexpr (VEC % 2 == 0) {
