@@ -230,8 +230,11 @@ def hbm_peak():
 
 
 def traffic_records() -> dict:
-    """Lines `traffic <workload>:<kernel> <DRAM bytes per launch at full size> from=<scale> l2hit=<pct at that scale>[,<pct at half of it>]`
-    of profiles/traffic.md (ncu captures of small cases, scaled to the full workload by the units processed)."""
+    """Lines `traffic <workload>:<kernel> ratio=<DRAM bytes / algorithmic bytes of a launch> from=<scale of the capture>
+    l2hit=<L2 hit rate at that capture>,<at the smaller one>` of profiles/traffic.md: ncu captures of reduced sizes (the
+    full-size workloads are beyond the size rule for multi-metric captures).  A launch's DRAM traffic is that ratio times
+    its algorithmic bytes; the ratio rises with the size of the capture (the L2 serves less and less of the gathered
+    rows), so the figure is a lower bound at full size."""
     out = {}
     path = os.path.join(ROOT, "profiles", "traffic.md")
     if not os.path.exists(path):
@@ -239,11 +242,13 @@ def traffic_records() -> dict:
     for line in open(path):
         parts = line.split()
         if len(parts) >= 3 and parts[0] == "traffic":
-            rec = {"bytes": float(parts[2])}
-            for extra in parts[3:]:
+            rec = {}
+            for extra in parts[2:]:
                 k, _, v = extra.partition("=")
                 rec[k] = v
-            out[parts[1]] = rec
+            if "ratio" in rec:
+                rec["ratio"] = float(rec["ratio"])
+                out[parts[1]] = rec
     return out
 
 
@@ -412,7 +417,7 @@ def measure(name: str, args, steps: int, world: int, rank: int, dev, full: bool)
              "algo_GBps": (s["algo_bytes"] / 1e9) / (s["total_ms"] * 1e-3) if s["total_ms"] > 0 else 0.0}
         t = traffic.get(f"{w.name}:{s['name']}")
         if t is not None and s["total_ms"] > 0:
-            k["dram_GBps"] = t["bytes"] * s["launches"] / 1e9 / (s["total_ms"] * 1e-3)
+            k["dram_GBps"] = t["ratio"] * k["algo_GBps"]
             k["dram_frac"] = k["dram_GBps"] / peak
         kernels.append(k)
     rec["kernels"] = kernels
@@ -421,15 +426,19 @@ def measure(name: str, args, steps: int, world: int, rank: int, dev, full: bool)
     achieved = (top["algo_bytes"] / 1e9) / (top["total_ms"] * 1e-3)
     t = traffic.get(f"{w.name}:{top['name']}")
     per_launch_ms = top["total_ms"] / max(1, top["launches"])
+    algo_per_launch = top["algo_bytes"] / max(1, top["launches"])
     rec["roofline"] = {
         "bound": "hbm", "kernel": top["name"], "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_source": peak_src, "traffic": None if t is None else t["bytes"],
-        "dram_GBps": None if t is None else t["bytes"] / 1e9 / (per_launch_ms * 1e-3),
-        "dram_frac": None if t is None else t["bytes"] / 1e9 / (per_launch_ms * 1e-3) / peak,
+        "peak_source": peak_src, "traffic": None if t is None else t["ratio"] * algo_per_launch,
+        "dram_GBps": None if t is None else t["ratio"] * achieved,
+        "dram_frac": None if t is None else t["ratio"] * achieved / peak,
+        "traffic_over_algorithmic": None if t is None else t["ratio"],
         "traffic_scaled_from": None if t is None else t.get("from"), "l2_hit_pct_at_capture": None if t is None else t.get("l2hit"),
-        "algo_bytes_per_launch": top["algo_bytes"] / max(1, top["launches"]), "ms_per_launch": per_launch_ms,
-        "note": "achieved = algorithmic bytes / event time (the L2 serves part of the gathered rows, so it can exceed the DRAM rate); "
-                "dram_* = ncu DRAM bytes of a smaller capture scaled to a full launch / the same event time"}
+        "algo_bytes_per_launch": algo_per_launch, "ms_per_launch": per_launch_ms,
+        "note": "achieved = algorithmic bytes / event time; traffic = the DRAM bytes of a launch: the ratio DRAM / algorithmic bytes that ncu "
+                "measured on a reduced-size capture (traffic_scaled_from) times the algorithmic bytes of a full-size launch.  The ratio "
+                "rises with the size of the capture (the L2 serves a share of the gathered rows that falls with the table size: "
+                "l2_hit_pct_at_capture, larger capture first), so dram_frac is a lower bound and frac the value it tends to"}
 
     # ---- per-layer edges/s (each layer alone, same buffers as a real pass)
     layer_stats = []
@@ -743,7 +752,7 @@ def run_ours(args):
             top = r["roofline"]
             others[name] = {"ms_per_step": r["ms_per_step"], "value": r["value"], "unit": UNIT, "steps": r["steps"],
                             "edges_per_sec_per_layer": r["edges_per_sec_per_layer"],
-                            "dominant_kernel": {k: top[k] for k in ("kernel", "achieved", "frac", "dram_GBps", "dram_frac", "traffic_scaled_from")},
+                            "dominant_kernel": {k: top[k] for k in ("kernel", "achieved", "frac", "dram_GBps", "dram_frac", "traffic_over_algorithmic", "traffic_scaled_from", "l2_hit_pct_at_capture")},
                             "kernels": [{k: v for k, v in kk.items() if k in ("name", "ms_per_step", "algo_GBps", "dram_frac")} for kk in r["kernels"][:4]],
                             "parity": r.get("parity"), "problems": r["problems"], "config": r["config"]["layers"], "dtype": r["dtype"]}
     problems = list(main["problems"]) + [f"{n}: {p}" for n, r in others.items() for p in r["problems"]]

@@ -701,7 +701,8 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
         IT_LAUNCH(kid_cta, bytes, 0, st, stream_cta_kernel<T, SB, LPR, Policy><<<blocks, THREADS, 0, st>>>(p, pol));
       }
     } else {
-      // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row
+      // about 256 edges per batch at most: 32 rows of <= 8 edges, 8 rows of <= 32, one longer row (measured: walking
+      // several longer rows as one stream, to pay the dependent loads at the start of a row once per batch, is slower)
       int br = bound <= 8 ? 32 : (bound <= 32 ? 8 : 1);
       if constexpr (SB == 16 && (LPR == 8 || (LPR == 16 && IT_SHORT_256 != 0))) {   // 128-byte rows (and 256-byte rows)
         if (bound <= IT_SHORT_BELOW) {   // one lane group per row
