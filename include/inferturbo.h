@@ -202,11 +202,15 @@ it_status it_layer_forward(const it_graph *g, const it_layer_desc *layer, const 
 
 /*
  * it_infer — L layers in order (Section "InferTurbo on Graph Processing System": one layer
- * per iteration over all vertices, a k-layer model after k of them): exactly the sequence of
+ * per iteration over all vertices, a k-layer model after k of them): the sequence of
  * it_layer_forward calls, intermediate layer outputs double-buffered inside the
  * workspace.  x [n, layers[0].in_dim]; out [n, layers[L-1].out_dim]; layers[i].out_dim must
  * equal layers[i+1].in_dim and all feat_dtype agree.  Bit-identical to calling
- * it_layer_forward layer by layer.  Asynchronous on `stream`.
+ * it_layer_forward layer by layer.  Where layer i + 1 transforms before it aggregates (its table is
+ * H_i W), the output H_i of layer i feeds that transform and nothing else; for bf16 layers whose
+ * widths are multiples of 64 the update of layer i and that transform then run as one kernel that
+ * rounds each tile of H_i to bf16 as it would be stored and keeps it on the SM, so H_i is neither
+ * written to nor read from device memory (same results, bit for bit).  Asynchronous on `stream`.
  */
 it_status it_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, const void *x,
                    void *out, void *workspace, size_t workspace_bytes, void *stream);
@@ -336,6 +340,9 @@ it_status it_graph_check(it_graph *g, void *stream);
  */
 it_status it_debug_expire_wait(it_graph *g, it_dtype dtype, const void *x, void *out, void *workspace, size_t workspace_bytes,
                                void *stream);
+/* The same hook for the kernel that it_infer uses where the update of one layer and the transform of the next run as one
+ * (two products back to back, bf16): x and out are device [128, 64] bf16. */
+it_status it_debug_expire_wait_fused(it_graph *g, const void *x, void *out, void *workspace, size_t workspace_bytes, void *stream);
 
 /* Frees the library-owned arrays of the graph.  NULL is accepted. */
 it_status it_graph_destroy(it_graph *g);

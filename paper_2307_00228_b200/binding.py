@@ -26,7 +26,7 @@ EXPORTS = ["it_graph_create", "it_split_hubs", "it_graph_get_split", "it_workspa
            "it_infer", "it_graph_destroy", "it_status_string", "it_last_error_message", "it_profile_begin",
            "it_profile_end", "it_kernel_launch_count", "it_layer_forward_static", "it_graph_check",
            "it_graph_set_edge_features", "it_debug_expire_wait", "it_graph_create_part", "it_layer_stages",
-           "it_layer_transform", "it_layer_gather", "it_layer_update", "it_aggregate_finish"]
+           "it_layer_transform", "it_layer_gather", "it_layer_update", "it_aggregate_finish", "it_debug_expire_wait_fused"]
 
 
 class ItError(RuntimeError):
@@ -352,6 +352,15 @@ def it_debug_expire_wait(g: Graph, x: torch.Tensor, out: torch.Tensor, workspace
     L.it_debug_expire_wait.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     _check(L.it_debug_expire_wait(g.handle, _dt(x.dtype), _ptr(x), _ptr(out), _ptr(workspace),
                                   workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def it_debug_expire_wait_fused(g: Graph, x: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """Test hook: the same for the kernel that runs two products back to back (bf16 [128, 64] in and out)."""
+    L = lib()
+    L.it_debug_expire_wait_fused.restype = C.c_int
+    L.it_debug_expire_wait_fused.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    _check(L.it_debug_expire_wait_fused(g.handle, _ptr(x), _ptr(out), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def it_graph_destroy(g: Graph):

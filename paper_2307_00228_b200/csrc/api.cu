@@ -96,7 +96,10 @@ LayerWs plan_layer(const it_graph *g, const it_layer_desc *L) {
       w.off_a = take(n * 2 * (size_t)L->heads * 4);  // scores
       w.off_b = take(n * fo * s);                    // Z
       // edge features in the logits: per edge its message row and one logit term per head
-      w.off_q = take(fe > 0 ? (size_t)g->e * fo * s + it_align_up((size_t)g->e * (size_t)L->heads * 4) : 0);
+      // ... or, without them, the source scores of every vertex on their own (read per edge at random: half the bytes
+      // of the interleaved score rows, and small enough to stay in the L2)
+      w.off_q = take(fe > 0 ? (size_t)g->e * fo * s + it_align_up((size_t)g->e * (size_t)L->heads * 4)
+                            : (size_t)g->n_src * (size_t)L->heads * 4);
       break;
     case PLAN_DENSE:
       w.off_B = take((fi + kpad) * fo * 8);
@@ -237,7 +240,9 @@ it_status stage_transform(const StageCtx &c, const void *h_self, void *table_out
 }
 
 // ---- stage 2: the Gather stage.  out: the aggregate [n, agg_dim] (plans with an update), else the layer output.
-it_status stage_gather(const StageCtx &c, const void *table, const float *scores, const float *scores_dst, bool raw, void *out) {
+// `self_term`: where a transform-first GraphSAGE layer finds S (NULL: its place in the workspace, where stage_transform puts it).
+it_status stage_gather(const StageCtx &c, const void *table, const float *scores, const float *scores_dst, bool raw, void *out,
+                       const void *self_term = nullptr) {
   const it_graph *g = c.g;
   const it_layer_desc *L = c.L;
   const it_dtype dt = L->feat_dtype;
@@ -253,6 +258,10 @@ it_status stage_gather(const StageCtx &c, const void *table, const float *scores
       float *sc = reinterpret_cast<float *>(c.ws + c.w.off_q + it_align_up((size_t)g->e * (size_t)L->out_dim * (size_t)it_dtype_size(dt)));
       IT_TRY(it_launch_gat_edge_rows(g, dt, L->out_dim, L->heads, table, scores, L->att_edge, Zj, sc, c.st));
       aa.z = Zj; aa.per_edge_rows = 1; aa.src_scores = sc;
+    } else {
+      float *dense = reinterpret_cast<float *>(c.ws + c.w.off_q);
+      IT_TRY(it_launch_compact_scores(g->n_src, L->heads, scores, dense, c.st));
+      aa.src_scores = dense;
     }
     return it_launch_gat(aa, c.st);
   }
@@ -265,7 +274,7 @@ it_status stage_gather(const StageCtx &c, const void *table, const float *scores
       return it_launch_gather(gg, c.st);
     case PLAN_SAGE_REORDER:
       gg.dim = L->out_dim; gg.src = table; gg.dst = out; gg.epi = IT_EPI_ADD_ACT;
-      gg.self_term = c.ws + c.w.off_a; gg.self_dtype = dt; gg.act = L->act;
+      gg.self_term = self_term ? self_term : c.ws + c.w.off_a; gg.self_dtype = dt; gg.act = L->act;
       return it_launch_gather(gg, c.st);
     case PLAN_MSG:
       gg.dim = L->msg_dim; gg.dst = out; gg.dst_ld = L->msg_dim; gg.epi = IT_EPI_STORE; gg.act = IT_ACT_NONE;
@@ -341,12 +350,56 @@ it_status layer_forward_impl(const it_graph *g, const it_layer_desc *L, const vo
   return stage_update(c, h_in, agg, h_out);
 }
 
-struct InferWs { size_t layer_bytes, buf_bytes, off_buf0, off_buf1, bytes; };
+// ---- the update of layer a and the transform of layer b = a + 1 as one kernel
+// When layer b transforms before it aggregates, the output H of layer a is read by that transform and by nothing
+// else, so the two dense products run back to back in one kernel that keeps each tile of H on the SM (rounded to the
+// storage type exactly as it would have been stored): H is neither written nor read back.  Taken for bf16 layers
+// whose shapes fit the kernel; everything else runs layer by layer.
+#ifndef IT_FUSE_UPDATE_TRANSFORM
+#define IT_FUSE_UPDATE_TRANSFORM 1
+#endif
+
+struct FusedPair {
+  it_gemm2_args ga;        // pointers filled in by the caller
+  it_prep_kind kind_a, kind_b;
+  int nb_b;                // columns of layer b's prepared weights
+  size_t s_bytes;          // bytes of S in front of Z in the buffer that would have held H (0: layer b keeps no self term)
+};
+
+bool fused_pair(const it_graph *g, const it_layer_desc *A, const it_layer_desc *Bn, FusedPair *out) {
+  if (!IT_FUSE_UPDATE_TRANSFORM || g->n_src != g->n) return false;
+  if (A->feat_dtype != IT_BF16 || Bn->feat_dtype != IT_BF16) return false;
+  const LayerPlan pa = plan_of(A), pb = plan_of(Bn);
+  if (pa != PLAN_SAGE && pa != PLAN_GCN && pa != PLAN_DENSE) return false;
+  if (pb != PLAN_SAGE_REORDER && pb != PLAN_GCN_REORDER) return false;
+  FusedPair f{};
+  f.ga.M = g->n;
+  const int a_ld = agg_dim_of(A);
+  if (pa == PLAN_SAGE) { f.ga.K1 = A->in_dim; f.ga.K2 = a_ld; f.kind_a = IT_PREP_SAGE; }
+  else if (pa == PLAN_GCN) { f.ga.K1 = a_ld; f.ga.K2 = 0; f.kind_a = IT_PREP_DENSE; }
+  else { f.ga.K1 = A->in_dim; f.ga.K2 = 0; f.kind_a = IT_PREP_DENSE; }
+  f.ga.N1 = A->out_dim; f.ga.bias1 = A->bias; f.ga.act1 = A->act;
+  if (pb == PLAN_SAGE_REORDER) { f.ga.n0 = Bn->out_dim; f.ga.bias0 = Bn->bias; f.ga.n1 = Bn->out_dim; f.kind_b = IT_PREP_SAGE_REORDER; }
+  else { f.ga.n0 = 0; f.ga.bias0 = nullptr; f.ga.n1 = Bn->out_dim; f.kind_b = IT_PREP_DENSE; }
+  f.nb_b = f.ga.n0 + f.ga.n1;
+  f.s_bytes = it_align_up((size_t)g->n * (size_t)f.ga.n0 * 2);
+  // S and Z take the place of H, so together they must not be larger (alignment padding of S included)
+  if (f.s_bytes + (size_t)g->n * (size_t)f.ga.n1 * 2 > it_align_up((size_t)g->n * (size_t)A->out_dim * 2)) return false;
+  // probe the shape with placeholder pointers (X2 only says whether there is a second operand)
+  it_gemm2_args probe = f.ga;
+  probe.X1 = g; probe.X2 = f.ga.K2 > 0 ? (const void *)g : nullptr;
+  if (!it_tc2_supported(probe)) return false;
+  *out = f;
+  return true;
+}
+
+struct InferWs { size_t layer_bytes, buf_bytes, off_buf0, off_buf1, off_B2, bytes; };
 
 it_status plan_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_layers, InferWs *out) {
   IT_REQUIRE(g != nullptr, IT_ERR_INVALID_ARG, "graph is NULL");
   IT_REQUIRE(layers != nullptr && n_layers >= 1, IT_ERR_INVALID_ARG, "need at least one layer");
-  InferWs w{0, 0, 0, 0, 0};
+  InferWs w{0, 0, 0, 0, 0, 0};
+  size_t b2_bytes = 0;   // prepared weights of a layer whose transform runs fused with the previous layer's update
   for (int i = 0; i < n_layers; ++i) {
     IT_TRY(check_layer(g, &layers[i]));
     if (i > 0) {
@@ -360,10 +413,15 @@ it_status plan_infer(const it_graph *g, const it_layer_desc *layers, int32_t n_l
       size_t hb = it_align_up((size_t)g->n * (size_t)layers[i].out_dim * (size_t)it_dtype_size(layers[i].feat_dtype));
       if (hb > w.buf_bytes) w.buf_bytes = hb;
     }
+    if (i > 0) {
+      const size_t wb = it_align_up(((size_t)layers[i].in_dim + 128) * 2 * (size_t)layers[i].out_dim * 8);
+      if (wb > b2_bytes) b2_bytes = wb;
+    }
   }
   w.off_buf0 = w.layer_bytes;
   w.off_buf1 = w.off_buf0 + (n_layers >= 2 ? w.buf_bytes : 0);
-  w.bytes = w.off_buf1 + (n_layers >= 3 ? w.buf_bytes : 0);
+  w.off_B2 = w.off_buf1 + (n_layers >= 3 ? w.buf_bytes : 0);
+  w.bytes = w.off_B2 + b2_bytes;
   *out = w;
   return IT_OK;
 }
@@ -550,9 +608,34 @@ extern "C" it_status it_infer(const it_graph *g, const it_layer_desc *layers, in
   char *ws = (char *)workspace;
   void *buf[2] = {ws + w.off_buf0, ws + w.off_buf1};
   const void *cur = x;
+  cudaStream_t st = (cudaStream_t)stream;
   for (int i = 0; i < n_layers; ++i) {
     void *dst = (i == n_layers - 1) ? out : buf[i & 1];
-    IT_TRY(layer_forward_impl(g, &layers[i], cur, dst, ws, w.layer_bytes, (cudaStream_t)stream));
+    FusedPair f;
+    if (g->n > 0 && i + 1 < n_layers && fused_pair(g, &layers[i], &layers[i + 1], &f)) {
+      // layer i up to its aggregate; its update with the transform of layer i + 1, S and Z landing where H would have
+      // been stored; then the rest of layer i + 1
+      const it_layer_desc *A = &layers[i], *Bn = &layers[i + 1];
+      StageCtx ca, cb;
+      IT_TRY(stage_ctx(g, A, ws, w.layer_bytes, st, &ca));
+      void *agg = agg_dim_of(A) > 0 ? (void *)(ws + ca.w.off_a) : nullptr;
+      if (agg) IT_TRY(stage_gather(ca, cur, nullptr, nullptr, false, agg));
+      void *B2 = ws + w.off_B2;
+      IT_TRY(it_launch_prep_weights_tc(f.kind_a, A, f.ga.N1, f.ga.K1, f.ga.K2, ca.B, st));
+      IT_TRY(it_launch_prep_weights_tc(f.kind_b, Bn, f.nb_b, f.ga.N1, 0, B2, st));
+      char *S = (char *)dst, *Z = (char *)dst + f.s_bytes;
+      if (plan_of(A) == PLAN_GCN) { f.ga.X1 = agg; f.ga.X2 = nullptr; }
+      else { f.ga.X1 = cur; f.ga.X2 = f.ga.K2 > 0 ? agg : nullptr; }
+      f.ga.out0 = S; f.ga.out1 = Z;
+      IT_TRY(it_launch_gemm2_tc(f.ga, ca.B, B2, g->num_sms, g->d_status, st));
+      void *dst2 = (i + 1 == n_layers - 1) ? out : buf[(i + 1) & 1];
+      IT_TRY(stage_ctx(g, Bn, ws, w.layer_bytes, st, &cb));
+      IT_TRY(stage_gather(cb, Z, nullptr, nullptr, false, dst2, S));
+      cur = dst2;
+      ++i;
+      continue;
+    }
+    IT_TRY(layer_forward_impl(g, &layers[i], cur, dst, ws, w.layer_bytes, st));
     cur = dst;
   }
   return IT_OK;

@@ -737,6 +737,286 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant
   }
 }
 
+// ----------------------------------------------------------------------------- two products back to back (bf16)
+// The update of one layer followed by the transform of the next, for a layer whose output feeds only that transform:
+//   H[M, N1]  = act1([X1 | X2] * B1 + bias1), rounded to bf16 exactly as it would be stored,
+//   C[M, N2]  = H * B2,  columns [0, n0) + bias0 -> out0, columns [n0, n0 + n1) -> out1.
+// H never leaves the SM: the epilogue warps drain the first accumulator into shared memory in the 128-byte-swizzled
+// K-major layout a TMA copy would have produced, and the second product reads it from there.  Same roles as the
+// single product: warp 0 copies operand tiles, warp 1 issues the MMAs, two groups of eight epilogue warps take
+// alternate tiles.  The MMA issuer runs one tile ahead with the first product (the second product of tile i is
+// issued after the first product of tile i + 1), so the tensor core and the copies do not wait for an epilogue.
+// A group's shared-memory tile holds H and then, once the second product has read it, the staged output.
+struct Tc2Params {
+  int64_t M;
+  int n_tiles;
+  int kb1, kb2;          // k-blocks of the first product that come from X1 / X2
+  int N1;                // columns of H (a multiple of 64): N1 / 64 k-blocks of the second product
+  int N2;                // columns of the second product (n0 + n1)
+  int n0, n1;            // multiples of 64 (whole 128-byte panels of bf16)
+  const float *bias1; int act1;
+  const float *bias0;
+  int stages;
+  int buf_panels;        // 16 KB panels of one group's tile: max(N1, N2) / 64
+  int *status;
+  uint32_t spin_limit;
+  int no_loads;          // test hook: the producer issues no copies, so every wait runs out
+};
+
+constexpr int TC2_GROUP_WARPS = TC_EPI_WARPS / 2;
+
+// One epilogue group drains `ncols` accumulator columns of its TMEM lane quarter into the panels of its tile:
+// column c of row r lands at byte 2 c of the row, panel (2 c) / 128, 16-byte chunk ((2 c) % 128) / 16 xor (r % 8).
+// `cst` holds one fp32 constant per column (added), `act_cols` columns from the left get the activation.
+__device__ __forceinline__ void tc2_drain(uint32_t taddr, int ncols, int gsub, const float *cst, int act, int act_cols,
+                                          uint32_t out_row, uint32_t swz, uint64_t *release_bar, int lane) {
+  const int n_groups = ncols >> 4;
+  int last = -1;
+  for (int gidx = n_groups - 1; gidx >= 0; --gidx)
+    if ((gidx & 1) == gsub) { last = gidx; break; }
+  bool released = false;
+  for (int gidx = gsub; gidx < n_groups; gidx += 2) {
+    const int c = gidx << 4;
+    uint32_t r[16];
+    tmem_ld16(taddr + (uint32_t)c, r);
+    tmem_ld_wait();
+    if (gidx == last) {   // everything this warp needs is in registers: hand the accumulator back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(release_bar);
+      released = true;
+    }
+    float v[16];
+    const float4 *c4 = reinterpret_cast<const float4 *>(cst + c);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 b4 = c4[i];
+      v[4 * i] = __uint_as_float(r[4 * i]) + b4.x; v[4 * i + 1] = __uint_as_float(r[4 * i + 1]) + b4.y;
+      v[4 * i + 2] = __uint_as_float(r[4 * i + 2]) + b4.z; v[4 * i + 3] = __uint_as_float(r[4 * i + 3]) + b4.w;
+    }
+    if (c < act_cols) {
+      if (act == IT_ACT_RELU) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+      } else if (act == IT_ACT_ELU) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = it_elu(v[i]);
+      }
+    }
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t *>(&h2);
+    }
+    const uint32_t boff = (uint32_t)c * 2u;
+    const uint32_t pbase = out_row + (boff >> 7) * (uint32_t)(TC_BM * TC_KBLOCK_BYTES);
+    const uint32_t ch = (boff & 127u) >> 4;
+    st_shared_v4(pbase + (((ch + 0) ^ swz) << 4), w[0], w[1], w[2], w[3]);
+    st_shared_v4(pbase + (((ch + 1) ^ swz) << 4), w[4], w[5], w[6], w[7]);
+  }
+  if (!released) {   // a warp that owns no columns still has to sign off
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(release_bar);
+  }
+}
+
+__global__ void __launch_bounds__(TC_THREADS_BF16, 1)
+gemm2_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant__ CUtensorMap map_x2,
+                const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
+                const __grid_constant__ CUtensorMap map_o0, const __grid_constant__ CUtensorMap map_o1, const Tc2Params p) {
+  extern __shared__ unsigned char smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KB1 = p.kb1 + p.kb2;
+  const int KB2 = p.N1 >> 6;
+  constexpr int a_tile_bytes = TC_BM * TC_KBLOCK_BYTES;          // 16 KB
+  const int b1_tile_bytes = p.N1 * TC_KBLOCK_BYTES, b2_tile_bytes = p.N2 * TC_KBLOCK_BYTES;
+  const int b1_bytes = KB1 * b1_tile_bytes, b2_bytes = KB2 * b2_tile_bytes;
+
+  // shared memory: weights of both products | operand stages | one tile per epilogue group | barriers | constants
+  unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char *smem_b1 = base;
+  unsigned char *smem_b2 = smem_b1 + b1_bytes;
+  unsigned char *smem_a = smem_b2 + b2_bytes;
+  unsigned char *smem_buf = smem_a + (size_t)p.stages * a_tile_bytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem_buf + (size_t)2 * p.buf_panels * a_tile_bytes);
+  uint64_t *full = bars;                    // [stages]  TMA landed
+  uint64_t *empty = bars + p.stages;        // [stages]  the MMAs that read the stage are done
+  uint64_t *b_full = bars + 2 * p.stages;   // [1]
+  uint64_t *acc1_full = b_full + 1;         // [2]  first product of a tile complete
+  uint64_t *acc1_empty = acc1_full + 2;     // [2]  its accumulator drained
+  uint64_t *h_full = acc1_empty + 2;        // [2]  H tile of the group written to shared memory
+  uint64_t *acc2_full = h_full + 2;         // [2]  second product complete (and H read)
+  uint64_t *acc2_empty = acc2_full + 2;     // [2]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc2_empty + 2);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  float *cst1 = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~(uintptr_t)15);   // [N1] bias of H
+  float *cst2 = cst1 + p.N1;                                                                                     // [N2] bias0 | 0
+
+  uint32_t tmem_cols = 32;
+  while (tmem_cols < (uint32_t)(2 * (p.N1 + p.N2))) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(b_full, 1);
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc1_full[a], 1);
+      mbar_init(&acc1_empty[a], TC2_GROUP_WARPS);
+      mbar_init(&h_full[a], TC2_GROUP_WARPS);
+      mbar_init(&acc2_full[a], 1);
+      mbar_init(&acc2_empty[a], TC2_GROUP_WARPS);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, tmem_cols);
+    tmem_relinquish();
+  }
+  for (int c = threadIdx.x; c < p.N1; c += blockDim.x) cst1[c] = p.bias1 ? p.bias1[c] : 0.f;
+  for (int c = threadIdx.x; c < p.N2; c += blockDim.x) cst2[c] = (p.bias0 && c < p.n0) ? p.bias0[c] : 0.f;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t acc2_col0 = 2u * (uint32_t)p.N1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && !p.no_loads) {
+      mbar_arrive_expect_tx(b_full, (uint32_t)(b1_bytes + b2_bytes));
+      for (int kb = 0; kb < KB1; ++kb) tma_load_2d(smem_b1 + (size_t)kb * b1_tile_bytes, &map_b1, kb * 64, 0, b_full);
+      for (int kb = 0; kb < KB2; ++kb) tma_load_2d(smem_b2 + (size_t)kb * b2_tile_bytes, &map_b2, kb * 64, 0, b_full);
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+        const int m0 = tile * TC_BM;
+        for (int kb = 0; kb < KB1; ++kb) {
+          ok = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.spin_limit, IT_TC_TMA_BACKOFF);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full[stage], (uint32_t)a_tile_bytes);
+          if (kb < p.kb1) tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x1, kb * 64, m0, &full[stage]);
+          else tma_load_2d(smem_a + (size_t)stage * a_tile_bytes, &map_x2, (kb - p.kb1) * 64, m0, &full[stage]);
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // aborting: give the copies that were issued time to land before the CTA may exit (bounded)
+        for (int s = 0; s < p.stages; ++s)
+          for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it)
+            if (mbar_try_wait(&full[s], 0) || mbar_try_wait(&full[s], 1)) break;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N1 >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N2 >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      bool ok = mbar_wait(b_full, 0, abort_flag, p.spin_limit);
+      uint32_t stage = 0, phase = 0;
+      // second product of this CTA's tile number j (accumulator and group j % 2, used for the (j / 2)-th time)
+      auto second = [&](int j) -> bool {
+        const uint32_t a = (uint32_t)j & 1u, ph = ((uint32_t)j >> 1) & 1u;
+        if (!mbar_wait(&acc2_empty[a], ph ^ 1u, abort_flag, p.spin_limit)) return false;
+        if (!mbar_wait(&h_full[a], ph, abort_flag, p.spin_limit)) return false;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc2_col0 + a * (uint32_t)p.N2;
+        const uint32_t h_s = smem_u32(smem_buf + (size_t)a * p.buf_panels * a_tile_bytes);
+        for (int kb = 0; kb < KB2; ++kb) {
+          const uint32_t a_s = h_s + (uint32_t)kb * (uint32_t)a_tile_bytes;
+          const uint32_t b_s = smem_u32(smem_b2 + (size_t)kb * b2_tile_bytes);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            tc_mma<false>(d_tmem, make_desc(a_s + k * 32), make_desc(b_s + k * 32), idesc2, (kb | k) != 0);
+        }
+        tc_commit(&acc2_full[a]);   // complete: the accumulator may be drained and the H tile overwritten
+        return true;
+      };
+      int it = 0;
+      for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
+        const uint32_t a = (uint32_t)it & 1u, ph = ((uint32_t)it >> 1) & 1u;
+        ok = mbar_wait(&acc1_empty[a], ph ^ 1u, abort_flag, p.spin_limit);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * (uint32_t)p.N1;
+        for (int kb = 0; kb < KB1; ++kb) {
+          ok = mbar_wait(&full[stage], phase, abort_flag, p.spin_limit);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_s = smem_u32(smem_a + (size_t)stage * a_tile_bytes);
+          const uint32_t b_s = smem_u32(smem_b1 + (size_t)kb * b1_tile_bytes);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            tc_mma<false>(d_tmem, make_desc(a_s + k * 32), make_desc(b_s + k * 32), idesc1, (kb | k) != 0);
+          tc_commit(&empty[stage]);
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(&acc1_full[a]);
+        if (it > 0) ok = second(it - 1);
+      }
+      if (ok && it > 0) second(it - 1);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue: group g takes the tiles it % 2 == g
+    const int quarter = warp & 3;   // a warp may only touch TMEM lanes [32 * (warp % 4), +32)
+    const int group = (warp - 2) / TC2_GROUP_WARPS;
+    const int gsub = ((warp - 2) % TC2_GROUP_WARPS) >> 2;   // which of the two warps of this quarter in the group
+    const int row_in_tile = quarter * 32 + lane;
+    unsigned char *my_buf = smem_buf + (size_t)group * p.buf_panels * a_tile_bytes;
+    const uint32_t out_row = smem_u32(my_buf) + (uint32_t)row_in_tile * 128u;
+    const uint32_t swz = (uint32_t)(row_in_tile & 7);
+    const bool issuer = (warp - 2) % TC2_GROUP_WARPS == 0 && lane == 0;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const int pan0 = p.n0 >> 6, pan1 = p.n1 >> 6;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++it) {
+      if ((it & 1) != group) continue;
+      const uint32_t ph = ((uint32_t)it >> 1) & 1u;
+      const int m0 = tile * TC_BM;
+      // ---- first accumulator -> H tile (bias, activation, bf16, swizzled)
+      bool ok = mbar_wait(&acc1_full[group], ph, abort_flag, p.spin_limit, IT_TC_EPI_BACKOFF);
+      if (issuer) tma_store_wait_read();   // the stores of this group's previous tile have read the tile
+      __syncwarp();
+      if (epi_bar_any(2, group, !ok)) break;   // one decision for all warps of the group
+      tc_fence_after();
+      tc2_drain(tmem_base + lane_base + (uint32_t)group * (uint32_t)p.N1, p.N1, gsub, cst1, p.act1, p.N1, out_row, swz,
+                &acc1_empty[group], lane);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the tensor core's reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&h_full[group]);
+      // ---- second accumulator -> staged output (the H tile has been read), then TMA stores
+      ok = mbar_wait(&acc2_full[group], ph, abort_flag, p.spin_limit, IT_TC_EPI_BACKOFF);
+      __syncwarp();
+      if (epi_bar_any(2, group, !ok)) break;
+      tc_fence_after();
+      tc2_drain(tmem_base + lane_base + acc2_col0 + (uint32_t)group * (uint32_t)p.N2, p.N2, gsub, cst2, IT_ACT_NONE, 0, out_row,
+                swz, &acc2_empty[group], lane);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA store's reads
+      epi_bar_sync(2, group);
+      if (issuer) {
+        for (int k = 0; k < pan0; ++k) tma_store_2d(&map_o0, my_buf + (size_t)k * a_tile_bytes, k * 64, m0);
+        for (int k = 0; k < pan1; ++k) tma_store_2d(&map_o1, my_buf + (size_t)(pan0 + k) * a_tile_bytes, k * 64, m0);
+        tma_store_commit();
+      }
+    }
+    if (issuer) tma_store_wait_all();   // the tile must outlive the last stores
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, 1);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
 // ----------------------------------------------------------------------------- weight prep (K-major, split)
 struct PrepTcParams {
   int kind, in_dim, out_dim, w_is_bf16, NB;
@@ -943,6 +1223,72 @@ it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *a
   return IT_OK;
 }
 
+// ----------------------------------------------------------------------------- two products back to back: host side
+namespace {
+struct Tc2Shape { int kb1, kb2, buf_panels, stages, smem; };
+
+bool tc2_shape(const it_gemm2_args &a, Tc2Shape *out) {
+  if (a.M <= 0 || a.M > (int64_t)INT32_MAX) return false;
+  const int K2 = a.X2 ? a.K2 : 0;
+  if (a.K1 <= 0 || (a.K1 * 2) % 16 != 0 || (K2 * 2) % 16 != 0) return false;
+  const int N2 = a.n0 + a.n1;
+  if (a.N1 <= 0 || a.N1 % 64 != 0 || a.N1 > 256) return false;           // H is a whole number of k-blocks of the second product
+  if (a.n0 % 64 != 0 || a.n1 % 64 != 0 || N2 <= 0 || N2 > 256) return false;   // outputs are whole 128-byte panels
+  if (2 * (a.N1 + N2) > 512) return false;                               // two accumulators per product in TMEM
+  Tc2Shape s;
+  s.kb1 = (a.K1 + 63) / 64; s.kb2 = (K2 + 63) / 64;
+  s.buf_panels = (a.N1 > N2 ? a.N1 : N2) / 64;
+  const int stage_bytes = TC_BM * TC_KBLOCK_BYTES;
+  const int fixed = (s.kb1 + s.kb2) * a.N1 * TC_KBLOCK_BYTES + (a.N1 / 64) * N2 * TC_KBLOCK_BYTES + 2 * s.buf_panels * stage_bytes +
+                    kSmemAux + (a.N1 + N2) * 4;
+  s.stages = (kSmemBudget - fixed) / stage_bytes;
+  if (s.stages < 3) return false;
+  if (s.stages > IT_TC_MAX_STAGES) s.stages = IT_TC_MAX_STAGES;
+  s.smem = fixed + s.stages * stage_bytes;
+  *out = s;
+  return true;
+}
+}  // namespace
+
+bool it_tc2_supported(const it_gemm2_args &a) {
+  Tc2Shape s;
+  return tc2_shape(a, &s);
+}
+
+// B1, B2: bf16 weights prepared by it_launch_prep_weights_tc ([N1, padded K1 + padded K2] and [n0 + n1, N1]).
+it_status it_launch_gemm2_tc(const it_gemm2_args &a, const void *B1, const void *B2, int num_sms, int *status, cudaStream_t st) {
+  if (a.M == 0) return IT_OK;
+  Tc2Shape s;
+  IT_REQUIRE(tc2_shape(a, &s), IT_ERR_UNSUPPORTED, "fused tensor-core apply: shape not supported");
+  const int K2 = a.X2 ? a.K2 : 0, N2 = a.n0 + a.n1;
+  CUtensorMap m1, m2, mb1, mb2;
+  IT_TRY(make_map(&m1, a.X1, 2, a.M, a.K1, TC_BM));
+  if (a.X2) IT_TRY(make_map(&m2, a.X2, 2, a.M, K2, TC_BM));
+  else m2 = m1;
+  IT_TRY(make_map(&mb1, B1, 2, a.N1, (int64_t)(s.kb1 + s.kb2) * 64, a.N1));
+  IT_TRY(make_map(&mb2, B2, 2, N2, a.N1, N2));
+  CUtensorMap mo0 = m1, mo1 = m1;   // placeholders where a segment is empty
+  if (a.n0 > 0) IT_TRY(make_map(&mo0, a.out0, 2, a.M, a.n0, TC_BM));
+  if (a.n1 > 0) IT_TRY(make_map(&mo1, a.out1, 2, a.M, a.n1, TC_BM));
+
+  Tc2Params p;
+  p.M = a.M; p.n_tiles = (int)((a.M + TC_BM - 1) / TC_BM);
+  p.kb1 = s.kb1; p.kb2 = s.kb2; p.N1 = a.N1; p.N2 = N2; p.n0 = a.n0; p.n1 = a.n1;
+  p.bias1 = a.bias1; p.act1 = a.act1; p.bias0 = a.bias0;
+  p.stages = s.stages; p.buf_panels = s.buf_panels; p.status = status;
+  p.spin_limit = a.spin_limit ? a.spin_limit : TC_SPIN_LIMIT; p.no_loads = a.no_loads;
+
+  int64_t grid = num_sms;
+  if (grid > p.n_tiles) grid = p.n_tiles;
+  const int K = a.K1 + K2;
+  const double bytes = (double)a.M * 2.0 * (K + N2) + 2.0 * ((double)K * a.N1 + (double)a.N1 * N2);
+  const double flops = 2.0 * (double)a.M * ((double)K * a.N1 + (double)a.N1 * N2);
+  IT_CUDA_TRY(cudaFuncSetAttribute(gemm2_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, s.smem));
+  IT_LAUNCH(IT_K_GEMM2_TC, bytes, flops, st, gemm2_tc_kernel<<<(unsigned)grid, TC_THREADS_BF16, s.smem, st>>>(m1, m2, mb1, mb2, mo0, mo1, p));
+  IT_CUDA_TRY(cudaGetLastError());
+  return IT_OK;
+}
+
 // Test hook for the bounded waits: a 128 x 64 product (bf16, or fp32 with its operand-splitting warps) whose producer issues no copies, with waits that give up
 // after a few thousand polls.  Every role runs out of patience, the CTA drains, frees its TMEM and returns, and the
 // status word of the graph is set, which the next it_graph_check reports as IT_ERR_TIMEOUT.
@@ -957,4 +1303,16 @@ extern "C" it_status it_debug_expire_wait(it_graph *g, it_dtype dtype, const voi
   a.n1 = 0; a.out1 = nullptr; a.dt1 = dtype; a.out2 = nullptr;
   a.spin_limit = 4096; a.no_loads = 1;
   return it_launch_gemm_tc(a, workspace, nullptr, nullptr, 1, 64, nullptr, g->num_sms, g->d_status, (cudaStream_t)stream);
+}
+
+// The same hook for the kernel that runs two products back to back (bf16: 128 x 64 times 64 x 64 times 64 x 64).
+extern "C" it_status it_debug_expire_wait_fused(it_graph *g, const void *x, void *out, void *workspace, size_t workspace_bytes,
+                                                 void *stream) {
+  IT_REQUIRE(g != nullptr && x != nullptr && out != nullptr && workspace != nullptr, IT_ERR_INVALID_ARG, "NULL argument");
+  IT_REQUIRE(workspace_bytes >= 64 * 1024 && ((uintptr_t)workspace % 256) == 0, IT_ERR_WORKSPACE, "needs 64 KB of aligned workspace");
+  it_gemm2_args a{};
+  a.M = 128; a.X1 = x; a.K1 = 64; a.X2 = nullptr; a.K2 = 0; a.N1 = 64; a.bias1 = nullptr; a.act1 = IT_ACT_NONE;
+  a.n0 = 0; a.out0 = nullptr; a.bias0 = nullptr; a.n1 = 64; a.out1 = out;
+  a.spin_limit = 4096; a.no_loads = 1;
+  return it_launch_gemm2_tc(a, workspace, (const char *)workspace + 32 * 1024, g->num_sms, g->d_status, (cudaStream_t)stream);
 }

@@ -42,7 +42,7 @@ void it_set_error(const char *fmt, ...);
 enum it_kernel_id {
   IT_K_VALIDATE = 0, IT_K_SPLIT_SCAN, IT_K_SPLIT_FILL, IT_K_BUCKET_SCAN, IT_K_PREP, IT_K_GATHER_CTA, IT_K_GATHER_FLAT,
   IT_K_GATHER_EMPTY, IT_K_COMBINE, IT_K_GEMM_FP32, IT_K_GEMM_TC, IT_K_GAT_CTA, IT_K_GAT_FLAT, IT_K_GAT_EMPTY,
-  IT_K_EDGE_MSG, IT_K_AGG_FINISH,
+  IT_K_EDGE_MSG, IT_K_AGG_FINISH, IT_K_GEMM2_TC,
   IT_K_COUNT
 };
 // Wraps one kernel launch: counts it and, while profiling is on, brackets it with events on `st`.
@@ -164,7 +164,8 @@ struct it_gat_args {
   const float *scores;    // [n_src, 2*heads]: source scores of the vertex, then its destination scores
   const float *scores_dst;   // the same layout, row v = local destination v (scores + first_vertex * 2*heads for a part; NULL: scores)
   int per_edge_rows;      // 1: z is [n_edges, dim] and src_scores [n_edges, heads], row j belonging to edge j (edge features in the logits)
-  const float *src_scores;   // per_edge_rows only: the logit term of every edge (source score + edge share)
+  const float *src_scores;   // [rows, heads], dense: the source-side logit term that is read per edge (row = source vertex, or the
+                             // edge itself with per_edge_rows); NULL: the first half of the rows of `scores`
   float *partials;        // it_gat_partial_bytes() of fp32 scratch for the groups of split vertices (may be NULL if none)
   int *counters;          // IT_MAX_BUCKETS device words of scratch from which warps claim their batches (NULL: fixed strides)
   float slope;
@@ -213,6 +214,22 @@ it_status it_launch_prep_weights_tc(it_prep_kind kind, const it_layer_desc *laye
 it_status it_launch_gemm_tc(const it_gemm_args &a, const void *B, const float *att_src, const float *att_dst,
                             int heads, int head_dim, float *scores, int num_sms, int *status, cudaStream_t stream);
 
+// The update of one layer and the transform of the next as one kernel (bf16 only): H = act1([X1 | X2] B1 + bias1) is
+// rounded to bf16 and multiplied by B2 without leaving the SM; columns [0, n0) of H B2, plus bias0, go to out0 and
+// columns [n0, n0 + n1) to out1.  N1 (columns of H), n0 and n1 must be multiples of 64.
+struct it_gemm2_args {
+  int64_t M;
+  const void *X1; int K1;
+  const void *X2; int K2;
+  int N1; const float *bias1; it_act act1;
+  int n0; void *out0; const float *bias0;
+  int n1; void *out1;
+  uint32_t spin_limit;   // polls after which a barrier wait gives up (0 = the default)
+  int no_loads;          // test hook: issue no operand copies
+};
+bool it_tc2_supported(const it_gemm2_args &a);
+it_status it_launch_gemm2_tc(const it_gemm2_args &a, const void *B1, const void *B2, int num_sms, int *status, cudaStream_t stream);
+
 // ----------------------------------------------------------------------------- message.cu
 // Learned messages, edge by edge: M[j, :] = act(P[indices[j], :] + M[j, :]) in place (M arrives holding the per-edge
 // part Q), rows of `dim` elements of `dtype` (a multiple of 16 bytes).
@@ -220,5 +237,8 @@ it_status it_launch_edge_messages(const it_graph *g, it_dtype dtype, int dim, co
 // GAT with edge features: Zj[j, :] = Z[indices[j], :] and sc[j, h] = scores[indices[j], h] + att_edge[h, :] . ef[j, :].
 it_status it_launch_gat_edge_rows(const it_graph *g, it_dtype dtype, int dim, int heads, const void *Z, const float *scores,
                                   const float *att_edge, void *Zj, float *sc, cudaStream_t stream);
+// dense[v, :] = scores[v, 0:heads]: the source scores on their own, 16 bytes per vertex for 4 heads instead of a 32-byte
+// row shared with the destination scores (the reduce reads one per edge, at random).
+it_status it_launch_compact_scores(int64_t n, int heads, const float *scores, float *dense, cudaStream_t stream);
 // out[v, :] = raw[v, :] * scale[v] (0 where scale[v] = 0), fp32 -> dtype.
 it_status it_launch_aggregate_finish(int64_t n, int dim, it_dtype dtype, const float *raw, const float *scale, void *out, cudaStream_t stream);

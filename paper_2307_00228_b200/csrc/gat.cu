@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(THREADS) gat_combine_kernel(GatCombineParams p
 template <typename T, int SB, int LPR>
 it_status launch_gat_lpr(const it_gat_args &a, StreamParams sp, int64_t bound_lo, int64_t bound_hi, cudaStream_t st) {
   GatPolicy<T, SB> pol;
-  pol.scores = a.per_edge_rows ? a.src_scores : a.scores; pol.src_stride = a.per_edge_rows ? a.heads : 2 * a.heads;
+  pol.scores = a.src_scores ? a.src_scores : a.scores; pol.src_stride = a.src_scores ? a.heads : 2 * a.heads;
   pol.scores_dst = a.scores_dst ? a.scores_dst : a.scores; pol.bias = a.bias; pol.dst = a.dst; pol.partials = a.partials;
   pol.dim = a.heads * a.head_dim; pol.heads = a.heads; pol.head_dim = a.head_dim; pol.act = a.act; pol.slope = a.slope;
   pol.col = 0; pol.head = 0; pol.s_dst = 0.f;

@@ -108,6 +108,15 @@ __global__ void __launch_bounds__(MSG_THREADS) gat_edge_scores_kernel(const int3
   }
 }
 
+__global__ void __launch_bounds__(MSG_THREADS) compact_scores_kernel(const float *__restrict__ scores, float *__restrict__ dense,
+                                                                     int64_t total, int heads) {
+  const int64_t stride = (int64_t)gridDim.x * MSG_THREADS;
+  for (int64_t t = (int64_t)blockIdx.x * MSG_THREADS + threadIdx.x; t < total; t += stride) {
+    const int64_t v = t / heads;
+    dense[t] = __ldcs(scores + v * 2 * heads + (t - v * heads));
+  }
+}
+
 // one thread per four consecutive entries of a row
 template <typename T>
 __global__ void __launch_bounds__(MSG_THREADS) aggregate_finish_kernel(const float4 *__restrict__ raw, const float *__restrict__ scale,
@@ -171,6 +180,16 @@ it_status it_launch_gat_edge_rows(const it_graph *g, it_dtype dtype, int dim, in
   else
     IT_LAUNCH(IT_K_EDGE_MSG, sbytes, 0, st, gat_edge_scores_kernel<__nv_bfloat16><<<blocks, MSG_THREADS, 0, st>>>(
         g->indices, scores, reinterpret_cast<const __nv_bfloat16 *>(g->edge_feat), att_edge, sc, g->e, heads, g->edge_dim));
+  IT_CUDA_TRY(cudaGetLastError());
+  return IT_OK;
+}
+
+it_status it_launch_compact_scores(int64_t n, int heads, const float *scores, float *dense, cudaStream_t st) {
+  if (n == 0) return IT_OK;
+  const int64_t total = n * heads;
+  const int64_t want = (total + MSG_THREADS - 1) / MSG_THREADS, cap = (int64_t)IT_NUM_SMS_FALLBACK * 32;
+  IT_LAUNCH(IT_K_EDGE_MSG, (double)n * heads * 12.0, 0, st,
+            compact_scores_kernel<<<(unsigned)(want < cap ? want : cap), MSG_THREADS, 0, st>>>(scores, dense, total, heads));
   IT_CUDA_TRY(cudaGetLastError());
   return IT_OK;
 }

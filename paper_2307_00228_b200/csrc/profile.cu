@@ -16,7 +16,8 @@ std::vector<Slot> g_pool;        // recycled event pairs
 int64_t g_launches = 0;
 const char *const kNames[IT_K_COUNT] = {"validate", "split_scan", "split_fill", "bucket_scan", "prep_weights",
                                         "gather_cta", "gather_flat", "gather_empty", "combine", "gemm_fp32",
-                                        "gemm_tc", "gat_cta", "gat_flat", "gat_empty", "edge_messages", "aggregate_finish"};
+                                        "gemm_tc", "gat_cta", "gat_flat", "gat_empty", "edge_messages", "aggregate_finish",
+                                        "gemm2_tc"};
 }  // namespace
 
 it_prof_scope::it_prof_scope(int kid, double bytes, double flops, cudaStream_t st) : slot_(-1), st_(st) {

@@ -97,7 +97,9 @@ class CudaEngine:
         return torch.empty(max(256, self.B.it_workspace_bytes(part, layers)), dtype=torch.uint8, device=self.device)
 
     def empty(self, rows, cols, dtype):
-        return torch.zeros((rows, cols), dtype=dtype, device=self.device)
+        # not cleared: every row that is later read is written first (the padding rows of a block are exchanged but no
+        # source id names them)
+        return torch.empty((rows, cols), dtype=dtype, device=self.device)
 
     def transform(self, part, layer, h_self, table_out, scores_out, ws):
         self.B.it_layer_transform(part, layer, h_self, table_out, scores_out, ws)

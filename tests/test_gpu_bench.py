@@ -37,3 +37,17 @@ def test_partitioned_arm_on_one_rank(layout):
     assert d["scaling"] == "strong" and d["n_gpus"] == 1 and d["value"] > 0 and d["rejected"] is False
     assert "vertex ranges" in d["config"]["parallelism"] and d["result_check"]["finite"]
     assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["gpu_launches"] > 0
+
+
+def test_tiny_latency_record_and_cuda_graph_replay():
+    """The Tiny workload as the benchmark reports it: latency of one it_infer, call by call and replayed from a CUDA
+    graph captured around the same call (the library allocates nothing and synchronises nothing inside it_infer)."""
+    import sys
+    sys.path.insert(0, ROOT)
+    import torch
+    import bench
+    rec = bench.measure_tiny(None, torch.device("cuda"))
+    assert rec["parity"]["ok"] and rec["problems"] == []
+    assert rec["us_per_infer"] > 0 and rec["launches_per_infer"] > 0
+    assert rec.get("cuda_graph_error") is None, rec.get("cuda_graph_error")
+    assert rec["cuda_graph_result_identical"] and rec["us_per_infer_cuda_graph"] > 0

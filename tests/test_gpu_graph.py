@@ -125,7 +125,7 @@ def test_invalid_arguments():
     assert B.lib().it_graph_destroy(None) == 0
 
 
-@pytest.mark.parametrize("tdtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("tdtype", [torch.bfloat16, torch.float32, "fused"])
 def test_a_wait_that_runs_out_is_reported_and_the_library_goes_on(tdtype):
     """The tensor-core apply waits on hardware barriers with a poll limit.  With its copy producer switched off
     every wait runs out: the kernel must return by itself, it_graph_check must say IT_ERR_TIMEOUT once, and a
@@ -135,10 +135,15 @@ def test_a_wait_that_runs_out_is_reported_and_the_library_goes_on(tdtype):
     w = small_workload(2, 600, 12, "bf16", [layer])
     got, d = run_device(w)
     check_against_oracle(w, got)
+    fused = tdtype == "fused"   # the kernel that runs two products back to back
+    tdtype = torch.bfloat16 if fused else tdtype
     x = torch.zeros((128, 64), dtype=tdtype, device="cuda")
     o = torch.empty((128, 64), dtype=tdtype, device="cuda")
     ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
-    B.it_debug_expire_wait(d.graph, x, o, ws)
+    if fused:
+        B.it_debug_expire_wait_fused(d.graph, x, o, ws)
+    else:
+        B.it_debug_expire_wait(d.graph, x, o, ws)
     with pytest.raises(B.ItError) as e:
         B.it_graph_check(d.graph)
     assert e.value.status_name == "IT_ERR_TIMEOUT"
