@@ -764,28 +764,18 @@ struct Tc2Params {
 };
 
 constexpr int TC2_GROUP_WARPS = TC_EPI_WARPS / 2;
+#ifndef IT_TC2_BACKOFF
+#define IT_TC2_BACKOFF 32   // ns between polls of the second accumulator's barrier
+#endif
 
 // One epilogue group drains `ncols` accumulator columns of its TMEM lane quarter into the panels of its tile:
 // column c of row r lands at byte 2 c of the row, panel (2 c) / 128, 16-byte chunk ((2 c) % 128) / 16 xor (r % 8).
 // `cst` holds one fp32 constant per column (added), `act_cols` columns from the left get the activation.
 __device__ __forceinline__ void tc2_drain(uint32_t taddr, int ncols, int gsub, const float *cst, int act, int act_cols,
                                           uint32_t out_row, uint32_t swz, uint64_t *release_bar, int lane) {
-  const int n_groups = ncols >> 4;
-  int last = -1;
-  for (int gidx = n_groups - 1; gidx >= 0; --gidx)
-    if ((gidx & 1) == gsub) { last = gidx; break; }
-  bool released = false;
-  for (int gidx = gsub; gidx < n_groups; gidx += 2) {
-    const int c = gidx << 4;
-    uint32_t r[16];
-    tmem_ld16(taddr + (uint32_t)c, r);
-    tmem_ld_wait();
-    if (gidx == last) {   // everything this warp needs is in registers: hand the accumulator back
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(release_bar);
-      released = true;
-    }
+  const int n_groups = ncols >> 4;   // 16-column groups; this warp takes those with index % 2 == gsub, two per TMEM wait
+  // bias, activation, bf16, swizzled store of one 16-column group held in r
+  auto finish = [&](int c, const uint32_t (&r)[16]) {
     float v[16];
     const float4 *c4 = reinterpret_cast<const float4 *>(cst + c);
 #pragma unroll
@@ -814,6 +804,22 @@ __device__ __forceinline__ void tc2_drain(uint32_t taddr, int ncols, int gsub, c
     const uint32_t ch = (boff & 127u) >> 4;
     st_shared_v4(pbase + (((ch + 0) ^ swz) << 4), w[0], w[1], w[2], w[3]);
     st_shared_v4(pbase + (((ch + 1) ^ swz) << 4), w[4], w[5], w[6], w[7]);
+  };
+  bool released = false;
+  for (int gidx = gsub; gidx < n_groups; gidx += 4) {
+    const bool two = gidx + 2 < n_groups;
+    uint32_t r0[16], r1[16];
+    tmem_ld16(taddr + (uint32_t)(gidx << 4), r0);
+    if (two) tmem_ld16(taddr + (uint32_t)((gidx + 2) << 4), r1);
+    tmem_ld_wait();
+    if (gidx + 4 >= n_groups) {   // everything this warp needs is in registers: hand the accumulator back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(release_bar);
+      released = true;
+    }
+    finish(gidx << 4, r0);
+    if (two) finish((gidx + 2) << 4, r1);
   }
   if (!released) {   // a warp that owns no columns still has to sign off
     tc_fence_before();
@@ -990,14 +996,17 @@ gemm2_tc_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constan
       __syncwarp();
       if (lane == 0) mbar_arrive(&h_full[group]);
       // ---- second accumulator -> staged output (the H tile has been read), then TMA stores
-      ok = mbar_wait(&acc2_full[group], ph, abort_flag, p.spin_limit, IT_TC_EPI_BACKOFF);
-      __syncwarp();
+      // (a short wait: the second product follows the H tile at once; a warp whose wait ran out skips the drain and the
+      // group decides together at the barrier below, which the stores need anyway)
+      ok = mbar_wait(&acc2_full[group], ph, abort_flag, p.spin_limit, IT_TC2_BACKOFF);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after();
+        tc2_drain(tmem_base + lane_base + acc2_col0 + (uint32_t)group * (uint32_t)p.N2, p.N2, gsub, cst2, IT_ACT_NONE, 0, out_row,
+                  swz, &acc2_empty[group], lane);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA store's reads
+      }
       if (epi_bar_any(2, group, !ok)) break;
-      tc_fence_after();
-      tc2_drain(tmem_base + lane_base + acc2_col0 + (uint32_t)group * (uint32_t)p.N2, p.N2, gsub, cst2, IT_ACT_NONE, 0, out_row,
-                swz, &acc2_empty[group], lane);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA store's reads
-      epi_bar_sync(2, group);
       if (issuer) {
         for (int k = 0; k < pan0; ++k) tma_store_2d(&map_o0, my_buf + (size_t)k * a_tile_bytes, k * 64, m0);
         for (int k = 0; k < pan1; ++k) tma_store_2d(&map_o1, my_buf + (size_t)(pan0 + k) * a_tile_bytes, k * 64, m0);

@@ -35,6 +35,14 @@ struct SagePolicy {
   __device__ __forceinline__ float extra(uint32_t) const { return 0.f; }
   __device__ __forceinline__ const float *extra_ptr(uint32_t) const { return nullptr; }
   __device__ __forceinline__ void edge(float (&st)[NS], const typename Slice::Raw &raw, float w, float) const {
+    if constexpr (RED == RED_SUM && !WEIGHTED && sizeof(T) == 2 && IT_MIXED_ADD != 0) {
+      // bf16 rows, plain sum: the mixed-precision add takes the bf16 operand as it is (same result as widening it first)
+      uint32_t w[SB / 4];
+      raw_words<SB>(raw, w);
+#pragma unroll
+      for (int i = 0; i < SB / 4; ++i) add_bf16x2_to_f32(st[2 * i], st[2 * i + 1], w[i]);
+      return;
+    }
     float f[VEC];
     Slice::unpack(raw, f);
     if constexpr (RED == RED_SUM && !WEIGHTED && VEC % 2 == 0) {   // two accumulators per instruction (measured: 1 % on the

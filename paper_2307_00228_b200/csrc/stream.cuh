@@ -158,6 +158,17 @@ __device__ __forceinline__ void add_f32x2(float &a0, float &a1, float b0, float 
   a0 += b0; a1 += b1;
 #endif
 }
+// a0 += low bf16 of w, a1 += high bf16 of w: mixed-precision adds (fp32 accumulator, bf16 addend; the addend is
+// widened exactly, so each result equals the fp32 add of the widened value).
+#ifndef IT_MIXED_ADD
+#define IT_MIXED_ADD 1
+#endif
+__device__ __forceinline__ void add_bf16x2_to_f32(float &a0, float &a1, uint32_t w) {
+  unsigned short lo, hi;
+  asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
+  asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(a0) : "h"(lo));
+  asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(a1) : "h"(hi));
+}
 // a = w * b + a * s (pairwise, scalars w and s): the running-softmax update
 __device__ __forceinline__ void scale_fma_f32x2(float &a0, float &a1, float s, float w, float b0, float b1) {
 #if IT_PACKED_F32
@@ -456,6 +467,9 @@ __global__ void __launch_bounds__(THREADS, IT_SHORT_MIN_BLOCKS) stream_short_row
 #ifndef IT_SHORT_PIPE_BLOCKS
 #define IT_SHORT_PIPE_BLOCKS 4   // resident CTAs per SM the pipelined kernel's register budget is set for (measured: five spill and gain nothing)
 #endif
+#ifndef IT_RING_SINGLE_ROW
+#define IT_RING_SINGLE_ROW 1     // the ring kernel walks a batch of one row as a stream without ends of rows
+#endif
 #ifndef IT_SHORT_PIPE_WAVES
 #define IT_SHORT_PIPE_WAVES 1    // grid = SMs x resident CTAs x this: every CTA is resident from the start and walks its rows
 #endif
@@ -523,12 +537,13 @@ __global__ void __launch_bounds__(THREADS, IT_SHORT_PIPE_BLOCKS) stream_short_ro
       asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
-      for (int k = 0; k < E; ++k)
+      for (int k = 0; k < E; ++k) {
         if (k0 + k < cur.len) {
           uint4 v;
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(my_buf + (uint32_t)k * (THREADS * 16)) : "memory");
           pol.edge(st, v, ww[k], xx[k]);
         }
+      }
       idx_c = idx_n; w_c = w_n;
     }
     if (cur.len > 0) pol.end_row(st, cur.dest, cur.owner, cur.len);
@@ -721,8 +736,10 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
       }
       if constexpr (RING) {   // a whole warp per batch
         constexpr int smem = (THREADS / 32) * ring_bytes_per_warp<SB, Policy::HAS_EXTRA>();
-        static std::atomic<uint64_t> configured{0};   // per template instance: one bit per device ordinal
-        IT_TRY(allow_dynamic_smem(stream_rows_ring_kernel<T, SB, LPR, Policy>, smem, configured));
+        static std::atomic<uint64_t> configured{0}, configured1{0};   // per template instance: one bit per device ordinal
+        const bool single = IT_RING_SINGLE_ROW && br == 1;
+        if (single) IT_TRY(allow_dynamic_smem(stream_rows_ring_kernel<T, SB, LPR, Policy, true>, smem, configured1));
+        else IT_TRY(allow_dynamic_smem(stream_rows_ring_kernel<T, SB, LPR, Policy, false>, smem, configured));
         p.batch_rows = br;
         const int64_t batches = (rows + br - 1) / br;
         // with a counter every CTA is resident from the start and its warps claim batches as they finish (rows of one
@@ -733,7 +750,8 @@ it_status launch_buckets(const it_graph *g, StreamParams p, const Policy &pol, B
         unsigned blocks = (unsigned)(want < ring_max ? want : ring_max);
         const int64_t per_warp = batches / ((int64_t)blocks * (THREADS / 32));
         p.claim = (int)(per_warp / IT_RING_CLAIMS_PER_WARP < 1 ? 1 : (per_warp / IT_RING_CLAIMS_PER_WARP > 4096 ? 4096 : per_warp / IT_RING_CLAIMS_PER_WARP));
-        IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_ring_kernel<T, SB, LPR, Policy><<<blocks, THREADS, smem, st>>>(p, pol));
+        if (single) IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_ring_kernel<T, SB, LPR, Policy, true><<<blocks, THREADS, smem, st>>>(p, pol));
+        else IT_LAUNCH(kid_rows, bytes, 0, st, stream_rows_ring_kernel<T, SB, LPR, Policy, false><<<blocks, THREADS, smem, st>>>(p, pol));
         p.counter = nullptr;
       } else {                                // a group of LPR lanes per batch
         if (br > LPR) br = LPR;

@@ -194,7 +194,10 @@ __device__ __forceinline__ void ring_stream(const RingWarp<T, SB, LPR, Policy> &
 
 // ----------------------------------------------------------------------------- batches of rows per warp
 // Rows handled here have at least one edge: empty rows live in their own bucket.
-template <typename T, int SB, int LPR, class Policy>
+// SINGLE: every batch is one row (p.batch_rows == 1): the stream is the row and its end is the end of the stream, so
+// there is no bookkeeping of row ends and no metadata spread over the lanes (fewer instructions per row, fewer
+// registers).
+template <typename T, int SB, int LPR, class Policy, bool SINGLE>
 __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_kernel(StreamParams p, Policy pol) {
   constexpr int NS = Policy::NS;
   extern __shared__ uint4 ring_raw[];
@@ -222,6 +225,25 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_
   const int64_t CH = p.counter ? p.claim : 1;
   for (int64_t c = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); c * CH < n_batches; c = next_claim(c))
   for (int64_t b = c * CH; b < (c + 1) * CH && b < n_batches; ++b) {
+    if constexpr (SINGLE) {
+      const it_row_meta m = load_meta(p.meta + p.row_lo + b);
+      const int32_t owner = Policy::NEEDS_OWNER ? __ldcs(p.owner + p.row_lo + b) : 0;
+      float st[NS];
+      pol.init(st);
+      pol.begin_row(m.dest, owner);
+      const int64_t a = m.j0;
+      const int total = m.len;
+      auto load_chunk = [&](int base, int32_t &idx, float &w, unsigned &ends) {
+        idx = 0; w = 1.f; ends = 0u;
+        if (base + lane < total) {
+          idx = p.indices ? __ldcs(p.indices + a + base + lane) : (int32_t)(a + base + lane);
+          if (Policy::WEIGHTED) w = __ldcs(p.weights + a + base + lane);
+        }
+      };
+      ring_stream<T, SB, LPR, Policy>(rw, pol, st, total, load_chunk, [] {});
+      rw.fold(pol, st);
+      if (slot == 0) pol.end_row(st, m.dest, owner, m.len);
+    } else {
     // ---- batch metadata: lane i owns row i of the batch
     const int64_t i = p.row_lo + b * BR + lane;
     int64_t my_j0 = 0;
@@ -282,6 +304,7 @@ __global__ void __launch_bounds__(THREADS, IT_RING_MIN_BLOCKS) stream_rows_ring_
       if (cur < BR && __shfl_sync(0xffffffffu, my_len, cur & 31) > 0) pol.begin_row(nd, no);
     };
     ring_stream<T, SB, LPR, Policy>(rw, pol, st, total, load_chunk, finish_row);
+    }
   }
 }
 
