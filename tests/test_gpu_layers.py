@@ -276,3 +276,29 @@ def test_exact_oracle_bounds_both_storage_types():
         outs, mags = run_oracle(w, storage=None, magnitudes=True)
         err = assert_close(got, outs[-1], mags[-1], dtype, "exact", label=dtype)
         print(dtype, err)
+
+
+@pytest.mark.parametrize("dtype,fi", [("bf16", 64), ("bf16", 128), ("f32", 32), ("f32", 64)])
+@pytest.mark.parametrize("max_deg", [3, 8])
+def test_buckets_of_very_short_rows(dtype, fi, max_deg):
+    """Rows of 128 and 256 bytes with at most 8 edges: when the bucket's rows hold at most 4 edges on average the
+    launch keeps two rows per lane group in flight (max_deg 3), otherwise one (max_deg 8).  Every reduce, with and
+    without edge weights, the transform-first epilogue, a hub that is split, and more rows than one sweep of the grid."""
+    for op, weights, fo in (("mean", False, fi), ("sum", True, fi), ("max", False, fi), ("min", True, fi),
+                            ("mean", False, fi // 2), ("sum", True, fi // 2)):
+        layer = make_sage_layer(7, op, "relu", fi, fo, dtype, weights=weights)
+        w = small_workload(8, 4000, max_deg, dtype, [layer], hubs=(300,), weights=weights, threshold=128, p_zero=0.1)
+        got, d = run_device(w)
+        B.it_graph_check(d.graph)
+        check_against_oracle(w, got, label=(dtype, fi, max_deg, op, weights, fo))
+
+
+def test_very_short_rows_beyond_one_sweep_of_the_grid():
+    """More rows of at most 3 edges than the resident lane groups of the whole GPU take in one sweep (148 SMs x 3
+    CTAs x 32 lane groups), so that every lane group walks several rows and the row records loaded ahead run past
+    the end of the bucket."""
+    layer = make_sage_layer(9, "mean", "none", 64, 64, "bf16")
+    w = small_workload(10, 60_000, 3, "bf16", [layer], p_zero=0.05)
+    got, d = run_device(w)
+    B.it_graph_check(d.graph)
+    check_against_oracle(w, got)
