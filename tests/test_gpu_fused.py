@@ -81,3 +81,28 @@ def test_tail_tile_and_single_tile():
         B.it_graph_check(d.graph)
         assert torch.equal(d.out, layer_by_layer(d, w))
         check_against_oracle(w, to_numpy(d.out))
+
+
+def test_fused_pair_replays_from_a_cuda_graph():
+    """it_infer with a fused pair captured in a CUDA graph on a side stream (the library allocates nothing and
+    synchronises nothing inside it_infer): the replay writes the same result bit for bit."""
+    w = small_workload(33, 3000, 16, "bf16", models()["sage_64_128_64"], hubs=(500,), threshold=128)
+    d = host.upload(w)
+    d.infer()
+    torch.cuda.synchronize()
+    eager = d.out.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        d.infer(stream=side)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            d.infer(stream=side)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        d.out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(d.out, eager)
+    B.it_graph_check(d.graph)
