@@ -51,3 +51,16 @@ def test_tiny_latency_record_and_cuda_graph_replay():
     assert rec["us_per_infer"] > 0 and rec["launches_per_infer"] > 0
     assert rec.get("cuda_graph_error") is None, rec.get("cuda_graph_error")
     assert rec["cuda_graph_result_identical"] and rec["us_per_infer_cuda_graph"] > 0
+
+
+def test_headline_workload_at_a_small_size_runs_the_fused_pair_and_the_unsplit_pass():
+    """The bf16 model of the headline workload: its two dense products around the layer boundary run as one kernel
+    (gemm2_tc in the kernel list, no gemm_tc), the sampled parity holds, and the pass without the vertex split is
+    timed beside it (the threshold is lowered so that this small graph has hubs to split)."""
+    d = run_bench("--workload", "large", "--scale", "0.002", "--threshold", "256", "--steps", "3", "--warmup", "3",
+                  "--cpu-seconds", "1", "--no-others")
+    assert d["rejected"] is False and d["problems"] == [] and d["dtype"] == "bf16"
+    names = {k["name"] for k in d["kernels"]}
+    assert "gemm2_tc" in names and "gemm_tc" not in names
+    assert d["parity"]["ok"] and d["parity"]["stored"]["max_rel"] <= 2e-2
+    assert d["split"]["split_owners"] > 0 and d["unsplit"]["ms_per_step"] > 0 and d["unsplit"]["value"] > 0
